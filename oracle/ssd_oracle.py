@@ -1,0 +1,258 @@
+"""CPU oracle for the Speech Speculative Decoding (SSD) verify step.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, float64 restatement of what one SSD verification step computes, written from the
+paper and used solely to check the CUDA path (tests, the smoke check, and the CPU-baseline leg of
+the benchmark).  It shares no code with the CUDA path and must never be imported by the product.
+
+What is computed, and from which passage:
+
+* `forward`      - the target model M_q run once over the pending token and the gamma draft
+                   tokens against the cached prefix, giving gamma+1 next-token distributions
+                   (Algorithm 1, the parallel-verification line; Eq. 4).  The decoder is the
+                   "Transformer adapted from Qwen2.5" of Sec. 3.1: pre-norm RMSNorm, grouped-query
+                   attention with biased q/k/v projections and rotate-half RoPE, SiLU-gated
+                   feed-forward, final RMSNorm, untied LM head.
+* `transform`    - temperature and top-k applied to a logit row before softmax.  The paper does
+                   not describe a sampler; this is the workload's (stated reading: z/T, keep the
+                   top_k largest with the lower id winning ties, softmax over what is kept).
+* `accept_step`  - the sequential tolerance test r_i < min(1, q_i(x_i)/p_i(x_i)) + beta (Eq. 5),
+                   the residual resample from normalize(max(0, q_i - p_i)) at the first rejection
+                   (Eq. 6), and the bonus token from q_{gamma+1} when nothing is rejected
+                   (Algorithm 1, last branch).  p is the DRAFT distribution and q the TARGET
+                   distribution, as in the paper (the reverse of the usual letters).
+* `commit`       - "append to T_in": the prefix grows by the accepted draft tokens plus the one
+                   corrected / bonus token (Algorithm 1).
+
+State convention: a stream holding n tokens keeps K/V for tokens 0..n-2 (`length` = n-1) and the
+last token as `pending`.  A verify step feeds [pending, x_1..x_gamma] at positions
+length..length+gamma, so row r predicts the token that follows x_r (row 0: the slot of x_1).
+
+Arithmetic is float64 throughout.  Storage formats are part of the problem, not of the
+arithmetic: weights arrive already rounded to the model's storage type, and K/V rows are rounded
+to the cache's storage type (bf16 or fp32) when they are appended.
+
+Pins (tests/test_oracle_*.py): forward vs gamma+1 sequential decodes; forward vs the
+`transformers` Qwen2 implementation and torch's scaled_dot_product_attention as black-box library
+routines; exact rational enumeration of the acceptance rule's output law (equal to q at beta = 0,
+and to the closed form for beta > 0); brute-force inverse CDF; monotonicity in beta; commit /
+rollback invariants.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest-even rounding of float64 values to bf16-representable values (via float32)."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(F64)
+
+
+class Model:
+    """Decoder weights (float32 arrays holding exact storage values) plus shape fields."""
+
+    def __init__(self, *, n_layers: int, d_model: int, n_q_heads: int, n_kv_heads: int,
+                 head_dim: int, d_ffn: int, vocab_out: int, vocab_text: int, rope_theta: float,
+                 rms_eps: float, kv_bf16: bool, weights: Dict[str, np.ndarray]):
+        self.L, self.d = n_layers, d_model
+        self.Hq, self.Hkv, self.hd = n_q_heads, n_kv_heads, head_dim
+        self.F, self.V, self.Vtext = d_ffn, vocab_out, vocab_text
+        self.theta, self.eps = float(rope_theta), float(rms_eps)
+        self.kv_bf16 = bool(kv_bf16)
+        self.w = weights
+
+
+class Stream:
+    """One utterance's state: cached K/V per layer, committed length, pending token."""
+
+    def __init__(self, model: Model, capacity: int):
+        self.K = [np.zeros((capacity, model.Hkv, model.hd), F64) for _ in range(model.L)]
+        self.V = [np.zeros((capacity, model.Hkv, model.hd), F64) for _ in range(model.L)]
+        self.capacity = capacity
+        self.length = 0          # tokens whose K/V are committed
+        self.pending = -1        # last token of T_in, not yet run through the model
+
+
+# ------------------------------------------------------------------ decoder pieces (Sec. 3.1)
+
+def rms_norm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain, row-wise."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain.astype(F64)
+
+
+def rope(x: np.ndarray, positions: np.ndarray, theta: float) -> np.ndarray:
+    """Rotate-half rotary embedding.  x: [rows, heads, hd]; positions: [rows] absolute."""
+    hd = x.shape[-1]
+    half = hd // 2
+    inv_freq = theta ** (-np.arange(half, dtype=F64) * 2.0 / hd)
+    ang = positions.astype(F64)[:, None] * inv_freq[None, :]          # [rows, half]
+    cos, sin = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * cos - x2 * sin, x2 * cos + x1 * sin], axis=-1)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def attention_rows(q: np.ndarray, K: np.ndarray, V: np.ndarray, first_pos: int) -> np.ndarray:
+    """Causal grouped-query attention of new rows against a cache that already contains them.
+
+    q: [R, Hq, hd] (row r sits at absolute position first_pos + r);
+    K, V: [>= first_pos + R, Hkv, hd].  Row r attends to keys 0..first_pos + r.
+    """
+    R, Hq, hd = q.shape
+    group = Hq // K.shape[1]
+    out = np.zeros((R, Hq, hd), F64)
+    for r in range(R):
+        n_keys = first_pos + r + 1
+        for h in range(Hq):
+            g = h // group
+            s = K[:n_keys, g, :] @ q[r, h, :] / np.sqrt(hd)
+            s = np.exp(s - s.max())
+            out[r, h, :] = (s / s.sum()) @ V[:n_keys, g, :]
+    return out
+
+
+def forward(model: Model, stream: Stream, ids: np.ndarray) -> np.ndarray:
+    """Run `ids` through M_q at positions stream.length.., appending their K/V (Eq. 4).
+
+    Returns logits [len(ids), V] in float64.  stream.length is NOT advanced: the appended rows
+    stay provisional until `commit` (or a prefill) moves the length.
+    """
+    w, m = model.w, model
+    ids = np.asarray(ids, dtype=np.int64)
+    R, p0 = len(ids), stream.length
+    assert p0 + R <= stream.capacity, "KV cache overflow"
+    pos = p0 + np.arange(R)
+    h = w["embed"][ids].astype(F64)
+    for l in range(m.L):
+        pre = f"l{l}."
+        xn = rms_norm(h, w[pre + "norm1"], m.eps)
+        q = (xn @ w[pre + "wq"].T.astype(F64) + w[pre + "bq"]).reshape(R, m.Hq, m.hd)
+        k = (xn @ w[pre + "wk"].T.astype(F64) + w[pre + "bk"]).reshape(R, m.Hkv, m.hd)
+        v = (xn @ w[pre + "wv"].T.astype(F64) + w[pre + "bv"]).reshape(R, m.Hkv, m.hd)
+        q, k = rope(q, pos, m.theta), rope(k, pos, m.theta)
+        if m.kv_bf16:
+            k, v = _round_to_bf16(k), _round_to_bf16(v)
+        else:
+            k, v = k.astype(np.float32).astype(F64), v.astype(np.float32).astype(F64)
+        stream.K[l][p0:p0 + R] = k
+        stream.V[l][p0:p0 + R] = v
+        att = attention_rows(q, stream.K[l], stream.V[l], p0).reshape(R, m.Hq * m.hd)
+        h = h + att @ w[pre + "wo"].T.astype(F64)
+        xn = rms_norm(h, w[pre + "norm2"], m.eps)
+        gate = xn @ w[pre + "wg"].T.astype(F64)
+        up = xn @ w[pre + "wu"].T.astype(F64)
+        h = h + (silu(gate) * up) @ w[pre + "wd"].T.astype(F64)
+    xn = rms_norm(h, w["norm_f"], m.eps)
+    return xn @ w["head"].T.astype(F64)
+
+
+def prefill(model: Model, stream: Stream, ids: np.ndarray, chunk: int = 64) -> None:
+    """Load a prefix T_in: K/V for all but the last id, which becomes the pending token."""
+    ids = np.asarray(ids, dtype=np.int64)
+    assert stream.length == 0 and len(ids) >= 1
+    for s in range(0, len(ids) - 1, chunk):
+        part = ids[s:min(s + chunk, len(ids) - 1)]
+        forward(model, stream, part)
+        stream.length += len(part)
+    stream.pending = int(ids[-1])
+
+
+# ------------------------------------------------------------------ sampling transform
+
+def transform(logits_row: np.ndarray, temperature: float, top_k: int) -> np.ndarray:
+    """Logit row -> the distribution the target's sampler draws from (q_i in Eq. 5-6)."""
+    z = np.asarray(logits_row, F64) / float(temperature)
+    V = z.shape[0]
+    if 0 < top_k < V:
+        order = np.argsort(-z, kind="stable")        # equal values: lower id first
+        keep = np.zeros(V, dtype=bool)
+        keep[order[:top_k]] = True
+    else:
+        keep = np.ones(V, dtype=bool)
+    e = np.where(keep, np.exp(z - z[keep].max()), 0.0)
+    return e / e.sum()
+
+
+# ------------------------------------------------------------------ acceptance (Eq. 5, 6)
+
+def categorical_draw(weights: np.ndarray, u: float) -> Tuple[int, float]:
+    """Inverse-CDF draw in ascending id: smallest t with sum_{s<=t} w_s > u * sum(w).
+
+    Also returns the draw's margin: the distance from u to the nearer CDF edge of the chosen
+    id, in units of total mass (used by parity tests to skip knife-edge draws).
+    """
+    cdf = np.cumsum(weights.astype(F64))
+    total = cdf[-1]
+    target = float(u) * total
+    t = int(np.searchsorted(cdf, target, side="right"))
+    t = min(t, len(cdf) - 1)
+    while t > 0 and weights[t] <= 0.0:       # never land on a zero-mass id
+        t -= 1
+    lo = cdf[t - 1] if t > 0 else 0.0
+    margin = min(target - lo, cdf[t] - target) / total
+    return t, float(margin)
+
+
+def accept_step(q_rows: np.ndarray, p_rows: np.ndarray, draft_tokens: np.ndarray,
+                uniforms: np.ndarray, beta: float) -> Dict[str, object]:
+    """Algorithm 1's inner loop for one stream.
+
+    q_rows [gamma+1, V] target distributions, p_rows [gamma, V] draft distributions,
+    draft_tokens [gamma], uniforms [gamma+1, 2] with [:, 0] = r_i and [:, 1] = the draw's u.
+    Returns accepted length k, the one new token y, and diagnostics (thresholds a_i, margins).
+    """
+    gamma = len(draft_tokens)
+    thresholds: List[float] = []
+    k = gamma
+    for i in range(gamma):
+        x = int(draft_tokens[i])
+        qi, pi = float(q_rows[i][x]), float(p_rows[i][x])
+        ratio = 1.0 if pi <= qi else qi / pi           # min(1, q/p) without dividing by zero
+        a = ratio + float(beta)
+        thresholds.append(a)
+        if float(uniforms[i][0]) < a:
+            continue                                    # accept x_i
+        k = i
+        break
+    if k < gamma:                                       # first rejection at position k+1
+        resid = np.maximum(0.0, q_rows[k].astype(F64) - p_rows[k].astype(F64))
+        if resid.sum() <= 0.0:                          # numerical corner: fall back to q
+            resid = q_rows[k].astype(F64)
+        y, margin = categorical_draw(resid, float(uniforms[k][1]))
+    else:                                               # all accepted: bonus from q_{gamma+1}
+        y, margin = categorical_draw(q_rows[gamma].astype(F64), float(uniforms[gamma][1]))
+    return {"k": k, "y": y, "thresholds": thresholds, "draw_margin": margin}
+
+
+def verify(model: Model, stream: Stream, draft_tokens: np.ndarray, p_rows: np.ndarray,
+           uniforms: np.ndarray, *, temperature: float, top_k: int, beta: float
+           ) -> Dict[str, object]:
+    """One full verification step for one stream (forward, transform, accept); no commit."""
+    ids = np.concatenate([[stream.pending], np.asarray(draft_tokens, np.int64)])
+    logits = forward(model, stream, ids)
+    q_rows = np.stack([transform(row, temperature, top_k) for row in logits])
+    res = accept_step(q_rows, p_rows, draft_tokens, uniforms, beta)
+    res["logits"] = logits
+    res["q_rows"] = q_rows
+    return res
+
+
+def commit(stream: Stream, k: int, y: int) -> None:
+    """T_in grows by the k accepted draft tokens and the new token y (Algorithm 1)."""
+    stream.length += 1 + int(k)
+    stream.pending = int(y)
+
+
+def truncate(stream: Stream, new_length: int, pending: int) -> None:
+    """Roll the stream back to an earlier prefix; later cache rows become dead."""
+    assert 0 <= new_length <= stream.length
+    stream.length, stream.pending = int(new_length), int(pending)

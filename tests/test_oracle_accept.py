@@ -1,0 +1,239 @@
+"""Pins for the oracle's acceptance rule, residual resample, bonus draw and sampling transform.
+
+The paper prints no numeric example of Eq. 5-6, so these pins are what the mathematics fixes:
+exact rational enumeration of the output law on tiny vocabularies (it equals the target
+distribution q at beta = 0, the claim that follows Eq. 6, and a closed form for beta > 0),
+brute-force inverse CDF, special cases and monotonicity in beta.
+"""
+from fractions import Fraction as Fr
+from itertools import product
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssd_oracle as orc
+from paper_2505_15380_b200 import synth
+
+N = 64                                   # grid: midpoints (j + 1/2) / N, exact for dyadic laws
+GRID = [(j + 0.5) / N for j in range(N)]
+
+
+def _law_one_position(p, q, q_bonus, beta):
+    """Exact law of (k, y) for gamma = 1 by enumerating x_1 ~ p and grids of r_1, u."""
+    V = len(p)
+    law = {}
+    for x in range(V):
+        if p[x] == 0:
+            continue
+        for r in GRID:
+            # the draw used is u_1 on rejection, u_2 on acceptance; enumerate one grid for it
+            for u in GRID:
+                uni = np.array([[r, u], [0.0, u]])
+                res = orc.accept_step(np.array([q, q_bonus], float), np.array([p], float),
+                                      np.array([x]), uni, beta)
+                key = (res["k"], res["y"])
+                law[key] = law.get(key, Fr(0)) + Fr(p[x]).limit_denominator(1 << 20) / (N * N)
+    return law
+
+
+def test_beta_zero_output_law_equals_target_exactly():
+    p = [4 / 8, 2 / 8, 1 / 8, 1 / 8]
+    q = [1 / 8, 1 / 8, 2 / 8, 4 / 8]
+    qb = [2 / 8, 2 / 8, 2 / 8, 2 / 8]
+    law = _law_one_position(p, q, qb, 0.0)
+    # accepted mass per draft token is p(x) * min(1, q/p) = min(p, q); recover it from the law
+    acc_total = sum(v for (k, _), v in law.items() if k == 1)
+    assert acc_total == sum(Fr(min(a, b)).limit_denominator(64) for a, b in zip(p, q))
+    rej = {y: v for (k, y), v in law.items() if k == 0}
+    # residual law: max(0, q - p) / sum  = [0, 0, 1/4, 3/4]; rejected mass = 1 - sum(min(p,q))
+    rej_mass = 1 - acc_total
+    assert rej == {2: rej_mass * Fr(1, 4), 3: rej_mass * Fr(3, 4)}
+    # overall first-token law: min(p,q)(x) + rej_mass * resid(x) == q(x), exactly
+    for x in range(4):
+        out = Fr(min(p[x], q[x])).limit_denominator(64) + rej.get(x, Fr(0))
+        assert out == Fr(q[x]).limit_denominator(64)
+    # bonus token after an acceptance follows q_{gamma+1} exactly
+    bonus = [sum(v for (k, y), v in law.items() if k == 1 and y == t) for t in range(4)]
+    assert bonus == [acc_total * Fr(1, 4)] * 4
+
+
+@pytest.mark.parametrize("beta", [0.25, 0.5])
+def test_beta_positive_output_law_matches_closed_form(beta):
+    p = [4 / 8, 2 / 8, 1 / 8, 1 / 8]
+    q = [1 / 8, 1 / 8, 2 / 8, 4 / 8]
+    qb = [1 / 8, 3 / 8, 2 / 8, 2 / 8]
+    law = _law_one_position(p, q, qb, beta)
+    A = [min(1.0, min(1.0, q[x] / p[x]) + beta) for x in range(4)]      # P(accept | x)
+    acc = sum(Fr(p[x] * A[x]).limit_denominator(1 << 12) for x in range(4))
+    assert sum(v for (k, _), v in law.items() if k == 1) == acc
+    w = [max(0.0, q[x] - p[x]) for x in range(4)]
+    for y in range(4):
+        want = (1 - acc) * Fr(w[y] / sum(w)).limit_denominator(64)
+        assert law.get((0, y), Fr(0)) == want
+
+
+def test_two_positions_sequence_law_is_target_ar_law():
+    """gamma = 2 with position-dependent targets: emitted tokens follow the target's chain."""
+    V = 2
+    p1, q1 = [1 / 2, 1 / 2], [1 / 4, 3 / 4]          # ratios 1/2 and 1: exact on the grid
+    p2 = {0: [1 / 2, 1 / 2], 1: [1 / 2, 1 / 2]}          # draft row 2 given x_1
+    q2 = {0: [1 / 4, 3 / 4], 1: [3 / 4, 1 / 4]}          # target row 2 given x_1
+    q3 = [1 / 2, 1 / 2]
+    n = 16
+    grid = [(j + 0.5) / n for j in range(n)]
+    seq_law = {}
+    for x1, x2 in product(range(V), range(V)):
+        w_draft = Fr(p1[x1]).limit_denominator(8) * Fr(p2[x1][x2]).limit_denominator(8)
+        for r1, r2, u in product(grid, grid, grid):
+            uni = np.array([[r1, u], [r2, u], [0.0, u]])
+            res = orc.accept_step(np.array([q1, q2[x1], q3]), np.array([p1, p2[x1]]),
+                                  np.array([x1, x2]), uni, 0.0)
+            emitted = tuple([x1, x2][:res["k"]]) + (res["y"],)
+            seq_law[emitted] = seq_law.get(emitted, Fr(0)) + w_draft / n ** 3
+    assert sum(seq_law.values()) == 1
+    first = [sum(v for s, v in seq_law.items() if s[0] == t) for t in range(V)]
+    assert first == [Fr(1, 4), Fr(3, 4)]                              # = q1
+    # given x_1 = a was accepted (sequence has >= 2 tokens), the second token follows q2[a]
+    for a in range(V):
+        mass = sum(v for s, v in seq_law.items() if len(s) >= 2 and s[0] == a)
+        for b in range(V):
+            got = sum(v for s, v in seq_law.items() if len(s) >= 2 and s[:2] == (a, b))
+            assert got == mass * Fr(q2[a][b]).limit_denominator(8)
+    # three tokens only when both drafts were accepted; the third follows q3
+    m3 = sum(v for s, v in seq_law.items() if len(s) == 3)
+    assert sum(v for s, v in seq_law.items() if len(s) == 3 and s[2] == 0) == m3 * Fr(1, 2)
+
+
+def test_control_flow_properties_random():
+    rng = np.random.default_rng(0)
+    V, gamma = 11, 4
+    for trial in range(300):
+        q = rng.dirichlet(np.ones(V), size=gamma + 1)
+        p = rng.dirichlet(np.ones(V), size=gamma)
+        x = np.array([rng.choice(V, p=p[i]) for i in range(gamma)])
+        uni = rng.random((gamma + 1, 2))
+        prev_k = -1
+        for beta in [0.0, 0.1, 0.4, 1.0]:
+            res = orc.accept_step(q, p, x, uni, beta)
+            k, y = res["k"], res["y"]
+            assert 0 <= k <= gamma and 0 <= y < V
+            assert k >= prev_k                       # larger beta never accepts fewer
+            prev_k = k
+            th = res["thresholds"]
+            assert all(uni[i, 0] < th[i] for i in range(k))
+            if k < gamma:
+                assert uni[k, 0] >= th[k]
+                resid = np.maximum(0, q[k] - p[k])
+                assert resid[y] > 0                  # resampled token has residual mass
+                assert y != x[k]                     # a rejected token has q < p: no residual
+            else:
+                assert q[gamma][y] > 0
+        assert prev_k == gamma                       # beta >= 1 accepts everything (r < 1)
+
+
+def test_identical_distributions_always_accept():
+    rng = np.random.default_rng(1)
+    q = rng.dirichlet(np.ones(7), size=4)
+    x = np.array([2, 5, 0])
+    res = orc.accept_step(q, q[:3].copy(), x, rng.random((4, 2)) * 0.999999, 0.0)
+    assert res["k"] == 3
+
+
+def test_zero_draft_probability_does_not_divide():
+    q = np.array([[0.5, 0.5], [0.5, 0.5]])
+    p = np.array([[0.0, 1.0]])
+    res = orc.accept_step(q, p, np.array([0]), np.array([[0.99, 0.3], [0.0, 0.3]]), 0.0)
+    assert res["k"] == 1 and res["thresholds"][0] == 1.0
+
+
+def test_zero_residual_falls_back_to_target_row():
+    q = np.array([[0.25, 0.75], [0.5, 0.5]])
+    p = q[:1].copy()                                  # p == q: residual is identically zero
+    # force a "rejection" with r >= 1 (not reachable with r in [0,1), exercised directly)
+    res = orc.accept_step(q, p, np.array([1]), np.array([[1.5, 0.1], [0.0, 0.0]]), 0.0)
+    assert res["k"] == 0 and res["y"] == 0            # u = 0.1 < 0.25 -> id 0 of q itself
+
+
+def test_categorical_draw_brute_force():
+    rng = np.random.default_rng(2)
+    for _ in range(200):
+        V = int(rng.integers(1, 9))
+        w = rng.random(V) * (rng.random(V) > 0.3)
+        if w.sum() == 0:
+            w[rng.integers(V)] = 1.0
+        u = float(rng.random())
+        acc, want = 0.0, None
+        for t in range(V):                            # definition: first id whose CDF exceeds u*S
+            acc += w[t]
+            if acc > u * w.sum():
+                want = t
+                break
+        got, margin = orc.categorical_draw(w, u)
+        assert got == want and w[got] > 0 and margin >= 0
+
+
+def test_categorical_draw_frequencies():
+    w = np.array([1.0, 0.0, 3.0, 4.0])
+    counts = np.zeros(4)
+    n = 8000
+    for j in range(n):
+        counts[orc.categorical_draw(w, (j + 0.5) / n)[0]] += 1
+    assert np.array_equal(counts, [1000, 0, 3000, 4000])
+
+
+def test_transform_against_torch_and_special_cases():
+    rng = np.random.default_rng(3)
+    z = rng.standard_normal(50) * 3
+    q = orc.transform(z, 0.8, 0)
+    ref = torch.softmax(torch.from_numpy(z) / 0.8, dim=0).numpy()
+    assert np.allclose(q, ref, atol=1e-15)
+    assert np.allclose(orc.transform(z, 0.8, 50), q) and np.allclose(orc.transform(z, 0.8, 500), q)
+    qk = orc.transform(z, 0.8, 5)
+    top = torch.topk(torch.from_numpy(z), 5)
+    assert set(np.nonzero(qk)[0]) == set(top.indices.tolist())
+    assert np.isclose(qk.sum(), 1.0)
+    ref_k = torch.softmax(top.values / 0.8, dim=0).numpy()
+    assert np.allclose(qk[top.indices.numpy()], ref_k, atol=1e-15)
+    # ties at the cut: the lower id is kept
+    zt = np.array([1.0, 5.0, 5.0, 5.0, 0.0])
+    assert list(np.nonzero(orc.transform(zt, 1.0, 2))[0]) == [1, 2]
+    # shift invariance and temperature -> argmax
+    assert np.allclose(orc.transform(z + 100.0, 1.0, 0), orc.transform(z, 1.0, 0))
+    assert orc.transform(z, 1e-3, 0).argmax() == z.argmax()
+
+
+def test_expected_tokens_per_iteration_geometric_identity():
+    """With i.i.d. acceptance probability alpha, E[k+1] = (1 - alpha^(gamma+1)) / (1 - alpha)."""
+    V, gamma, alpha = 4, 4, 0.5
+    p = np.tile(np.array([0.5, 0.5, 0.0, 0.0]), (gamma, 1))
+    q = np.tile(np.array([0.25, 0.25, 0.25, 0.25]), (gamma + 1, 1))      # q/p = 1/2 on support
+    uni = synth.verify_uniforms(7, 4000, gamma + 1).astype(np.float64)
+    tot = 0
+    for b in range(4000):
+        tot += orc.accept_step(q, p, np.zeros(gamma, int), uni[b], 0.0)["k"] + 1
+    want = (1 - alpha ** (gamma + 1)) / (1 - alpha)
+    assert abs(tot / 4000 - want) < 0.06
+
+
+def test_verify_wires_rows_to_positions():
+    """Row i of the forward is tested against draft token i+1 (a shifted index must fail)."""
+    from tests.helpers import oracle_model, small_shape
+    shape = small_shape()
+    w = synth.make_weights(shape, 4)
+    m = oracle_model(shape, w)
+    st = orc.Stream(m, 32)
+    orc.prefill(m, st, np.arange(9) % shape.vocab_in)
+    draft = np.array([3, 7, 11])
+    logits = orc.forward(m, st, np.concatenate([[st.pending], draft]))
+    q_rows = np.stack([orc.transform(r, 1.0, 0) for r in logits])
+    p_rows = q_rows[:3].copy().astype(np.float32)                 # p == q: must accept all
+    res = orc.verify(m, st, draft, p_rows, np.full((4, 2), 0.999), temperature=1.0, top_k=0,
+                     beta=0.0)
+    assert res["k"] == 3
+    p_bad = np.roll(q_rows[:3], 1, axis=0).astype(np.float32)     # mis-indexed rows
+    p_bad[:, draft] *= 50.0
+    res2 = orc.verify(m, st, draft, p_bad, np.full((4, 2), 0.999), temperature=1.0, top_k=0,
+                      beta=0.0)
+    assert res2["k"] < 3
+    assert np.allclose(res["logits"], logits)
