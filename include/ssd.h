@@ -1,0 +1,189 @@
+/*
+ * ssd.h - C ABI of the B200 (sm_100a) verify step of Speech Speculative Decoding (SSD).
+ *
+ * One SSD iteration (Algorithm 1) drafts gamma speech tokens with a small model M_p, runs the
+ * target model M_q once over them ("parallel verification", Eq. 4), accepts a prefix of the
+ * draft with the tolerance test r_i < min(1, q_i(x_i)/p_i(x_i)) + beta (Eq. 5), and emits one
+ * more token: a resample from normalize(max(0, q_i - p_i)) at the first rejection (Eq. 6) or a
+ * bonus token from q_{gamma+1} when nothing was rejected.  This library is that hot path.
+ * Letters follow the paper: p = DRAFT distribution, q = TARGET distribution.
+ *
+ * Conventions for every call
+ *  - Pointers named dev_* are device pointers, host_* are host pointers.  `stream` is a
+ *    cudaStream_t passed as void* (NULL = the legacy default stream).
+ *  - All device memory (weights arena, KV cache, workspace, inputs, outputs) is allocated and
+ *    owned by the caller; handles returned by *_create are small host objects freed by *_destroy.
+ *    The library never frees or reallocates caller memory and keeps the pointers it was given
+ *    until the handle is destroyed.
+ *  - Calls that take a stream only enqueue work on it and return without synchronising, unless
+ *    stated otherwise.  Inputs are read-only.
+ *  - Return value: SSD_OK (0) or a negative SSD_ERR_* code; nothing is enqueued on error.
+ *    Conditions only the device can see (cache overflow, bad token id, non-finite logits) set
+ *    bits of a device status word read back by ssd_last_status; kernels always terminate and
+ *    never touch memory outside the buffers they were given.
+ *
+ * Stream state: a stream (utterance) whose prefix T_in has n tokens keeps K/V for tokens
+ * 0..n-2 (`len` = n-1) and token n-1 as `pending`.  ssd_verify feeds [pending, x_1..x_gamma] at
+ * positions len..len+gamma and writes their K/V; ssd_kv_commit makes k+1 of them permanent.
+ * Rolling back rejected positions is O(1): slots at or beyond `len` are dead and get
+ * overwritten by the next step.
+ *
+ * KV cache layout (caller-owned buffer of ssd_kv_bytes bytes), storage type = weight_dtype:
+ *     kv[layer][stream][2 (0 = K, 1 = V)][kv_head][capacity][head_dim]
+ * K is stored after the rotary embedding.
+ */
+#ifndef SSD_H_
+#define SSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ssd_model ssd_model;     /* packed weights of one decoder (target or draft) */
+typedef struct ssd_streams ssd_streams; /* B streams' KV cache descriptors, len[], pending[] */
+
+enum {
+  SSD_OK = 0,
+  SSD_ERR_NULL = -1,        /* a required pointer was NULL */
+  SSD_ERR_BAD_CONFIG = -2,  /* unsupported or inconsistent model / stream configuration */
+  SSD_ERR_BAD_GAMMA = -3,   /* gamma outside 1..max_gamma given at ssd_streams_create */
+  SSD_ERR_KV_OVERFLOW = -4, /* a length would exceed the cache capacity */
+  SSD_ERR_MISALIGNED = -5,  /* a buffer is not aligned as required (256 bytes for arenas) */
+  SSD_ERR_TOO_SMALL = -6,   /* a caller buffer is smaller than the *_bytes call reports */
+  SSD_ERR_CUDA = -7,        /* a CUDA runtime call failed; see ssd_last_cuda_error */
+  SSD_ERR_BAD_PARAM = -8    /* temperature <= 0, beta < 0, n_in out of range, ... */
+};
+
+/* bits of the device status word (ssd_last_status) */
+enum {
+  SSD_STATUS_KV_OVERFLOW = 1, /* len + rows > capacity: rows beyond capacity were not written */
+  SSD_STATUS_BAD_TOKEN = 2,   /* a token id outside the embedding table was clamped */
+  SSD_STATUS_NONFINITE = 4,   /* a logit row held NaN/Inf */
+  SSD_STATUS_BAD_PROB = 8     /* a draft probability p_i(x_i) was negative or not finite */
+};
+
+/* Decoder shape: the "Transformer adapted from Qwen2.5" of Sec. 3.1 (pre-norm RMSNorm, GQA with
+ * biased q/k/v projections, rotate-half RoPE, SiLU-gated FFN, final RMSNorm, untied head). */
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn;
+  int32_t vocab_out;    /* speech vocabulary = rows of the LM head */
+  int32_t vocab_text;   /* extra embedding rows [vocab_out, vocab_out + vocab_text) for text ids */
+  float rope_theta, rms_eps;
+  int32_t weight_dtype; /* 0 = fp32, 1 = bf16; the KV cache uses the same type */
+  int32_t qkv_bias;     /* must be 1 (the blob always carries q/k/v biases) */
+} ssd_model_config;
+
+/* Per-call parameters of the sampler and of the acceptance rule. */
+typedef struct {
+  int32_t gamma;     /* draft length L_d of Algorithm 1 */
+  float temperature; /* > 0; logits are divided by it */
+  int32_t top_k;     /* <= 0 or >= vocab_out: off; else keep the top_k largest (lower id wins ties) */
+  float beta;        /* tolerance factor of Eq. 5, >= 0 */
+} ssd_verify_params;
+
+/* ---- model ------------------------------------------------------------------------------- */
+
+/* Bytes of device memory the packed model needs (0 if cfg is invalid). */
+size_t ssd_model_arena_bytes(const ssd_model_config* cfg);
+
+/* Packs a model into dev_arena (256-byte aligned, >= ssd_model_arena_bytes) and returns a handle.
+ * host_weights is a flat blob of nbytes in this order, every element in weight_dtype:
+ *   embed[vocab_out+vocab_text, d];
+ *   per layer: norm1[d], wq[Hq*hd, d], bq[Hq*hd], wk[Hkv*hd, d], bk, wv[Hkv*hd, d], bv,
+ *              wo[d, Hq*hd], norm2[d], w_gate[F, d], w_up[F, d], w_down[d, F];
+ *   norm_f[d]; head[vocab_out, d].            (all matrices row-major [out, in])
+ * Synchronous: returns after the copies finished; the blob may be freed afterwards. */
+int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size_t nbytes,
+                     void* dev_arena, size_t arena_bytes, ssd_model** out);
+void ssd_model_destroy(ssd_model* m);
+
+/* ---- streams ----------------------------------------------------------------------------- */
+
+size_t ssd_kv_bytes(const ssd_model_config* cfg, int32_t batch, int32_t capacity_tokens);
+size_t ssd_workspace_bytes(const ssd_model_config* cfg, int32_t batch, int32_t max_gamma,
+                           int32_t capacity_tokens);
+
+/* Binds `batch` streams of `capacity_tokens` cache slots each to caller buffers dev_kv and
+ * dev_workspace (both 256-byte aligned).  The workspace holds len[], pending[], the status word
+ * and all scratch of the kernels; it is zeroed here (synchronously), the KV buffer is not. */
+int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_tokens,
+                       int32_t max_gamma, void* dev_kv, size_t kv_bytes, void* dev_workspace,
+                       size_t ws_bytes, ssd_streams** out);
+void ssd_streams_destroy(ssd_streams* s);
+
+/* Explicit rollback / state load: len[b] = host_len[b], pending[b] = host_pending[b].
+ * O(1) per stream, no cache data moves.  Synchronous with respect to `stream`. */
+int ssd_kv_truncate(ssd_streams* s, const int32_t* host_len, const int32_t* host_pending,
+                    void* stream);
+/* Same rollback with DEVICE arrays (int32 [B] each), enqueued on `stream` without synchronising:
+ * the form a serving loop uses to discard a step or to re-run one from a saved state. */
+int ssd_kv_restore(ssd_streams* s, const int32_t* dev_len, const int32_t* dev_pending, void* stream);
+/* Reads len[] and pending[] back (either output may be NULL).  Synchronises `stream`. */
+int ssd_streams_get_state(ssd_streams* s, int32_t* host_len, int32_t* host_pending, void* stream);
+
+/* Loads prefixes T_in through the model: stream b receives ids dev_ids[host_offsets[b] ..
+ * host_offsets[b+1]) (>= 1 id each), appended after its current len.  K/V are written for all
+ * but the last id, which becomes `pending`.  Enqueues work only. */
+int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int32_t* host_offsets,
+                void* stream);
+
+/* ---- the SSD iteration ------------------------------------------------------------------- */
+
+/* Draft generation (Algorithm 1, the lines that produce p_i and x_i ~ p_i; Eq. 2-3), one
+ * autoregressive step of the draft model for every stream: feeds n_in (1 or 2) tokens
+ * dev_in_ids[b, 0..n_in) at positions len[b].., commits them (len += n_in), applies the
+ * sampling transform to the last row's logits and draws x ~ p with dev_uniform[b].
+ * n_in = 2 serves the step after a fully accepted iteration, when the draft has no K/V yet for
+ * x_gamma.  Outputs: dev_out_token[b], and the full row p (float [B, vocab_out]) the token was
+ * drawn from, as Eq. 5-6 need it.  `pending` of the draft streams is set to the drawn token. */
+int ssd_draft_step(ssd_model* draft, ssd_streams* draft_streams, const int32_t* dev_in_ids,
+                   int32_t n_in, const float* dev_uniform, const ssd_verify_params* params,
+                   int32_t* dev_out_token, float* dev_out_prob_row, void* stream);
+
+/* Parallel verification and acceptance (Algorithm 1 from the M_q line to the bonus token;
+ * Eq. 4-6) for all B streams:
+ *   in  dev_draft_tokens int32 [B, gamma]       x_1..x_gamma
+ *       dev_draft_probs  float [B, gamma, V]    rows p_i the tokens were drawn from
+ *       dev_uniforms     float [B, gamma+1, 2]  [..,0] = r_i of Eq. 5 (row gamma unused),
+ *                                               [..,1] = uniform of the categorical draw made
+ *                                               at that row (resample at row i, bonus at gamma)
+ *   out dev_accepted_len int32 [B]   k in [0, gamma]: draft tokens accepted
+ *       dev_next_token   int32 [B]   the resampled (k < gamma) or bonus (k = gamma) token
+ *       dev_logits_or_null float [B, gamma+1, V]  raw target logits, for parity checks
+ * Writes provisional K/V at slots len..len+gamma; len/pending change only in ssd_kv_commit.
+ * All uniforms must lie in [0, 1). */
+int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens,
+               const float* dev_draft_probs, const float* dev_uniforms,
+               const ssd_verify_params* params, int32_t* dev_accepted_len,
+               int32_t* dev_next_token, float* dev_logits_or_null, void* stream);
+
+/* Same step with HOST buffers: copies the three inputs to the device, runs ssd_verify and
+ * ssd_kv_commit, copies accepted_len / next_token back and synchronises `stream`.  Host
+ * buffers should be pinned for the copies to be asynchronous. */
+int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft_tokens,
+                    const float* host_draft_probs, const float* host_uniforms,
+                    const ssd_verify_params* params, int32_t* host_accepted_len,
+                    int32_t* host_next_token, void* stream);
+
+/* "Append to T_in" (Algorithm 1): len[b] += 1 + accepted_len[b]; pending[b] = next_token[b].
+ * Rejected positions need no work: they lie beyond the new len. */
+int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
+                  void* stream);
+
+/* ---- diagnostics ------------------------------------------------------------------------- */
+
+/* Reads and clears the device status word (SSD_STATUS_* bits).  Synchronises `stream`. */
+int ssd_last_status(ssd_streams* s, int32_t* status, void* stream);
+/* Number of kernels this library has enqueued in this process so far (all handles). */
+uint64_t ssd_kernel_launch_count(void);
+/* Text of the last CUDA error seen by this library on this thread ("" if none). */
+const char* ssd_last_cuda_error(void);
+const char* ssd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSD_H_ */

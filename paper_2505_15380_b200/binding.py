@@ -1,0 +1,253 @@
+"""Thin ctypes binding over the C ABI declared in include/ssd.h.
+
+Argument marshalling only: every step of the verify path runs in the CUDA library.  torch is used
+for device memory and streams.  There is no CPU fallback: if the library is missing or no CUDA
+device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libssd_b200.so")
+_lib = None
+
+EXPORTS = [
+    "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
+    "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_kv_truncate",
+    "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
+    "ssd_kv_commit", "ssd_kv_restore", "ssd_kernel_launch_count", "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
+]
+
+
+class ModelConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn",
+                 "vocab_out", "vocab_text")] + \
+               [("rope_theta", ctypes.c_float), ("rms_eps", ctypes.c_float),
+                ("weight_dtype", ctypes.c_int32), ("qkv_bias", ctypes.c_int32)]
+
+
+class VerifyParams(ctypes.Structure):
+    _fields_ = [("gamma", ctypes.c_int32), ("temperature", ctypes.c_float),
+                ("top_k", ctypes.c_int32), ("beta", ctypes.c_float)]
+
+
+class SsdError(RuntimeError):
+    pass
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libssd_b200.so (built in-tree by `python -m paper_2505_15380_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise SsdError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_15380_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
+    cfgp, parp = ctypes.POINTER(ModelConfig), ctypes.POINTER(VerifyParams)
+    L.ssd_model_arena_bytes.restype = sz
+    L.ssd_model_arena_bytes.argtypes = [cfgp]
+    L.ssd_model_create.argtypes = [cfgp, vp, sz, vp, sz, ctypes.POINTER(vp)]
+    L.ssd_model_destroy.restype = None
+    L.ssd_model_destroy.argtypes = [vp]
+    L.ssd_kv_bytes.restype = sz
+    L.ssd_kv_bytes.argtypes = [cfgp, i32, i32]
+    L.ssd_workspace_bytes.restype = sz
+    L.ssd_workspace_bytes.argtypes = [cfgp, i32, i32, i32]
+    L.ssd_streams_create.argtypes = [vp, i32, i32, i32, vp, sz, vp, sz, ctypes.POINTER(vp)]
+    L.ssd_streams_destroy.restype = None
+    L.ssd_streams_destroy.argtypes = [vp]
+    L.ssd_kv_truncate.argtypes = [vp, vp, vp, vp]
+    L.ssd_streams_get_state.argtypes = [vp, vp, vp, vp]
+    L.ssd_prefill.argtypes = [vp, vp, vp, vp, vp]
+    L.ssd_draft_step.argtypes = [vp, vp, vp, i32, vp, parp, vp, vp, vp]
+    L.ssd_verify.argtypes = [vp, vp, vp, vp, vp, parp, vp, vp, vp, vp]
+    L.ssd_verify_host.argtypes = [vp, vp, vp, vp, vp, parp, vp, vp, vp]
+    L.ssd_kv_commit.argtypes = [vp, vp, vp, vp]
+    L.ssd_kv_restore.argtypes = [vp, vp, vp, vp]
+    L.ssd_kernel_launch_count.restype = ctypes.c_uint64
+    L.ssd_kernel_launch_count.argtypes = []
+    L.ssd_last_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    L.ssd_last_cuda_error.restype = ctypes.c_char_p
+    L.ssd_strerror.restype = ctypes.c_char_p
+    L.ssd_strerror.argtypes = [ctypes.c_int]
+    _lib = L
+    return L
+
+
+def check(rc: int) -> None:
+    if rc != 0:
+        L = lib()
+        msg = L.ssd_strerror(rc).decode()
+        detail = L.ssd_last_cuda_error().decode()
+        raise SsdError(f"ssd error {rc}: {msg}" + (f" ({detail})" if detail and rc == -7 else ""))
+
+
+def _require_cuda() -> None:
+    if not torch.cuda.is_available():
+        raise SsdError("no CUDA device: the SSD verify path has no CPU fallback")
+
+
+def make_config(shape) -> ModelConfig:
+    """ModelConfig from any object with the fields of synth.ModelShape."""
+    return ModelConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads,
+                       shape.head_dim, shape.d_ffn, shape.vocab_out, shape.vocab_text,
+                       shape.rope_theta, shape.rms_eps, shape.weight_dtype, shape.qkv_bias)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _alloc(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+class Model:
+    """ssd_model handle plus the torch tensor that owns its device arena."""
+
+    def __init__(self, shape, blob: np.ndarray, device="cuda:0"):
+        _require_cuda()
+        L = lib()
+        self.shape = shape
+        self.cfg = make_config(shape)
+        self.device = torch.device(device)
+        nbytes = L.ssd_model_arena_bytes(ctypes.byref(self.cfg))
+        if nbytes == 0:
+            raise SsdError("unsupported model configuration")
+        with torch.cuda.device(self.device):
+            self.arena = _alloc(nbytes, self.device)
+            blob = np.ascontiguousarray(blob)
+            h = ctypes.c_void_p()
+            check(L.ssd_model_create(ctypes.byref(self.cfg), blob.ctypes.data, blob.nbytes,
+                                     self.arena.data_ptr(), nbytes, ctypes.byref(h)))
+        self.handle = h
+
+    def __del__(self):
+        if getattr(self, "handle", None) is not None and _lib is not None:
+            _lib.ssd_model_destroy(self.handle)
+            self.handle = None
+
+
+class Streams:
+    """ssd_streams handle plus the torch tensors that own the KV cache and the workspace."""
+
+    def __init__(self, model: Model, batch: int, capacity: int, max_gamma: int):
+        L = lib()
+        self.model, self.B, self.capacity, self.max_gamma = model, batch, capacity, max_gamma
+        cfg = model.cfg
+        dev = model.device
+        kvb = L.ssd_kv_bytes(ctypes.byref(cfg), batch, capacity)
+        wsb = L.ssd_workspace_bytes(ctypes.byref(cfg), batch, max_gamma, capacity)
+        if kvb == 0 or wsb == 0:
+            raise SsdError("unsupported stream configuration")
+        with torch.cuda.device(dev):
+            self.kv_raw = _alloc(kvb, dev)
+            self.ws = _alloc(wsb, dev)
+            h = ctypes.c_void_p()
+            check(L.ssd_streams_create(model.handle, batch, capacity, max_gamma,
+                                       self.kv_raw.data_ptr(), kvb, self.ws.data_ptr(), wsb,
+                                       ctypes.byref(h)))
+        self.handle = h
+        s = model.shape
+        dt = torch.float32 if s.weight_dtype == 0 else torch.bfloat16
+        self.kv = self.kv_raw[:kvb].view(dt).view(s.n_layers, batch, 2, s.n_kv_heads, capacity,
+                                                  s.head_dim)
+
+    def __del__(self):
+        if getattr(self, "handle", None) is not None and _lib is not None:
+            _lib.ssd_streams_destroy(self.handle)
+            self.handle = None
+
+    # -- state ------------------------------------------------------------------------------
+    def kv_truncate(self, lens: Sequence[int], pending: Sequence[int], stream=None) -> None:
+        a = np.ascontiguousarray(lens, dtype=np.int32)
+        p = np.ascontiguousarray(pending, dtype=np.int32)
+        assert a.shape == (self.B,) and p.shape == (self.B,)
+        check(lib().ssd_kv_truncate(self.handle, a.ctypes.data, p.ctypes.data, _stream_ptr(stream)))
+
+    def kv_restore(self, dev_len: torch.Tensor, dev_pending: torch.Tensor, stream=None) -> None:
+        assert dev_len.dtype == torch.int32 and dev_pending.dtype == torch.int32
+        assert dev_len.is_cuda and dev_len.numel() == self.B and dev_pending.numel() == self.B
+        check(lib().ssd_kv_restore(self.handle, dev_len.data_ptr(), dev_pending.data_ptr(),
+                                   _stream_ptr(stream)))
+
+    def get_state(self, stream=None) -> Tuple[np.ndarray, np.ndarray]:
+        a = np.zeros(self.B, np.int32)
+        p = np.zeros(self.B, np.int32)
+        check(lib().ssd_streams_get_state(self.handle, a.ctypes.data, p.ctypes.data,
+                                          _stream_ptr(stream)))
+        return a, p
+
+    def last_status(self, stream=None) -> int:
+        v = ctypes.c_int32(0)
+        check(lib().ssd_last_status(self.handle, ctypes.byref(v), _stream_ptr(stream)))
+        return v.value
+
+    # -- the calls --------------------------------------------------------------------------
+    def prefill(self, prefixes: Sequence[np.ndarray], stream=None) -> None:
+        assert len(prefixes) == self.B
+        offs = np.zeros(self.B + 1, np.int32)
+        offs[1:] = np.cumsum([len(p) for p in prefixes])
+        ids = torch.from_numpy(np.concatenate(prefixes).astype(np.int32)).to(self.model.device)
+        check(lib().ssd_prefill(self.model.handle, self.handle, ids.data_ptr(), offs.ctypes.data,
+                                _stream_ptr(stream)))
+        torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+
+    def verify(self, draft_tokens: torch.Tensor, draft_probs: torch.Tensor,
+               uniforms: torch.Tensor, params: VerifyParams, accepted_len: torch.Tensor,
+               next_token: torch.Tensor, logits: Optional[torch.Tensor] = None,
+               stream=None) -> None:
+        g = params.gamma
+        assert draft_tokens.dtype == torch.int32 and draft_tokens.numel() == self.B * g
+        assert draft_probs.dtype == torch.float32 and \
+            draft_probs.numel() == self.B * g * self.model.shape.vocab_out
+        assert uniforms.dtype == torch.float32 and uniforms.numel() == self.B * (g + 1) * 2
+        assert accepted_len.dtype == torch.int32 and next_token.dtype == torch.int32
+        for t in (draft_tokens, draft_probs, uniforms, accepted_len, next_token):
+            assert t.is_cuda and t.is_contiguous()
+        if logits is not None:
+            assert logits.dtype == torch.float32 and logits.is_contiguous() and \
+                logits.numel() == self.B * (g + 1) * self.model.shape.vocab_out
+        check(lib().ssd_verify(self.model.handle, self.handle, draft_tokens.data_ptr(),
+                               draft_probs.data_ptr(), uniforms.data_ptr(), ctypes.byref(params),
+                               accepted_len.data_ptr(), next_token.data_ptr(), _ptr(logits),
+                               _stream_ptr(stream)))
+
+    def verify_host(self, draft_tokens: torch.Tensor, draft_probs: torch.Tensor,
+                    uniforms: torch.Tensor, params: VerifyParams, accepted_len: torch.Tensor,
+                    next_token: torch.Tensor, stream=None) -> None:
+        """Host-buffer variant (pinned CPU tensors); includes the commit and a stream sync."""
+        for t in (draft_tokens, draft_probs, uniforms, accepted_len, next_token):
+            assert not t.is_cuda and t.is_contiguous()
+        check(lib().ssd_verify_host(self.model.handle, self.handle, draft_tokens.data_ptr(),
+                                    draft_probs.data_ptr(), uniforms.data_ptr(),
+                                    ctypes.byref(params), accepted_len.data_ptr(),
+                                    next_token.data_ptr(), _stream_ptr(stream)))
+
+    def kv_commit(self, accepted_len: torch.Tensor, next_token: torch.Tensor, stream=None) -> None:
+        check(lib().ssd_kv_commit(self.handle, accepted_len.data_ptr(), next_token.data_ptr(),
+                                  _stream_ptr(stream)))
+
+    def draft_step(self, in_ids: torch.Tensor, n_in: int, uniform: torch.Tensor,
+                   params: VerifyParams, out_token: torch.Tensor, out_prob_row: torch.Tensor,
+                   stream=None) -> None:
+        assert in_ids.dtype == torch.int32 and in_ids.numel() == self.B * n_in
+        assert uniform.dtype == torch.float32 and uniform.numel() == self.B
+        assert out_prob_row.dtype == torch.float32 and \
+            out_prob_row.numel() == self.B * self.model.shape.vocab_out
+        check(lib().ssd_draft_step(self.model.handle, self.handle, in_ids.data_ptr(), n_in,
+                                   uniform.data_ptr(), ctypes.byref(params), out_token.data_ptr(),
+                                   out_prob_row.data_ptr(), _stream_ptr(stream)))

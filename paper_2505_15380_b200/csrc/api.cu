@@ -1,0 +1,487 @@
+// C ABI of the SSD verify library: handles, argument checks, and the launch sequence of one
+// decoder forward (Sec. 3.1 decoder; Eq. 4) followed by the acceptance kernel (Eq. 5-6).
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "kernels.h"
+
+using namespace ssd;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%.120s: %.120s", what, cudaGetErrorString(e));
+  return SSD_ERR_CUDA;
+}
+#define SSD_CUDA(call)                                  \
+  do {                                                  \
+    cudaError_t e_ = (call);                            \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+bool cfg_ok(const ssd_model_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  if (c->n_q_heads / c->n_kv_heads > 16) return false;
+  if ((c->d_model & 7) || (c->d_ffn & 7) || c->d_ffn < 8) return false;
+  if (c->vocab_out < 2 || c->vocab_text < 0) return false;
+  if ((size_t)c->vocab_out * 4 > 180 * 1024) return false;  // a logit row must fit in shared memory
+  if (c->weight_dtype != 0 && c->weight_dtype != 1) return false;
+  if (c->qkv_bias != 1) return false;
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return false;
+  return true;
+}
+
+struct LayerOff {
+  size_t norm1, w_qkv, b_qkv, w_o, norm2, w_gu, w_d;
+};
+struct ArenaPlan {
+  size_t embed, norm_f, head, inv_freq, total;
+  std::vector<LayerOff> layers;
+};
+
+ArenaPlan plan_arena(const ssd_model_config& c) {
+  ArenaPlan p;
+  size_t el = c.weight_dtype == 0 ? 4 : 2, off = 0;
+  size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+  size_t F = c.d_ffn;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  p.embed = take((size_t)(c.vocab_out + c.vocab_text) * d * el);
+  p.layers.resize(c.n_layers);
+  for (auto& L : p.layers) {
+    L.norm1 = take(d * el);
+    L.w_qkv = take((qd + 2 * kvd) * d * el);
+    L.b_qkv = take((qd + 2 * kvd) * el);
+    L.w_o = take(d * qd * el);
+    L.norm2 = take(d * el);
+    L.w_gu = take(2 * F * d * el);
+    L.w_d = take(d * F * el);
+  }
+  p.norm_f = take(d * el);
+  p.head = take((size_t)c.vocab_out * d * el);
+  p.inv_freq = take((size_t)(c.head_dim / 2) * sizeof(double));
+  p.total = off;
+  return p;
+}
+
+size_t blob_elems(const ssd_model_config& c) {
+  size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+  size_t F = c.d_ffn;
+  size_t per_layer = d + qd * d + qd + 2 * (kvd * d + kvd) + d * qd + d + 3 * F * d;
+  return (size_t)(c.vocab_out + c.vocab_text) * d + per_layer * c.n_layers + d + (size_t)c.vocab_out * d;
+}
+
+struct WsPlan {
+  size_t len, pending, status, counters, row_ids, accept_flags;
+  size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
+  size_t st_tokens, st_k, st_y, st_probs, st_uni;
+  size_t total;
+  int max_rows, nsplit_max;
+};
+
+WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
+  WsPlan p;
+  size_t off = 0;
+  size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+  size_t F = c.d_ffn, V = c.vocab_out;
+  size_t M = (size_t)B * (max_gamma + 1);
+  p.max_rows = (int)M;
+  p.nsplit_max = (cap + ATTN_CHUNK - 1) / ATTN_CHUNK;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  p.len = take(B * 4);
+  p.pending = take(B * 4);
+  p.status = take(4);
+  p.counters = take(B * 4);
+  p.row_ids = take(M * 4);
+  p.accept_flags = take(M * 4);
+  p.h = take(M * d * 4);
+  p.qkv = take(M * (qd + 2 * kvd) * 4);
+  p.qrot = take(M * qd * 4);
+  p.rope_cs = take(M * c.head_dim * 4);
+  p.part = take(M * c.n_q_heads * (size_t)p.nsplit_max * (c.head_dim + 2) * 4);
+  p.logits = take(M * V * 4);
+  p.row_stats = take(M * 4 * 4);
+  p.xn = take(M * d * 4);
+  p.attn_out = take(M * qd * 4);
+  p.act = take(M * F * 4);
+  p.st_tokens = take((size_t)B * max_gamma * 4);
+  p.st_k = take(B * 4);
+  p.st_y = take(B * 4);
+  p.st_probs = take((size_t)B * max_gamma * V * 4);
+  p.st_uni = take(M * 2 * 4);
+  p.total = off;
+  return p;
+}
+
+bool streams_args_ok(const ssd_model_config* c, int B, int max_gamma, int cap) {
+  return cfg_ok(c) && B >= 1 && B <= 4096 && max_gamma >= 1 && max_gamma + 1 <= R_MAX &&
+         cap >= max_gamma + 1 && cap <= (1 << 20);
+}
+
+bool same_shape(const ssd_model_config& a, const ssd_model_config& b) {
+  return a.n_layers == b.n_layers && a.d_model == b.d_model && a.n_q_heads == b.n_q_heads &&
+         a.n_kv_heads == b.n_kv_heads && a.head_dim == b.head_dim && a.d_ffn == b.d_ffn &&
+         a.vocab_out == b.vocab_out && a.vocab_text == b.vocab_text &&
+         a.weight_dtype == b.weight_dtype;
+}
+
+// One decoder forward over the rows described by rm (ids already in s->row_ids).  Appends the
+// rows' K/V at len + r; when logits_out is non-null also runs the final norm and the LM head.
+int forward(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cudaStream_t st) {
+  const ssd_model_config& c = m->cfg;
+  const int dt = c.weight_dtype, M = rm.nb * rm.R, d = c.d_model;
+  const int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn;
+  launch_embed(dt, m->embed, c.vocab_out + c.vocab_text, d, s->row_ids, M, s->h, s->status, st);
+  launch_rope_table(s->len, rm, m->inv_freq, c.head_dim / 2, s->rope_cs, st);
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerW& w = m->layers[l];
+    void* kv_layer = s->kv + (size_t)l * s->kv_layer_elems * s->el;
+    launch_rmsnorm(dt, s->h, w.norm1, s->xn, M, d, c.rms_eps, st);
+    SSD_CUDA(launch_gemm_simt(dt, EPI_STORE_F32, s->xn, d, w.w_qkv, w.b_qkv, s->qkv,
+                              qd + 2 * kvd, M, qd + 2 * kvd, d, st));
+    launch_qkv_post(dt, s->qkv, s->rope_cs, s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads,
+                    c.n_kv_heads, c.head_dim, s->status, st);
+    SSD_CUDA(launch_attention_simt(dt, s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads,
+                                   c.n_kv_heads, c.head_dim, s->part, s->nsplit_max, s->attn_out,
+                                   st));
+    SSD_CUDA(launch_gemm_simt(dt, EPI_RESIDUAL, s->attn_out, qd, w.w_o, nullptr, s->h, d,
+                              M, d, qd, st));
+    launch_rmsnorm(dt, s->h, w.norm2, s->xn, M, d, c.rms_eps, st);
+    SSD_CUDA(launch_gemm_simt(dt, EPI_SWIGLU, s->xn, d, w.w_gu, nullptr, s->act, F, M,
+                              2 * F, d, st));
+    SSD_CUDA(launch_gemm_simt(dt, EPI_RESIDUAL, s->act, F, w.w_d, nullptr, s->h, d, M, d,
+                              F, st));
+  }
+  if (logits_out) {
+    launch_rmsnorm(dt, s->h, m->norm_f, s->xn, M, d, c.rms_eps, st);
+    SSD_CUDA(launch_gemm_simt(dt, EPI_STORE_F32, s->xn, d, m->head, nullptr, logits_out,
+                              c.vocab_out, M, c.vocab_out, d, st));
+  }
+  SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
+int params_ok(const ssd_streams* s, const ssd_verify_params* p, bool need_gamma) {
+  if (!p) return SSD_ERR_NULL;
+  if (need_gamma && (p->gamma < 1 || p->gamma > s->max_gamma)) return SSD_ERR_BAD_GAMMA;
+  if (!(p->temperature > 0.f) || !isfinite(p->temperature)) return SSD_ERR_BAD_PARAM;
+  if (!(p->beta >= 0.f) || !isfinite(p->beta)) return SSD_ERR_BAD_PARAM;
+  return SSD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t ssd_model_arena_bytes(const ssd_model_config* cfg) {
+  if (!cfg_ok(cfg)) return 0;
+  return plan_arena(*cfg).total;
+}
+
+int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size_t nbytes,
+                     void* dev_arena, size_t arena_bytes, ssd_model** out) {
+  if (!cfg || !host_weights || !dev_arena || !out) return SSD_ERR_NULL;
+  if (!cfg_ok(cfg)) return SSD_ERR_BAD_CONFIG;
+  if ((uintptr_t)dev_arena & 255) return SSD_ERR_MISALIGNED;
+  const ssd_model_config& c = *cfg;
+  ArenaPlan p = plan_arena(c);
+  const size_t el = c.weight_dtype == 0 ? 4 : 2;
+  if (arena_bytes < p.total) return SSD_ERR_TOO_SMALL;
+  if (nbytes != blob_elems(c) * el) return SSD_ERR_BAD_CONFIG;
+  ssd_model* m = new (std::nothrow) ssd_model();
+  if (!m) return SSD_ERR_CUDA;
+  m->cfg = c;
+  m->el = (int)el;
+  m->arena = (char*)dev_arena;
+  const char* src = (const char*)host_weights;
+  char* A = m->arena;
+  const size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+  const size_t F = c.d_ffn;
+  cudaError_t e = cudaSuccess;
+  auto put = [&](size_t dst_off, size_t elems) {
+    if (e == cudaSuccess) e = cudaMemcpy(A + dst_off, src, elems * el, cudaMemcpyHostToDevice);
+    src += elems * el;
+  };
+  put(p.embed, (size_t)(c.vocab_out + c.vocab_text) * d);
+  m->embed = A + p.embed;
+  m->layers.resize(c.n_layers);
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerOff& o = p.layers[l];
+    put(o.norm1, d);
+    put(o.w_qkv, qd * d);                        // wq
+    put(o.b_qkv, qd);                            // bq
+    put(o.w_qkv + qd * d * el, kvd * d);         // wk
+    put(o.b_qkv + qd * el, kvd);                 // bk
+    put(o.w_qkv + (qd + kvd) * d * el, kvd * d); // wv
+    put(o.b_qkv + (qd + kvd) * el, kvd);         // bv
+    put(o.w_o, d * qd);
+    put(o.norm2, d);
+    // gate and up rows interleaved (row 2j = gate_j, row 2j+1 = up_j) so that one thread / one
+    // accumulator tile owns both halves of SiLU(gate) * up
+    if (e == cudaSuccess)
+      e = cudaMemcpy2D(A + o.w_gu, 2 * d * el, src, d * el, d * el, F, cudaMemcpyHostToDevice);
+    src += F * d * el;
+    if (e == cudaSuccess)
+      e = cudaMemcpy2D(A + o.w_gu + d * el, 2 * d * el, src, d * el, d * el, F, cudaMemcpyHostToDevice);
+    src += F * d * el;
+    put(o.w_d, d * F);
+    m->layers[l] = LayerW{A + o.norm1, A + o.w_qkv, A + o.b_qkv, A + o.w_o, A + o.norm2, A + o.w_gu, A + o.w_d};
+  }
+  put(p.norm_f, d);
+  put(p.head, (size_t)c.vocab_out * d);
+  m->norm_f = A + p.norm_f;
+  m->head = A + p.head;
+  std::vector<double> inv(c.head_dim / 2);
+  for (int j = 0; j < c.head_dim / 2; ++j)
+    inv[j] = pow((double)c.rope_theta, -2.0 * j / (double)c.head_dim);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(A + p.inv_freq, inv.data(), inv.size() * sizeof(double), cudaMemcpyHostToDevice);
+  m->inv_freq = (const double*)(A + p.inv_freq);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete m;
+    return cuda_fail(e, "ssd_model_create copy");
+  }
+  *out = m;
+  return SSD_OK;
+}
+
+void ssd_model_destroy(ssd_model* m) { delete m; }
+
+size_t ssd_kv_bytes(const ssd_model_config* cfg, int32_t batch, int32_t capacity_tokens) {
+  if (!cfg_ok(cfg) || batch < 1 || capacity_tokens < 1) return 0;
+  size_t el = cfg->weight_dtype == 0 ? 4 : 2;
+  return (size_t)cfg->n_layers * batch * 2 * cfg->n_kv_heads * (size_t)capacity_tokens * cfg->head_dim * el;
+}
+
+size_t ssd_workspace_bytes(const ssd_model_config* cfg, int32_t batch, int32_t max_gamma,
+                           int32_t capacity_tokens) {
+  if (!streams_args_ok(cfg, batch, max_gamma, capacity_tokens)) return 0;
+  return plan_ws(*cfg, batch, max_gamma, capacity_tokens).total;
+}
+
+int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_tokens,
+                       int32_t max_gamma, void* dev_kv, size_t kv_bytes, void* dev_workspace,
+                       size_t ws_bytes, ssd_streams** out) {
+  if (!m || !dev_kv || !dev_workspace || !out) return SSD_ERR_NULL;
+  if (!streams_args_ok(&m->cfg, batch, max_gamma, capacity_tokens)) return SSD_ERR_BAD_CONFIG;
+  if (((uintptr_t)dev_kv & 255) || ((uintptr_t)dev_workspace & 255)) return SSD_ERR_MISALIGNED;
+  const ssd_model_config& c = m->cfg;
+  if (kv_bytes < ssd_kv_bytes(&c, batch, capacity_tokens)) return SSD_ERR_TOO_SMALL;
+  WsPlan p = plan_ws(c, batch, max_gamma, capacity_tokens);
+  if (ws_bytes < p.total) return SSD_ERR_TOO_SMALL;
+  SSD_CUDA(cudaMemset(dev_workspace, 0, p.total));
+  SSD_CUDA(cudaDeviceSynchronize());
+  ssd_streams* s = new (std::nothrow) ssd_streams();
+  if (!s) return SSD_ERR_CUDA;
+  s->cfg = c;
+  s->el = c.weight_dtype == 0 ? 4 : 2;
+  s->B = batch;
+  s->cap = capacity_tokens;
+  s->max_gamma = max_gamma;
+  s->max_rows = p.max_rows;
+  s->nsplit_max = p.nsplit_max;
+  s->kv = (char*)dev_kv;
+  s->kv_layer_elems = (size_t)batch * 2 * c.n_kv_heads * (size_t)capacity_tokens * c.head_dim;
+  char* W = (char*)dev_workspace;
+  s->ws = W;
+  s->ws_bytes = p.total;
+  s->len = (int32_t*)(W + p.len);
+  s->pending = (int32_t*)(W + p.pending);
+  s->status = (int32_t*)(W + p.status);
+  s->counters = (int32_t*)(W + p.counters);
+  s->row_ids = (int32_t*)(W + p.row_ids);
+  s->accept_flags = (int32_t*)(W + p.accept_flags);
+  s->h = (float*)(W + p.h);
+  s->qkv = (float*)(W + p.qkv);
+  s->qrot = (float*)(W + p.qrot);
+  s->rope_cs = (float*)(W + p.rope_cs);
+  s->part = (float*)(W + p.part);
+  s->logits = (float*)(W + p.logits);
+  s->row_stats = (float*)(W + p.row_stats);
+  s->xn = (float*)(W + p.xn);
+  s->attn_out = (float*)(W + p.attn_out);
+  s->act = (float*)(W + p.act);
+  s->st_tokens = (int32_t*)(W + p.st_tokens);
+  s->st_k = (int32_t*)(W + p.st_k);
+  s->st_y = (int32_t*)(W + p.st_y);
+  s->st_probs = (float*)(W + p.st_probs);
+  s->st_uni = (float*)(W + p.st_uni);
+  *out = s;
+  return SSD_OK;
+}
+
+void ssd_streams_destroy(ssd_streams* s) { delete s; }
+
+int ssd_kv_truncate(ssd_streams* s, const int32_t* host_len, const int32_t* host_pending,
+                    void* stream) {
+  if (!s || !host_len || !host_pending) return SSD_ERR_NULL;
+  for (int b = 0; b < s->B; ++b)
+    if (host_len[b] < 0 || host_len[b] > s->cap) return SSD_ERR_KV_OVERFLOW;
+  cudaStream_t st = (cudaStream_t)stream;
+  SSD_CUDA(cudaMemcpyAsync(s->len, host_len, s->B * 4, cudaMemcpyHostToDevice, st));
+  SSD_CUDA(cudaMemcpyAsync(s->pending, host_pending, s->B * 4, cudaMemcpyHostToDevice, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+int ssd_kv_restore(ssd_streams* s, const int32_t* dev_len, const int32_t* dev_pending, void* stream) {
+  if (!s || !dev_len || !dev_pending) return SSD_ERR_NULL;
+  launch_kv_restore(s->len, s->pending, dev_len, dev_pending, s->B, s->cap, (cudaStream_t)stream);
+  SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
+int ssd_streams_get_state(ssd_streams* s, int32_t* host_len, int32_t* host_pending, void* stream) {
+  if (!s) return SSD_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (host_len) SSD_CUDA(cudaMemcpyAsync(host_len, s->len, s->B * 4, cudaMemcpyDeviceToHost, st));
+  if (host_pending)
+    SSD_CUDA(cudaMemcpyAsync(host_pending, s->pending, s->B * 4, cudaMemcpyDeviceToHost, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int32_t* host_offsets,
+                void* stream) {
+  if (!m || !s || !dev_ids || !host_offsets) return SSD_ERR_NULL;
+  if (!same_shape(m->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
+  for (int b = 0; b < s->B; ++b) {
+    int n = host_offsets[b + 1] - host_offsets[b];
+    if (n < 1) return SSD_ERR_BAD_PARAM;
+    if (n - 1 > s->cap) return SSD_ERR_KV_OVERFLOW;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const int chunk = s->max_gamma + 1;
+  for (int b = 0; b < s->B; ++b) {
+    const int32_t* ids = dev_ids + host_offsets[b];
+    int n = host_offsets[b + 1] - host_offsets[b];
+    for (int done = 0; done < n - 1; done += chunk) {
+      int rows = n - 1 - done < chunk ? n - 1 - done : chunk;
+      SSD_CUDA(cudaMemcpyAsync(s->row_ids, ids + done, rows * 4, cudaMemcpyDeviceToDevice, st));
+      int rc = forward(m, s, RowMap{b, 1, rows}, nullptr, st);
+      if (rc != SSD_OK) return rc;
+      launch_advance_len(s->len, s->pending, b, rows, ids, -1, st);
+    }
+    launch_advance_len(s->len, s->pending, b, 0, ids, n - 1, st);
+  }
+  SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
+int ssd_draft_step(ssd_model* draft, ssd_streams* ds, const int32_t* dev_in_ids, int32_t n_in,
+                   const float* dev_uniform, const ssd_verify_params* params,
+                   int32_t* dev_out_token, float* dev_out_prob_row, void* stream) {
+  if (!draft || !ds || !dev_in_ids || !dev_uniform || !dev_out_token || !dev_out_prob_row)
+    return SSD_ERR_NULL;
+  if (!same_shape(draft->cfg, ds->cfg)) return SSD_ERR_BAD_CONFIG;
+  int rc = params_ok(ds, params, false);
+  if (rc != SSD_OK) return rc;
+  if (n_in < 1 || n_in > 2 || n_in > ds->max_gamma + 1) return SSD_ERR_BAD_PARAM;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int V = draft->cfg.vocab_out;
+  SSD_CUDA(cudaMemcpyAsync(ds->row_ids, dev_in_ids, (size_t)ds->B * n_in * 4, cudaMemcpyDeviceToDevice, st));
+  rc = forward(draft, ds, RowMap{0, ds->B, n_in}, ds->logits, st);
+  if (rc != SSD_OK) return rc;
+  launch_advance_all(ds->len, ds->B, n_in, ds->cap, ds->status, st);
+  SSD_CUDA(launch_draft_sampler(ds->logits + (size_t)(n_in - 1) * V, n_in * V, V, dev_uniform, ds->B,
+                                1.0f / params->temperature, params->top_k, dev_out_token,
+                                dev_out_prob_row, ds->pending, ds->status, st));
+  return SSD_OK;
+}
+
+int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens,
+               const float* dev_draft_probs, const float* dev_uniforms,
+               const ssd_verify_params* params, int32_t* dev_accepted_len,
+               int32_t* dev_next_token, float* dev_logits_or_null, void* stream) {
+  if (!target || !s || !dev_draft_tokens || !dev_draft_probs || !dev_uniforms || !dev_accepted_len ||
+      !dev_next_token)
+    return SSD_ERR_NULL;
+  if (!same_shape(target->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
+  int rc = params_ok(s, params, true);
+  if (rc != SSD_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int gamma = params->gamma;
+  float* logits = dev_logits_or_null ? dev_logits_or_null : s->logits;
+  launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
+  rc = forward(target, s, RowMap{0, s->B, gamma + 1}, logits, st);
+  if (rc != SSD_OK) return rc;
+  SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
+                                 dev_uniforms, s->B, gamma, 1.0f / params->temperature,
+                                 params->top_k, params->beta, s->row_stats, s->accept_flags,
+                                 s->counters, dev_accepted_len, dev_next_token, s->status, st));
+  return SSD_OK;
+}
+
+int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
+                  void* stream) {
+  if (!s || !dev_accepted_len || !dev_next_token) return SSD_ERR_NULL;
+  launch_kv_commit(s->len, s->pending, dev_accepted_len, dev_next_token, s->B, s->cap, s->status,
+                   (cudaStream_t)stream);
+  SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
+int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft_tokens,
+                    const float* host_draft_probs, const float* host_uniforms,
+                    const ssd_verify_params* params, int32_t* host_accepted_len,
+                    int32_t* host_next_token, void* stream) {
+  if (!target || !s || !host_draft_tokens || !host_draft_probs || !host_uniforms ||
+      !host_accepted_len || !host_next_token)
+    return SSD_ERR_NULL;
+  int rc = params_ok(s, params, true);
+  if (rc != SSD_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t B = s->B, g = params->gamma, V = target->cfg.vocab_out;
+  SSD_CUDA(cudaMemcpyAsync(s->st_tokens, host_draft_tokens, B * g * 4, cudaMemcpyHostToDevice, st));
+  SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, st));
+  SSD_CUDA(cudaMemcpyAsync(s->st_uni, host_uniforms, B * (g + 1) * 2 * 4, cudaMemcpyHostToDevice, st));
+  rc = ssd_verify(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr,
+                  stream);
+  if (rc != SSD_OK) return rc;
+  rc = ssd_kv_commit(s, s->st_k, s->st_y, stream);
+  if (rc != SSD_OK) return rc;
+  SSD_CUDA(cudaMemcpyAsync(host_accepted_len, s->st_k, B * 4, cudaMemcpyDeviceToHost, st));
+  SSD_CUDA(cudaMemcpyAsync(host_next_token, s->st_y, B * 4, cudaMemcpyDeviceToHost, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+int ssd_last_status(ssd_streams* s, int32_t* status, void* stream) {
+  if (!s || !status) return SSD_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  SSD_CUDA(cudaMemcpyAsync(status, s->status, 4, cudaMemcpyDeviceToHost, st));
+  SSD_CUDA(cudaMemsetAsync(s->status, 0, 4, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+uint64_t ssd_kernel_launch_count(void) { return launch_count(); }
+
+const char* ssd_last_cuda_error(void) { return g_cuda_err; }
+
+const char* ssd_strerror(int code) {
+  switch (code) {
+    case SSD_OK: return "ok";
+    case SSD_ERR_NULL: return "null pointer argument";
+    case SSD_ERR_BAD_CONFIG: return "unsupported or inconsistent configuration";
+    case SSD_ERR_BAD_GAMMA: return "gamma out of range";
+    case SSD_ERR_KV_OVERFLOW: return "KV cache capacity exceeded";
+    case SSD_ERR_MISALIGNED: return "buffer not 256-byte aligned";
+    case SSD_ERR_TOO_SMALL: return "caller buffer too small";
+    case SSD_ERR_CUDA: return "CUDA runtime error";
+    case SSD_ERR_BAD_PARAM: return "parameter out of range";
+  }
+  return "unknown error";
+}
+
+}  // extern "C"

@@ -1,0 +1,364 @@
+// Fused logits -> sampling transform -> acceptance test -> residual resample / bonus draw
+// (Algorithm 1's inner loop, Eq. 5 and Eq. 6), plus the KV commit.  Probability rows q_i never
+// reach global memory: each (stream, row) CTA keeps its row in shared memory and leaves only four
+// words of statistics; the CTA that finishes last for a stream reduces the accept flags to the
+// accepted length k, rebuilds row k on chip and draws the new token.
+//
+// p = DRAFT distribution, q = TARGET distribution, as in the paper.
+#include <math_constants.h>
+
+#include "kernels.h"
+
+namespace ssd {
+
+constexpr int SAMP_THREADS = 256;
+
+struct RowStats {
+  float zmax;        // max of z = logit / T over the row
+  float sum;         // sum of exp(z - zmax) over the kept set
+  uint32_t thr_key;  // order-preserving key of the smallest kept value (0 when top-k is off)
+  int tie_id_max;    // among values equal to the threshold, ids <= this are kept
+};
+
+// Monotone map float -> uint32 (larger float <=> larger key).
+__device__ __forceinline__ uint32_t order_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ bool is_kept(float z, int t, const RowStats& s) {
+  uint32_t k = order_key(z);
+  return k > s.thr_key || (k == s.thr_key && t <= s.tie_id_max);
+}
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = red[0];
+  for (int i = 1; i < SAMP_THREADS / 32; ++i) r = fmaxf(r, red[i]);
+  __syncthreads();
+  return r;
+}
+__device__ __forceinline__ double block_sum_d(double v, double* red) {
+  v = warp_sum_d(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double r = 0.0;
+  for (int i = 0; i < SAMP_THREADS / 32; ++i) r += red[i];
+  __syncthreads();
+  return r;
+}
+
+struct SampSmem {
+  double red_d[SAMP_THREADS / 32];
+  double scan[SAMP_THREADS];
+  float red_f[SAMP_THREADS / 32];
+  int hist[256];
+  uint32_t prefix;
+  int k_rem, eq_count, tie_id, bad, last, k_acc, y;
+};
+
+// Row statistics of the sampling transform: z/T is already in `z` (shared).  Block-collective.
+__device__ RowStats compute_row_stats(const float* z, int V, int top_k, SampSmem& sm) {
+  RowStats st;
+  float mx = -CUDART_INF_F;
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) mx = fmaxf(mx, z[t]);
+  st.zmax = block_max(mx, sm.red_f);
+  st.thr_key = 0u;
+  st.tie_id_max = V;
+  if (top_k > 0 && top_k < V) {
+    // radix select (4 passes of 8 bits, most significant first) of the top_k-th largest key
+    if (threadIdx.x == 0) { sm.prefix = 0u; sm.k_rem = top_k; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int i = threadIdx.x; i < 256; i += SAMP_THREADS) sm.hist[i] = 0;
+      __syncthreads();
+      const uint32_t prefix = sm.prefix;
+      const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+      for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+        uint32_t k = order_key(z[t]);
+        if ((k & mask) == prefix) atomicAdd(&sm.hist[(k >> shift) & 0xFF], 1);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        int rem = sm.k_rem, bin = 255;
+        for (; bin > 0; --bin) {
+          if (sm.hist[bin] >= rem) break;
+          rem -= sm.hist[bin];
+        }
+        sm.prefix = prefix | ((uint32_t)bin << shift);
+        sm.k_rem = rem;
+        sm.eq_count = sm.hist[bin];
+      }
+      __syncthreads();
+    }
+    st.thr_key = sm.prefix;
+    if (sm.eq_count > sm.k_rem) {  // equal values straddle the cut: keep the k_rem lowest ids
+      if (threadIdx.x == 0) {
+        int need = sm.k_rem, t = 0;
+        for (; t < V; ++t)
+          if (order_key(z[t]) == st.thr_key && --need == 0) break;
+        sm.tie_id = t;
+      }
+      __syncthreads();
+      st.tie_id_max = sm.tie_id;
+    }
+    __syncthreads();
+  }
+  double s = 0.0;
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS)
+    if (is_kept(z[t], t, st)) s += (double)expf(z[t] - st.zmax);
+  st.sum = (float)block_sum_d(s, sm.red_d);
+  return st;
+}
+
+// Inverse-CDF draw in ascending id over weights w[0..V) (shared): smallest t whose inclusive
+// cumulative sum exceeds u * total.  Returns -1 through *total_out <= 0.  Block-collective.
+__device__ int block_inverse_cdf(const float* w, int V, float u, SampSmem& sm, double* total_out) {
+  const int seg = (V + SAMP_THREADS - 1) / SAMP_THREADS;
+  const int t0 = min(threadIdx.x * seg, V), t1 = min(t0 + seg, V);
+  double s = 0.0;
+  for (int t = t0; t < t1; ++t) s += (double)w[t];
+  sm.scan[threadIdx.x] = s;
+  if (threadIdx.x == 0) sm.y = -1;
+  __syncthreads();
+  if (threadIdx.x == 0) {  // 256 adds: a serial scan is cheap and order-exact
+    double run = 0.0;
+    for (int i = 0; i < SAMP_THREADS; ++i) {
+      run += sm.scan[i];
+      sm.scan[i] = run;
+    }
+  }
+  __syncthreads();
+  const double total = sm.scan[SAMP_THREADS - 1];
+  *total_out = total;
+  if (!(total > 0.0)) {
+    __syncthreads();
+    return -1;
+  }
+  const double target = (double)u * total;
+  const double incl = sm.scan[threadIdx.x];
+  const double excl = threadIdx.x == 0 ? 0.0 : sm.scan[threadIdx.x - 1];
+  if (excl <= target && target < incl) {
+    double run = excl;
+    int y = -1;
+    for (int t = t0; t < t1; ++t) {
+      run += (double)w[t];
+      if (w[t] > 0.f) {
+        y = t;
+        if (run > target) break;
+      }
+    }
+    sm.y = y;
+  }
+  __syncthreads();
+  if (sm.y < 0 && threadIdx.x == 0) {  // u * total rounded up to total: last id with mass
+    int t = V - 1;
+    while (t > 0 && !(w[t] > 0.f)) --t;
+    sm.y = t;
+  }
+  __syncthreads();
+  int y = sm.y;
+  __syncthreads();
+  return y;
+}
+
+// Grid (R, B), R = gamma + 1.
+__global__ void __launch_bounds__(SAMP_THREADS)
+verify_sampler_kernel(const float* __restrict__ logits, int V,
+                      const int32_t* __restrict__ draft_tokens,
+                      const float* __restrict__ draft_probs, const float* __restrict__ uniforms,
+                      int gamma, float inv_t, int top_k, float beta, float* row_stats,
+                      int32_t* accept_flags, int32_t* counters, int32_t* __restrict__ accepted_len,
+                      int32_t* __restrict__ next_token, int32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SampSmem& sm = *reinterpret_cast<SampSmem*>(smem_raw);
+  float* z = reinterpret_cast<float*>(smem_raw + sizeof(SampSmem));
+  const int r = blockIdx.x, b = blockIdx.y, R = gamma + 1;
+  const float* lrow = logits + ((size_t)b * R + r) * V;
+  if (threadIdx.x == 0) sm.bad = 0;
+  __syncthreads();
+  int bad = 0;
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+    float v = lrow[t];
+    if (!isfinite(v)) bad = 1;
+    z[t] = v * inv_t;
+  }
+  if (bad) sm.bad = 1;
+  __syncthreads();
+  if (sm.bad && threadIdx.x == 0) atomicOr(status, SSD_STATUS_NONFINITE);
+  RowStats st = compute_row_stats(z, V, top_k, sm);
+  if (threadIdx.x == 0) {
+    int flag = 0;
+    if (r < gamma) {  // Eq. 5: accept x_i iff r_i < min(1, q_i(x_i) / p_i(x_i)) + beta
+      int x = draft_tokens[b * gamma + r];
+      float qx = 0.f, px = 0.f;
+      if (x < 0 || x >= V) {
+        atomicOr(status, SSD_STATUS_BAD_TOKEN);
+      } else {
+        if (is_kept(z[x], x, st)) qx = expf(z[x] - st.zmax) / st.sum;
+        px = draft_probs[((size_t)b * gamma + r) * V + x];
+        if (!(px >= 0.f) || !isfinite(px)) {
+          atomicOr(status, SSD_STATUS_BAD_PROB);
+          px = 0.f;
+        }
+      }
+      float ratio = px <= qx ? 1.f : qx / px;
+      flag = uniforms[((size_t)b * R + r) * 2] < ratio + beta;
+    }
+    float* rs = row_stats + ((size_t)b * R + r) * 4;
+    rs[0] = st.zmax;
+    rs[1] = st.sum;
+    rs[2] = __uint_as_float(st.thr_key);
+    rs[3] = __int_as_float(st.tie_id_max);
+    accept_flags[b * R + r] = flag;
+    __threadfence();
+    int prev = atomicAdd(&counters[b], 1);
+    sm.last = prev == R - 1;
+  }
+  __syncthreads();
+  if (!sm.last) return;
+  // ---- last CTA of this stream: first rejection, then the one new token ----
+  if (threadIdx.x == 0) {
+    __threadfence();
+    counters[b] = 0;
+    int k = gamma;
+    for (int i = 0; i < gamma; ++i)
+      if (__ldcg(&accept_flags[b * R + i]) == 0) { k = i; break; }
+    sm.k_acc = k;
+  }
+  __syncthreads();
+  const int k = sm.k_acc;
+  const float* rs = row_stats + ((size_t)b * R + k) * 4;
+  RowStats sk;
+  sk.zmax = __ldcg(rs + 0);
+  sk.sum = __ldcg(rs + 1);
+  sk.thr_key = __float_as_uint(__ldcg(rs + 2));
+  sk.tie_id_max = __float_as_int(__ldcg(rs + 3));
+  const float* krow = logits + ((size_t)b * R + k) * V;
+  const float* prow = k < gamma ? draft_probs + ((size_t)b * gamma + k) * V : nullptr;
+  // Eq. 6: w = max(0, q_k - p_k) on a rejection; the bonus row q_{gamma+1} otherwise
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+    float zz = krow[t] * inv_t;
+    float q = is_kept(zz, t, sk) ? expf(zz - sk.zmax) / sk.sum : 0.f;
+    z[t] = prow ? fmaxf(0.f, q - prow[t]) : q;
+  }
+  __syncthreads();
+  const float u = uniforms[((size_t)b * R + k) * 2 + 1];
+  double total;
+  int y = block_inverse_cdf(z, V, u, sm, &total);
+  if (y < 0) {  // residual has no mass (numerical corner): draw from q_k itself
+    for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+      float zz = krow[t] * inv_t;
+      z[t] = is_kept(zz, t, sk) ? expf(zz - sk.zmax) / sk.sum : 0.f;
+    }
+    __syncthreads();
+    y = block_inverse_cdf(z, V, u, sm, &total);
+    if (y < 0) y = 0;
+  }
+  if (threadIdx.x == 0) {
+    accepted_len[b] = k;
+    next_token[b] = y;
+  }
+}
+
+cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* draft_tokens,
+                                  const float* draft_probs, const float* uniforms, int B,
+                                  int gamma, float inv_temperature, int top_k, float beta,
+                                  float* row_stats, int32_t* accept_flags, int32_t* counters,
+                                  int32_t* accepted_len, int32_t* next_token, int32_t* status,
+                                  cudaStream_t st) {
+  size_t smem = sizeof(SampSmem) + (size_t)V * sizeof(float);
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(verify_sampler_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid(gamma + 1, B);
+  verify_sampler_kernel<<<grid, SAMP_THREADS, smem, st>>>(
+      logits, V, draft_tokens, draft_probs, uniforms, gamma, inv_temperature, top_k, beta,
+      row_stats, accept_flags, counters, accepted_len, next_token, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// Draft side (Eq. 2-3): p = transform(logits row), x ~ p by inverse CDF; p is written out in full
+// because the verifier needs the whole row (Eq. 6).  One CTA per stream.
+__global__ void __launch_bounds__(SAMP_THREADS)
+draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
+                     const float* __restrict__ uniform, float inv_t, int top_k,
+                     int32_t* __restrict__ out_token, float* __restrict__ out_prob,
+                     int32_t* pending, int32_t* status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SampSmem& sm = *reinterpret_cast<SampSmem*>(smem_raw);
+  float* z = reinterpret_cast<float*>(smem_raw + sizeof(SampSmem));
+  const int b = blockIdx.x;
+  const float* lrow = logits + (size_t)b * ld_logits;
+  if (threadIdx.x == 0) sm.bad = 0;
+  __syncthreads();
+  int bad = 0;
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+    float v = lrow[t];
+    if (!isfinite(v)) bad = 1;
+    z[t] = v * inv_t;
+  }
+  if (bad) sm.bad = 1;
+  __syncthreads();
+  if (sm.bad && threadIdx.x == 0) atomicOr(status, SSD_STATUS_NONFINITE);
+  RowStats st = compute_row_stats(z, V, top_k, sm);
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+    float p = is_kept(z[t], t, st) ? expf(z[t] - st.zmax) / st.sum : 0.f;
+    z[t] = p;
+    out_prob[(size_t)b * V + t] = p;
+  }
+  __syncthreads();
+  double total;
+  int y = block_inverse_cdf(z, V, uniform[b], sm, &total);
+  if (y < 0) y = 0;
+  if (threadIdx.x == 0) {
+    out_token[b] = y;
+    pending[b] = y;
+  }
+}
+
+cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, const float* uniform,
+                                 int B, float inv_temperature, int top_k, int32_t* out_token,
+                                 float* out_prob_row, int32_t* pending, int32_t* status,
+                                 cudaStream_t st) {
+  size_t smem = sizeof(SampSmem) + (size_t)V * sizeof(float);
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(draft_sampler_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  draft_sampler_kernel<<<B, SAMP_THREADS, smem, st>>>(logits, ld_logits, V, uniform,
+                                                      inv_temperature, top_k, out_token,
+                                                      out_prob_row, pending, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// "Append to T_in" (Algorithm 1): the prefix grows by the k accepted tokens plus the new one.
+__global__ void kv_commit_kernel(int32_t* len, int32_t* pending, const int32_t* accepted_len,
+                                 const int32_t* next_token, int B, int cap, int32_t* status) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int nl = len[b] + 1 + accepted_len[b];
+  if (nl > cap) {
+    atomicOr(status, SSD_STATUS_KV_OVERFLOW);
+    nl = cap;
+  }
+  len[b] = nl;
+  pending[b] = next_token[b];
+}
+
+void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_len,
+                      const int32_t* next_token, int B, int cap, int32_t* status, cudaStream_t st) {
+  kv_commit_kernel<<<(B + 127) / 128, 128, 0, st>>>(len, pending, accepted_len, next_token, B, cap,
+                                                    status);
+  count_launch();
+}
+
+}  // namespace ssd

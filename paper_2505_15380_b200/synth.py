@@ -253,3 +253,19 @@ def sample_from_rows(p: np.ndarray, seed: int) -> np.ndarray:
     cdf = np.cumsum(p.astype(np.float64), axis=1)
     idx = (cdf > (u * cdf[:, -1])[:, None]).argmax(axis=1)
     return idx.astype(np.int32)
+
+
+def fill_synthetic_kv(kv, lens, seed: int, std: float = 0.6) -> None:
+    """Seeded random prefix K/V written into a device cache tensor
+    kv[layer, stream, 2, kv_head, capacity, head_dim] for slots < lens[stream].
+
+    Stand-in for a real prefill where that would take too long: entries ~ N(0, std^2) in the
+    cache's storage type (std 0.6 is what random-init projections of unit-RMS inputs produce).
+    """
+    import torch
+    g = torch.Generator(device=kv.device)
+    g.manual_seed(seed)
+    for b, n in enumerate(lens):
+        blk = torch.randn((kv.shape[0], 2, kv.shape[3], int(n), kv.shape[5]), generator=g,
+                          device=kv.device, dtype=torch.float32) * std
+        kv[:, b, :, :, :int(n), :] = blk.to(kv.dtype)

@@ -1,0 +1,190 @@
+"""Runs one verify-step workload on the CUDA path and on the oracle and compares them.
+
+Used by the GPU parity tests and by the smoke check.  The comparison rules:
+
+* logits: max-abs difference within `logit_tol` (3e-2 for bf16 storage, 2e-4 for fp32);
+* token decisions, strict: the oracle's acceptance arithmetic applied to the GPU's own logits
+  must reproduce the GPU's (k, y) exactly, except for draws closer than 1e-3 to a decision
+  boundary (|r_i - a_i| < 1e-3, a categorical draw within 1e-3 of a CDF edge, or a top-k cut
+  whose neighbours differ by < 1e-3), after which the stream-step is no longer compared;
+* token decisions, end to end: the pure oracle's (k, y) must equal the GPU's unless r_i falls
+  between the two sides' thresholds (widened by 1e-3), i.e. unless the logit rounding moved a
+  boundary across the uniform.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from oracle import ssd_oracle as orc
+from paper_2505_15380_b200 import binding, synth
+from tests.helpers import crafted_draft_rows, oracle_model
+
+WINDOW = 1e-3
+
+
+@dataclasses.dataclass
+class CaseResult:
+    max_logit_err: float
+    n_streams: int
+    n_strict_excluded: int
+    n_e2e_excluded: int
+    ks: List[int]
+
+
+def synthetic_kv(streams: binding.Streams, lens, seed: int, std: float = 0.6) -> None:
+    synth.fill_synthetic_kv(streams.kv, lens, seed, std)
+
+
+def oracle_stream_from_gpu_kv(model: orc.Model, streams: binding.Streams, b: int, n: int,
+                              pending: int) -> orc.Stream:
+    st = orc.Stream(model, streams.capacity)
+    kv = streams.kv[:, b, :, :, :n, :].to(torch.float32).cpu().numpy().astype(np.float64)
+    for l in range(model.L):
+        st.K[l][:n] = kv[l, 0].transpose(1, 0, 2)
+        st.V[l][:n] = kv[l, 1].transpose(1, 0, 2)
+    st.length, st.pending = n, pending
+    return st
+
+
+def _topk_gap_small(logits_row: np.ndarray, temperature: float, top_k: int) -> bool:
+    V = logits_row.shape[0]
+    if not (0 < top_k < V):
+        return False
+    z = np.sort(logits_row / temperature)[::-1]
+    return bool(z[top_k - 1] - z[top_k] < WINDOW)
+
+
+def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "prefill",
+             oracle_streams: Optional[List[int]] = None, logit_tol: Optional[float] = None,
+             uniform_seed: int = 0, commit_and_repeat: bool = False,
+             capacity: Optional[int] = None) -> CaseResult:
+    """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
+    'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
+    shape = wl.target
+    B, gamma, R, V = wl.batch, wl.gamma, wl.gamma + 1, shape.vocab_out
+    if logit_tol is None:
+        logit_tol = 2e-4 if shape.weight_dtype == synth.F32 else 3e-2
+    w = synth.make_weights(shape, wl.model_seed)
+    omodel = oracle_model(shape, w)
+    gmodel = binding.Model(shape, synth.weights_blob(shape, w))
+    cap = capacity or (max(wl.prefix_lens) + 2 * R + 8)
+    gs = binding.Streams(gmodel, B, cap, gamma)
+    which = list(range(B)) if oracle_streams is None else list(oracle_streams)
+    prefixes = [synth.make_prefix(wl, b) for b in range(B)]
+    ostreams = {}
+    if kv_mode == "prefill":
+        gs.prefill(prefixes)
+        for b in which:
+            st = orc.Stream(omodel, cap)
+            orc.prefill(omodel, st, prefixes[b])
+            ostreams[b] = st
+    else:
+        lens = [len(p) - 1 for p in prefixes]
+        synthetic_kv(gs, lens, seed=wl.data_seed + 100)
+        gs.kv_truncate(lens, [int(p[-1]) for p in prefixes])
+        for b in which:
+            ostreams[b] = oracle_stream_from_gpu_kv(omodel, gs, b, lens[b], int(prefixes[b][-1]))
+    lens_g, pend_g = gs.get_state()
+    for b in which:
+        assert lens_g[b] == ostreams[b].length and pend_g[b] == ostreams[b].pending
+
+    n_steps = 2 if commit_and_repeat else 1
+    res = CaseResult(0.0, 0, 0, 0, [])
+    dev = gmodel.device
+    for step in range(n_steps):
+        uni = synth.verify_uniforms(uniform_seed, B, R, step=step)
+        # ---- draft rows: crafted from sequential ORACLE decodes for the checked streams,
+        #      generic random rows elsewhere
+        p_rows = synth.random_prob_rows(B * gamma, V, seed=wl.data_seed + step, support=64
+                                        ).reshape(B, gamma, V)
+        draft = synth.sample_from_rows(p_rows.reshape(-1, V), seed=wl.data_seed + 5 + step
+                                       ).reshape(B, gamma)
+        for b in which:
+            st = ostreams[b]
+            base_len = st.length
+            tok = st.pending
+            for i in range(gamma):
+                lg = orc.forward(omodel, st, np.array([tok]))[0]
+                st.length += 1
+                row = crafted_draft_rows(lg[None], sigma, wl.temperature, wl.top_k,
+                                         seed=1000 * b + 10 * i + step)[0]
+                p_rows[b, i] = row
+                tok = int(synth.sample_from_rows(row[None], seed=77 + 1000 * b + i + step)[0])
+                draft[b, i] = tok
+            st.length = base_len
+        # ---- GPU
+        params = binding.VerifyParams(gamma, wl.temperature, wl.top_k, beta)
+        d_tok = torch.from_numpy(draft.astype(np.int32)).to(dev)
+        d_p = torch.from_numpy(p_rows.astype(np.float32)).to(dev)
+        d_u = torch.from_numpy(uni).to(dev)
+        d_k = torch.zeros(B, dtype=torch.int32, device=dev)
+        d_y = torch.zeros(B, dtype=torch.int32, device=dev)
+        d_logits = torch.zeros((B, R, V), dtype=torch.float32, device=dev)
+        gs.verify(d_tok, d_p, d_u, params, d_k, d_y, d_logits)
+        torch.cuda.synchronize()
+        assert gs.last_status() == 0
+        # same call again without a commit: must be bit-identical (no races, no stale state)
+        d_k2, d_y2, d_l2 = torch.zeros_like(d_k), torch.zeros_like(d_y), torch.zeros_like(d_logits)
+        gs.verify(d_tok, d_p, d_u, params, d_k2, d_y2, d_l2)
+        torch.cuda.synchronize()
+        assert torch.equal(d_k, d_k2) and torch.equal(d_y, d_y2) and torch.equal(d_logits, d_l2)
+        g_k, g_y, g_logits = d_k.cpu().numpy(), d_y.cpu().numpy(), d_logits.cpu().numpy()
+        assert ((g_k >= 0) & (g_k <= gamma)).all() and ((g_y >= 0) & (g_y < V)).all()
+        # ---- oracle and comparison
+        for b in which:
+            st = ostreams[b]
+            o = orc.verify(omodel, st, draft[b], p_rows[b], uni[b], temperature=wl.temperature,
+                           top_k=wl.top_k, beta=beta)
+            err = float(np.abs(o["logits"] - g_logits[b]).max())
+            res.max_logit_err = max(res.max_logit_err, err)
+            assert err <= logit_tol, f"stream {b}: logits differ by {err}"
+            # strict: oracle arithmetic on the GPU's logits
+            gl = g_logits[b].astype(np.float64)
+            q_g = np.stack([orc.transform(r, wl.temperature, wl.top_k) for r in gl])
+            o2 = orc.accept_step(q_g, p_rows[b], draft[b], uni[b], beta)
+            res.n_streams += 1
+            res.ks.append(int(g_k[b]))
+            strict_excl = False
+            n_eval = min(o2["k"] + 1, gamma)
+            for i in range(n_eval):
+                if abs(o2["thresholds"][i] - float(uni[b, i, 0])) < WINDOW or \
+                        _topk_gap_small(gl[i], wl.temperature, wl.top_k):
+                    strict_excl = True
+                    break
+            if not strict_excl:
+                assert g_k[b] == o2["k"], f"stream {b}: accepted length {g_k[b]} vs {o2['k']}"
+                if o2["draw_margin"] < WINDOW or _topk_gap_small(gl[o2["k"]], wl.temperature,
+                                                                 wl.top_k):
+                    strict_excl = True
+                else:
+                    assert g_y[b] == o2["y"], f"stream {b}: token {g_y[b]} vs {o2['y']}"
+            res.n_strict_excluded += int(strict_excl)
+            # end to end: pure oracle
+            e2e_excl = strict_excl
+            for i in range(min(max(o["k"], o2["k"]) + 1, gamma)):
+                lo = min(o["thresholds"][i] if i < len(o["thresholds"]) else 9.0,
+                         o2["thresholds"][i] if i < len(o2["thresholds"]) else 9.0) - WINDOW
+                hi = max(o["thresholds"][i] if i < len(o["thresholds"]) else -9.0,
+                         o2["thresholds"][i] if i < len(o2["thresholds"]) else -9.0) + WINDOW
+                if lo <= float(uni[b, i, 0]) <= hi:
+                    e2e_excl = True
+            if not e2e_excl:
+                assert g_k[b] == o["k"], f"stream {b}: e2e accepted length {g_k[b]} vs {o['k']}"
+                if o["y"] == o2["y"] and o["draw_margin"] >= WINDOW:
+                    assert g_y[b] == o["y"]
+                else:
+                    e2e_excl = True
+            res.n_e2e_excluded += int(e2e_excl)
+            if commit_and_repeat:
+                orc.commit(st, int(g_k[b]), int(g_y[b]))      # follow the GPU's trajectory
+        if commit_and_repeat:
+            gs.kv_commit(d_k, d_y)
+            torch.cuda.synchronize()
+            lens_g, pend_g = gs.get_state()
+            for b in which:
+                assert lens_g[b] == ostreams[b].length and pend_g[b] == ostreams[b].pending
+    return res

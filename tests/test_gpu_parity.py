@@ -1,0 +1,170 @@
+"""GPU parity: the CUDA verify path (through the C ABI) against the CPU oracle."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_15380_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(*a, **k):
+    from tests.gpu_case import run_case
+    return run_case(*a, **k)
+
+
+def _small(dtype, hd, hq=4, hkv=2, d=64, f=96, v=300, layers=2, vt=8):
+    return synth.ModelShape(layers, d, hq, hkv, hd, f, v, vt, 1e4, weight_dtype=dtype)
+
+
+def _wl(shape, batch, gamma, lens, temperature=1.0, top_k=0, n_text=2, seed=11):
+    return synth.Workload("custom", shape, shape, batch, gamma, temperature, top_k, tuple(lens),
+                          n_text, seed, seed + 1)
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.4])
+@pytest.mark.parametrize("sigma", [0.0, 0.3, 1.0, 3.0])
+def test_cfg0_tiny_fp32(beta, sigma):
+    r = _case(synth.workload(0), beta=beta, sigma=sigma, commit_and_repeat=True)
+    assert r.max_logit_err < 2e-4
+
+
+def test_accepted_lengths_cover_all_branches():
+    """Across draft qualities every k in 0..gamma and both draw branches must occur."""
+    seen = set()
+    for sigma, beta, seed in [(0.0, 0.0, 0), (0.5, 0.0, 1), (1.0, 0.0, 2), (1.0, 0.4, 3),
+                              (2.0, 0.0, 4), (3.0, 0.0, 5), (0.7, 0.0, 6), (1.5, 0.2, 7)]:
+        shape = _small(synth.F32, 32)
+        wl = _wl(shape, 6, 4, [40, 33, 70, 64, 65, 12], seed=seed + 20)
+        r = _case(wl, beta=beta, sigma=sigma, uniform_seed=seed)
+        seen.update(r.ks)
+    assert seen == {0, 1, 2, 3, 4}
+
+
+@pytest.mark.parametrize("hd", [32, 64, 128])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_small_shapes_ragged_batch(hd, dtype):
+    shape = _small(dtype, hd, hq=6, hkv=2, d=128, f=200)
+    # lengths straddle the 64-key attention chunk and include the minimum (a 1-token prefix)
+    wl = _wl(shape, 5, 3, [1, 2, 64, 65, 130])
+    _case(wl, beta=0.0, sigma=0.5)
+    _case(wl, beta=0.4, sigma=2.0, commit_and_repeat=True)
+
+
+@pytest.mark.parametrize("gamma", [1, 2, 8, 15])
+def test_gamma_range(gamma):
+    shape = _small(synth.BF16, 64, hq=14, hkv=2, d=128, f=256)
+    wl = _wl(shape, 2, gamma, [70, 129])
+    _case(wl, beta=0.0, sigma=0.7)
+
+
+@pytest.mark.parametrize("top_k,temperature", [(25, 0.8), (1, 1.0), (299, 0.5), (1000, 1.3)])
+def test_top_k_and_temperature(top_k, temperature):
+    shape = _small(synth.BF16, 64)
+    wl = _wl(shape, 4, 4, [50, 64, 100, 7], temperature=temperature, top_k=top_k)
+    _case(wl, beta=0.0, sigma=0.5)
+    _case(wl, beta=0.4, sigma=1.5)
+
+
+def test_mha_no_grouping_and_single_kv_head():
+    _case(_wl(_small(synth.F32, 32, hq=4, hkv=4), 2, 4, [30, 90]), beta=0.0, sigma=0.5)
+    _case(_wl(_small(synth.BF16, 64, hq=8, hkv=1, d=128), 2, 4, [30, 90]), beta=0.0, sigma=0.5)
+
+
+def test_cfg1_qwen2_style_prefill_300():
+    r = _case(synth.workload(1), beta=0.0, sigma=0.5, commit_and_repeat=True)
+    assert r.max_logit_err < 3e-2
+
+
+@pytest.mark.parametrize("gamma,prefix", [(2, 256), (4, 512), (6, 1024), (8, 2048)])
+def test_cfg2_sweep_synthetic_kv(gamma, prefix):
+    _case(synth.workload(2, gamma=gamma, prefix=prefix), beta=0.4, sigma=1.0, kv_mode="synthetic")
+
+
+def test_cfg3_batch16_ragged_topk():
+    r = _case(synth.workload(3), beta=0.0, sigma=0.7, kv_mode="synthetic",
+              oracle_streams=[0, 3, 7, 12, 15])
+    assert r.n_streams == 5
+
+
+def test_cfg4_large_batch64_sampled_streams():
+    """Full-size launch (64 streams x 4096-token prefixes); oracle on sampled streams."""
+    r = _case(synth.workload(4), beta=0.4, sigma=1.0, kv_mode="synthetic", oracle_streams=[0, 37, 63])
+    assert r.n_streams == 3
+
+
+def test_verify_host_matches_device_call():
+    from paper_2505_15380_b200 import binding
+    shape = _small(synth.BF16, 64)
+    wl = _wl(shape, 3, 4, [20, 64, 90])
+    w = synth.make_weights(shape, 3)
+    model = binding.Model(shape, synth.weights_blob(shape, w))
+    gs = binding.Streams(model, 3, 128, 4)
+    gs.prefill([synth.make_prefix(wl, b) for b in range(3)])
+    lens0, pend0 = gs.get_state()
+    V = shape.vocab_out
+    p = synth.random_prob_rows(12, V, 1).reshape(3, 4, V)
+    x = synth.sample_from_rows(p.reshape(-1, V), 2).reshape(3, 4).astype(np.int32)
+    u = synth.verify_uniforms(3, 3, 5)
+    par = binding.VerifyParams(4, 1.0, 0, 0.3)
+    dev = model.device
+    k = torch.zeros(3, dtype=torch.int32, device=dev)
+    y = torch.zeros(3, dtype=torch.int32, device=dev)
+    gs.verify(torch.from_numpy(x).to(dev), torch.from_numpy(p).to(dev), torch.from_numpy(u).to(dev),
+              par, k, y)
+    torch.cuda.synchronize()
+    hk = torch.zeros(3, dtype=torch.int32).pin_memory()
+    hy = torch.zeros(3, dtype=torch.int32).pin_memory()
+    gs.verify_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(p).pin_memory(),
+                   torch.from_numpy(u).pin_memory(), par, hk, hy)
+    assert torch.equal(hk, k.cpu()) and torch.equal(hy, y.cpu())
+    lens1, pend1 = gs.get_state()                      # verify_host commits
+    assert np.array_equal(lens1, lens0 + 1 + hk.numpy()) and np.array_equal(pend1, hy.numpy())
+    gs.kv_truncate(lens0, pend0)                       # O(1) rollback restores the step
+    gs.verify_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(p).pin_memory(),
+                   torch.from_numpy(u).pin_memory(), par, hk, hy)
+    assert torch.equal(hk, k.cpu()) and torch.equal(hy, y.cpu())
+
+
+def test_device_status_flags_and_host_errors():
+    from paper_2505_15380_b200 import binding
+    shape = _small(synth.F32, 32)
+    w = synth.make_weights(shape, 3)
+    model = binding.Model(shape, synth.weights_blob(shape, w))
+    gs = binding.Streams(model, 1, 16, 4)
+    V = shape.vocab_out
+    dev = model.device
+    p = torch.from_numpy(synth.random_prob_rows(4, V, 1)).to(dev)
+    u = torch.from_numpy(synth.verify_uniforms(0, 1, 5)).to(dev)
+    k = torch.zeros(1, dtype=torch.int32, device=dev)
+    y = torch.zeros(1, dtype=torch.int32, device=dev)
+    # cache of 16 slots, len 14: rows at 14..18 overflow -> flagged, nothing written out of range
+    gs.kv_truncate([14], [3])
+    x = torch.tensor([[1, 2, 3, 4]], dtype=torch.int32, device=dev)
+    gs.verify(x, p, u, binding.VerifyParams(4, 1.0, 0, 0.0), k, y)
+    assert gs.last_status() & 1
+    assert gs.last_status() == 0                       # reading clears
+    # a token id outside the table is clamped and flagged
+    gs.kv_truncate([2], [3])
+    bad = torch.tensor([[1, 2, 10 ** 6, 4]], dtype=torch.int32, device=dev)
+    gs.verify(bad, p, u, binding.VerifyParams(4, 1.0, 0, 0.0), k, y)
+    assert gs.last_status() & 2
+    # host-side argument errors enqueue nothing
+    x9 = torch.zeros((1, 9), dtype=torch.int32, device=dev)
+    p9 = torch.zeros((1, 9, V), dtype=torch.float32, device=dev)
+    u9 = torch.zeros((1, 10, 2), dtype=torch.float32, device=dev)
+    with pytest.raises(binding.SsdError, match="gamma"):       # streams were created for gamma <= 4
+        gs.verify(x9, p9, u9, binding.VerifyParams(9, 1.0, 0, 0.0), k, y)
+    with pytest.raises(binding.SsdError, match="parameter"):
+        gs.verify(x, p, u, binding.VerifyParams(4, 0.0, 0, 0.0), k, y)
+    with pytest.raises(binding.SsdError, match="capacity"):
+        gs.kv_truncate([17], [0])
+    L = binding.lib()
+    assert L.ssd_kv_commit(gs.handle, None, None, None) == -1
+    h = ctypes.c_void_p()
+    assert L.ssd_streams_create(model.handle, 1, 16, 4, gs.kv_raw.data_ptr(), 8,
+                                gs.ws.data_ptr(), gs.ws.numel(), ctypes.byref(h)) == -6
+    assert L.ssd_streams_create(model.handle, 1, 16, 4, gs.kv_raw.data_ptr() + 2, 1 << 30,
+                                gs.ws.data_ptr(), gs.ws.numel(), ctypes.byref(h)) == -5
