@@ -173,6 +173,28 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
 int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
                   void* stream);
 
+/* Acceptance step without any device allocation (the paper has no counterpart: this is a
+ * packaging variant of the acceptance kernel behind ssd_verify, not a step of the method).
+ * For callers that may not allocate device memory at all - e.g. a serving loop whose memory pool
+ * is fixed at start-up, or a plug-in that only receives device pointers from its host process -
+ * and so cannot provide the workspace ssd_streams_create needs.  Given target logits the caller
+ * already holds, it applies the sampling transform, the tolerance test of Eq. 5 and the resample /
+ * bonus draw of Eq. 6 exactly as ssd_verify does, and writes the same two outputs.
+ *   in  dev_logits float [batch, gamma+1, vocab]; dev_draft_tokens, dev_draft_probs, dev_uniforms
+ *       as in ssd_verify;  out dev_accepted_len, dev_next_token int32 [batch].
+ * The kernel's scratch lives in a fixed array inside the library (about 84 KB, held by every GPU
+ * that loads the library until the process exits), sized for at most 256 streams and
+ * gamma + 1 <= 16 rows: larger batches return SSD_ERR_TOO_SMALL, larger gamma SSD_ERR_BAD_GAMMA.
+ * No cudaMalloc / cudaFree or allocating library routine is called.  The first call on a device
+ * looks up the array's address (cudaGetSymbolAddress, with that device current); make that first
+ * call before starting any stream capture.  All calls share the one array, which keeps the last
+ * call's contents: the per-stream counters are cleared on `stream` at the start of each call, and
+ * two calls that overlap on the GPU (different streams, or different threads) race on it. */
+int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_draft_tokens,
+                       const float* dev_draft_probs, const float* dev_uniforms,
+                       const ssd_verify_params* params, int32_t batch, int32_t vocab,
+                       int32_t* dev_accepted_len, int32_t* dev_next_token, void* stream);
+
 /* ---- diagnostics ------------------------------------------------------------------------- */
 
 /* Reads and clears the device status word (SSD_STATUS_* bits).  Synchronises `stream`. */

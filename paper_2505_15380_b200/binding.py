@@ -21,7 +21,8 @@ EXPORTS = [
     "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
     "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
-    "ssd_kv_commit", "ssd_kv_restore", "ssd_kernel_launch_count", "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
+    "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_kernel_launch_count",
+    "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
 
 
@@ -72,6 +73,7 @@ def lib() -> ctypes.CDLL:
     L.ssd_verify_host.argtypes = [vp, vp, vp, vp, vp, parp, vp, vp, vp]
     L.ssd_kv_commit.argtypes = [vp, vp, vp, vp]
     L.ssd_kv_restore.argtypes = [vp, vp, vp, vp]
+    L.ssd_accept_noalloc.argtypes = [vp, vp, vp, vp, parp, i32, i32, vp, vp, vp]
     L.ssd_kernel_launch_count.restype = ctypes.c_uint64
     L.ssd_kernel_launch_count.argtypes = []
     L.ssd_last_status.argtypes = [vp, ctypes.POINTER(i32), vp]
@@ -251,3 +253,21 @@ class Streams:
         check(lib().ssd_draft_step(self.model.handle, self.handle, in_ids.data_ptr(), n_in,
                                    uniform.data_ptr(), ctypes.byref(params), out_token.data_ptr(),
                                    out_prob_row.data_ptr(), _stream_ptr(stream)))
+
+
+def accept_noalloc(logits: torch.Tensor, draft_tokens: torch.Tensor, draft_probs: torch.Tensor,
+                   uniforms: torch.Tensor, params: VerifyParams, accepted_len: torch.Tensor,
+                   next_token: torch.Tensor, stream=None) -> None:
+    """ssd_accept_noalloc: the acceptance step on caller-held logits [B, gamma+1, V], for callers
+    that cannot allocate device memory (the kernel's scratch is a fixed array in the library).
+    Limits: at most 256 streams, gamma + 1 <= 16.  Calls share that array, so calls that overlap
+    on the GPU race; make the first call on a device outside any stream capture."""
+    B, R, V = logits.shape
+    assert logits.dtype == torch.float32 and logits.is_cuda and logits.is_contiguous()
+    assert R == params.gamma + 1 and draft_tokens.numel() == B * params.gamma
+    assert draft_probs.numel() == B * params.gamma * V and uniforms.numel() == B * R * 2
+    with torch.cuda.device(logits.device):
+        check(lib().ssd_accept_noalloc(logits.data_ptr(), draft_tokens.data_ptr(),
+                                       draft_probs.data_ptr(), uniforms.data_ptr(),
+                                       ctypes.byref(params), B, V, accepted_len.data_ptr(),
+                                       next_token.data_ptr(), _stream_ptr(stream)))

@@ -180,6 +180,10 @@ int params_ok(const ssd_streams* s, const ssd_verify_params* p, bool need_gamma)
 
 }  // namespace
 
+namespace ssd {
+int report_cuda_error(cudaError_t e, const char* what) { return cuda_fail(e, what); }
+}  // namespace ssd
+
 extern "C" {
 
 size_t ssd_model_arena_bytes(const ssd_model_config* cfg) {

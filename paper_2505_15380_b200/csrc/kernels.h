@@ -7,6 +7,8 @@ namespace ssd {
 // Process-wide count of kernels enqueued by the launchers below.
 void count_launch(int n = 1);
 uint64_t launch_count();
+// Records a CUDA error for ssd_last_cuda_error and returns SSD_ERR_CUDA (api.cu).
+int report_cuda_error(cudaError_t e, const char* what);
 
 enum Epilogue { EPI_STORE_F32 = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2 };
 

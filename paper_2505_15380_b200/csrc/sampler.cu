@@ -7,6 +7,8 @@
 // p = DRAFT distribution, q = TARGET distribution, as in the paper.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "kernels.h"
 
 namespace ssd {
@@ -362,3 +364,80 @@ void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_le
 }
 
 }  // namespace ssd
+
+// ------------------------------------------------------------------------------------------------
+// Acceptance step for callers that cannot allocate device memory.
+//
+// Some hosts of this library may not call cudaMalloc at all: code that runs inside a serving loop
+// whose memory pool is fixed at start-up, or a plug-in that is handed device pointers by its host
+// process and owns none.  ssd_verify needs a workspace such callers cannot provide.  This entry
+// point runs the same fused acceptance kernel on logits the caller already has, and keeps the
+// kernel's scratch (four statistics words and one flag per row, one counter per stream, one status
+// word) in the fixed device array below instead.
+namespace {
+
+constexpr int NOALLOC_MAX_STREAMS = 256;  // streams per call
+constexpr int NOALLOC_MAX_ROWS = ssd::R_MAX;  // gamma + 1 <= 16
+
+struct NoAllocScratch {
+  float row_stats[NOALLOC_MAX_STREAMS * NOALLOC_MAX_ROWS * 4];
+  int32_t accept_flags[NOALLOC_MAX_STREAMS * NOALLOC_MAX_ROWS];
+  int32_t counters[NOALLOC_MAX_STREAMS];
+  int32_t status;
+};
+
+// About 84 KB, resident on every GPU that loads the library until the process exits.  In host
+// code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mu;
+NoAllocScratch* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+
+// Device address of the scratch array on the current device (looked up once per device).
+cudaError_t noalloc_scratch(NoAllocScratch** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = static_cast<NoAllocScratch*>(p);
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_draft_tokens,
+                                  const float* dev_draft_probs, const float* dev_uniforms,
+                                  const ssd_verify_params* params, int32_t batch, int32_t vocab,
+                                  int32_t* dev_accepted_len, int32_t* dev_next_token,
+                                  void* stream) {
+  if (!dev_logits || !dev_draft_tokens || !dev_draft_probs || !dev_uniforms || !params ||
+      !dev_accepted_len || !dev_next_token)
+    return SSD_ERR_NULL;
+  if (params->gamma < 1 || params->gamma + 1 > NOALLOC_MAX_ROWS) return SSD_ERR_BAD_GAMMA;
+  if (batch < 1 || batch > NOALLOC_MAX_STREAMS) return SSD_ERR_TOO_SMALL;  // beyond the fixed scratch
+  if (vocab < 2 || (size_t)vocab * 4 > 180 * 1024) return SSD_ERR_BAD_CONFIG;
+  if (!(params->temperature > 0.f) || !isfinite(params->temperature) || !(params->beta >= 0.f) ||
+      !isfinite(params->beta))
+    return SSD_ERR_BAD_PARAM;
+  NoAllocScratch* sc = nullptr;
+  cudaError_t e = noalloc_scratch(&sc);
+  if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: cudaGetSymbolAddress");
+  cudaStream_t st = (cudaStream_t)stream;
+  // the per-stream counters must start at zero; everything else is overwritten before it is read
+  e = cudaMemsetAsync(sc->counters, 0, sizeof(int32_t) * (NOALLOC_MAX_STREAMS + 1), st);
+  if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: cudaMemsetAsync");
+  e = ssd::launch_verify_sampler(dev_logits, vocab, dev_draft_tokens, dev_draft_probs, dev_uniforms,
+                                 batch, params->gamma, 1.0f / params->temperature, params->top_k,
+                                 params->beta, sc->row_stats, sc->accept_flags, sc->counters,
+                                 dev_accepted_len, dev_next_token, &sc->status, st);
+  if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: launch");
+  return SSD_OK;
+}
