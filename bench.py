@@ -172,7 +172,7 @@ def run_cuda(args):
     del w
     cap = max(wl.prefix_lens) + 2 * R + 8
     gs = binding.Streams(model, B, cap, g)
-    if max(wl.prefix_lens) <= 512:
+    if max(wl.prefix_lens) <= 512 and not args.synthetic_kv:
         gs.prefill([synth.make_prefix(wl, b) for b in range(B)])
     else:           # long prefixes: seeded random K/V written straight into the cache
         lens = [n - 1 for n in wl.prefix_lens]
@@ -333,6 +333,8 @@ def main():
     ap.add_argument("--beta", type=float, default=0.4)
     ap.add_argument("--draft-noise", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--synthetic-kv", action="store_true",
+                    help="seed the prefix K/V with noise instead of running a prefill (short profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
