@@ -62,7 +62,9 @@ enum {
   SSD_STATUS_KV_OVERFLOW = 1, /* len + rows > capacity: rows beyond capacity were not written */
   SSD_STATUS_BAD_TOKEN = 2,   /* a token id outside the embedding table was clamped */
   SSD_STATUS_NONFINITE = 4,   /* a logit row held NaN/Inf */
-  SSD_STATUS_BAD_PROB = 8     /* a draft probability p_i(x_i) was negative or not finite */
+  SSD_STATUS_BAD_PROB = 8,    /* a draft probability p_i(x_i) was negative or not finite */
+  SSD_STATUS_TIMEOUT = 16     /* a bounded wait inside a kernel ran out; the streams object refuses
+                                 further small-batch launches until it is created anew */
 };
 
 /* Decoder shape: the "Transformer adapted from Qwen2.5" of Sec. 3.1 (pre-norm RMSNorm, GQA with
@@ -113,6 +115,21 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
                        int32_t max_gamma, void* dev_kv, size_t kv_bytes, void* dev_workspace,
                        size_t ws_bytes, ssd_streams** out);
 void ssd_streams_destroy(ssd_streams* s);
+
+/* Which kernels run the decoder forward (Eq. 4) for these streams.  path 0 (default): forwards of
+ * at most 16 rows over a bf16 model run in one persistent kernel (one CTA per SM, weights streamed
+ * through shared-memory rings), larger ones in the generic per-operation kernels; path 1: generic
+ * kernels only.  Both produce the same results up to fp32 summation order. */
+int ssd_streams_set_path(ssd_streams* s, int32_t path);
+
+/* Phase trace of the persistent kernel (a profiling aid, not part of the method).  With a device
+ * buffer of ctas x events_per_cta int64 (ctas >= 256), thread 0 of every CTA stores its SM clock
+ * (clock64) at each phase boundary of every later small-batch forward: after set-up, after the
+ * embedding, after its grid barrier, then after each phase (per layer QKV, attention, O, gate/up,
+ * down; finally the LM head) and after the barrier that follows it.  Event i of CTA c lands at
+ * dev_trace[c * events_per_cta + i]; later launches overwrite earlier ones.  Clocks of different
+ * SMs are not synchronised: compare within a CTA.  dev_trace = NULL turns the trace off. */
+int ssd_streams_set_trace(ssd_streams* s, int64_t* dev_trace, int32_t ctas, int32_t events_per_cta);
 
 /* Explicit rollback / state load: len[b] = host_len[b], pending[b] = host_pending[b].
  * O(1) per stream, no cache data moves.  Synchronous with respect to `stream`. */

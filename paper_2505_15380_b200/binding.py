@@ -19,7 +19,8 @@ _lib = None
 
 EXPORTS = [
     "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
-    "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_kv_truncate",
+    "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_streams_set_path",
+    "ssd_streams_set_trace", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
     L.ssd_streams_create.argtypes = [vp, i32, i32, i32, vp, sz, vp, sz, ctypes.POINTER(vp)]
     L.ssd_streams_destroy.restype = None
     L.ssd_streams_destroy.argtypes = [vp]
+    L.ssd_streams_set_path.argtypes = [vp, i32]
+    L.ssd_streams_set_trace.argtypes = [vp, vp, i32, i32]
     L.ssd_kv_truncate.argtypes = [vp, vp, vp, vp]
     L.ssd_streams_get_state.argtypes = [vp, vp, vp, vp]
     L.ssd_prefill.argtypes = [vp, vp, vp, vp, vp]
@@ -172,6 +175,20 @@ class Streams:
         if getattr(self, "handle", None) is not None and _lib is not None:
             _lib.ssd_streams_destroy(self.handle)
             self.handle = None
+
+    def set_path(self, path: int) -> None:
+        """0: persistent small-batch kernel where the forward fits it (default); 1: generic kernels."""
+        check(lib().ssd_streams_set_path(self.handle, path))
+
+    def set_trace(self, buf: Optional[torch.Tensor]) -> None:
+        """buf: int64 CUDA tensor [ctas >= 256, events_per_cta] that receives the persistent
+        kernel's phase-boundary clocks, or None to turn the trace off."""
+        if buf is None:
+            check(lib().ssd_streams_set_trace(self.handle, None, 0, 0))
+        else:
+            assert buf.dtype == torch.int64 and buf.is_cuda and buf.is_contiguous() and buf.dim() == 2
+            check(lib().ssd_streams_set_trace(self.handle, buf.data_ptr(), buf.shape[0], buf.shape[1]))
+        self._trace = buf
 
     # -- state ------------------------------------------------------------------------------
     def kv_truncate(self, lens: Sequence[int], pending: Sequence[int], stream=None) -> None:

@@ -6,6 +6,7 @@
 
 #include <new>
 
+#include "fast.h"
 #include "kernels.h"
 
 using namespace ssd;
@@ -47,9 +48,25 @@ struct LayerOff {
 struct ArenaPlan {
   size_t embed, norm_f, head, inv_freq, total;
   std::vector<LayerOff> layers;
+  // weights packed for the persistent small-batch kernel (bf16 models only)
+  bool fast;
+  size_t f_stream, f_stream_off, f_chunks, f_chunk_cnt, f_unit_cnt, f_unit_off, f_unit_tile, f_bias,
+      f_gains;
 };
 
-ArenaPlan plan_arena(const ssd_model_config& c) {
+// CTAs of the persistent kernel: one per SM of the current device (148 when none is present, the
+// SM count of a B200, so that sizes can be computed without a GPU).
+int fast_cta_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+    cudaGetLastError();
+    return 148;
+  }
+  return sms > FAST_MAX_CTAS ? FAST_MAX_CTAS : sms;
+}
+
+ArenaPlan plan_arena(const ssd_model_config& c, const FastPlan* fp = nullptr) {
   ArenaPlan p;
   size_t el = c.weight_dtype == 0 ? 4 : 2, off = 0;
   size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
@@ -69,6 +86,24 @@ ArenaPlan plan_arena(const ssd_model_config& c) {
   p.norm_f = take(d * el);
   p.head = take((size_t)c.vocab_out * d * el);
   p.inv_freq = take((size_t)(c.head_dim / 2) * sizeof(double));
+  p.fast = fast_supported(c);
+  if (p.fast) {
+    FastPlan local;
+    if (!fp) {
+      local = fast_make_plan(c, fast_cta_count());
+      fp = &local;
+    }
+    const size_t nq = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+    p.f_stream = take(fp->total_bytes);
+    p.f_stream_off = take(fp->stream_off.size() * 8);
+    p.f_chunks = take(fp->chunks.size());
+    p.f_chunk_cnt = take(fp->chunk_cnt.size() * 4);
+    p.f_unit_cnt = take(fp->unit_cnt.size() * 4);
+    p.f_unit_off = take(fp->unit_off.size() * 4);
+    p.f_unit_tile = take(fp->unit_tile.size() * 4);
+    p.f_bias = take((size_t)c.n_layers * nq * 4);
+    p.f_gains = take(((size_t)c.n_layers * 2 + 1) * d * 4);
+  }
   p.total = off;
   return p;
 }
@@ -84,6 +119,7 @@ struct WsPlan {
   size_t len, pending, status, counters, row_ids, accept_flags;
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
+  size_t hfix, fpart, attn_counters, flags, epoch_base;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -118,6 +154,11 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.st_y = take(B * 4);
   p.st_probs = take((size_t)B * max_gamma * V * 4);
   p.st_uni = take(M * 2 * 4);
+  p.hfix = take((size_t)FAST_MAX_T * d * 8);
+  p.fpart = take((size_t)FAST_MAX_T * c.n_q_heads * FAST_NSPLIT_CAP * (c.head_dim + 2) * 4);
+  p.attn_counters = take((size_t)FAST_MAX_T * c.n_q_heads * 4);
+  p.flags = take(64);
+  p.epoch_base = take(2 * 4);
   p.total = off;
   return p;
 }
@@ -136,7 +177,71 @@ bool same_shape(const ssd_model_config& a, const ssd_model_config& b) {
 
 // One decoder forward over the rows described by rm (ids already in s->row_ids).  Appends the
 // rows' K/V at len + r; when logits_out is non-null also runs the final norm and the LM head.
+// The persistent kernel covers forwards of at most FAST_MAX_T rows over a bf16 model.
+bool use_fast(const ssd_model* m, const ssd_streams* s, RowMap rm) {
+  return m->fast.enabled && s->path == 0 && rm.nb * rm.R <= FAST_MAX_T;
+}
+
+int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* row_ids,
+                 const int32_t* draft_tokens, float* logits_out, cudaStream_t st) {
+  const ssd_model_config& c = m->cfg;
+  const ssd_fast_model& f = m->fast;
+  FastParams p{};
+  p.m.wstream = f.wstream;
+  p.m.stream_off = f.stream_off;
+  p.m.chunks = f.chunks;
+  p.m.chunk_cnt = f.chunk_cnt;
+  p.m.unit_cnt = f.unit_cnt;
+  p.m.unit_off = f.unit_off;
+  p.m.unit_tile = f.unit_tile;
+  p.m.bias_qkv = f.bias_qkv;
+  p.m.gains = f.gains;
+  p.m.n_cta = f.n_cta;
+  p.m.max_units = f.max_units;
+  p.m.down_split = f.down_split;
+  p.m.max_stage_k = f.max_stage_k;
+  p.embed = (const bf16*)m->embed;
+  p.inv_freq = m->inv_freq;
+  p.L = c.n_layers;
+  p.d = c.d_model;
+  p.Hq = c.n_q_heads;
+  p.Hkv = c.n_kv_heads;
+  p.hd = c.head_dim;
+  p.hd_shift = c.head_dim == 32 ? 5 : c.head_dim == 64 ? 6 : 7;
+  p.F = c.d_ffn;
+  p.V = c.vocab_out;
+  p.vocab_in = c.vocab_out + c.vocab_text;
+  p.eps = c.rms_eps;
+  p.kv = (bf16*)s->kv;
+  p.kv_layer_elems = s->kv_layer_elems;
+  p.cap = s->cap;
+  p.len = s->len;
+  p.pending = s->pending;
+  p.status = s->status;
+  p.b0 = rm.b0;
+  p.nb = rm.nb;
+  p.R = rm.R;
+  p.T = rm.nb * rm.R;
+  p.row_ids = row_ids;
+  p.draft_tokens = draft_tokens;
+  p.hfix = s->hfix;
+  p.qrot = s->qrot;
+  p.attn_out = s->attn_out;
+  p.act = s->act;
+  p.rope_cs = s->rope_cs;
+  p.part = s->fpart;
+  p.logits = logits_out;
+  p.attn_counters = s->attn_counters;
+  p.flags = s->flags;
+  p.epoch_base = s->epoch_base;
+  p.trace = s->trace;
+  p.trace_cap = s->trace_cap;
+  SSD_CUDA(launch_fast_forward(p, st));
+  return SSD_OK;
+}
+
 int forward(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cudaStream_t st) {
+  if (use_fast(m, s, rm)) return forward_fast(m, s, rm, s->row_ids, nullptr, logits_out, st);
   const ssd_model_config& c = m->cfg;
   const int dt = c.weight_dtype, M = rm.nb * rm.R, d = c.d_model;
   const int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn;
@@ -197,7 +302,10 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
   if (!cfg_ok(cfg)) return SSD_ERR_BAD_CONFIG;
   if ((uintptr_t)dev_arena & 255) return SSD_ERR_MISALIGNED;
   const ssd_model_config& c = *cfg;
-  ArenaPlan p = plan_arena(c);
+  FastPlan fplan;
+  const bool fast = fast_supported(c);
+  if (fast) fplan = fast_make_plan(c, fast_cta_count());
+  ArenaPlan p = plan_arena(c, fast ? &fplan : nullptr);
   const size_t el = c.weight_dtype == 0 ? 4 : 2;
   if (arena_bytes < p.total) return SSD_ERR_TOO_SMALL;
   if (nbytes != blob_elems(c) * el) return SSD_ERR_BAD_CONFIG;
@@ -250,6 +358,48 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
   if (e == cudaSuccess)
     e = cudaMemcpy(A + p.inv_freq, inv.data(), inv.size() * sizeof(double), cudaMemcpyHostToDevice);
   m->inv_freq = (const double*)(A + p.inv_freq);
+  if (fast && e == cudaSuccess) {
+    // second copy of the projection weights, tiled and ordered for the persistent kernel
+    std::vector<uint8_t> packed(fplan.total_bytes);
+    std::vector<float> bias, gains;
+    fast_pack_streams(c, fplan, (const uint16_t*)host_weights, packed.data());
+    fast_pack_aux(c, (const uint16_t*)host_weights, bias, gains);
+    auto up = [&](size_t dst_off, const void* srcp, size_t bytes) {
+      if (e == cudaSuccess && bytes) e = cudaMemcpy(A + dst_off, srcp, bytes, cudaMemcpyHostToDevice);
+    };
+    up(p.f_stream, packed.data(), packed.size());
+    up(p.f_stream_off, fplan.stream_off.data(), fplan.stream_off.size() * 8);
+    up(p.f_chunks, fplan.chunks.data(), fplan.chunks.size());
+    up(p.f_chunk_cnt, fplan.chunk_cnt.data(), fplan.chunk_cnt.size() * 4);
+    up(p.f_unit_cnt, fplan.unit_cnt.data(), fplan.unit_cnt.size() * 4);
+    up(p.f_unit_off, fplan.unit_off.data(), fplan.unit_off.size() * 4);
+    up(p.f_unit_tile, fplan.unit_tile.data(), fplan.unit_tile.size() * 4);
+    up(p.f_bias, bias.data(), bias.size() * 4);
+    up(p.f_gains, gains.data(), gains.size() * 4);
+    ssd_fast_model& f = m->fast;
+    f.wstream = (const uint8_t*)(A + p.f_stream);
+    f.stream_off = (const uint64_t*)(A + p.f_stream_off);
+    f.chunks = (const uint8_t*)(A + p.f_chunks);
+    f.chunk_cnt = (const int32_t*)(A + p.f_chunk_cnt);
+    f.unit_cnt = (const int32_t*)(A + p.f_unit_cnt);
+    f.unit_off = (const int32_t*)(A + p.f_unit_off);
+    f.unit_tile = (const int32_t*)(A + p.f_unit_tile);
+    f.bias_qkv = (const float*)(A + p.f_bias);
+    f.gains = (const float*)(A + p.f_gains);
+    f.n_cta = fplan.n_cta;
+    f.down_split = fplan.ops[FOP_DOWN].ksplit;
+    f.max_units = 0;
+    for (int32_t v : fplan.unit_cnt) f.max_units = v > f.max_units ? v : f.max_units;
+    int down_w = 0;
+    for (int cta = 0; cta < fplan.n_cta; ++cta) {
+      int w = (fast_slice_k1(fplan.ops[FOP_DOWN], cta) - fast_slice_k0(fplan.ops[FOP_DOWN], cta)) * 16;
+      down_w = w > down_w ? w : down_w;
+    }
+    f.max_stage_k = c.d_model;
+    if (c.n_q_heads * c.head_dim > f.max_stage_k) f.max_stage_k = c.n_q_heads * c.head_dim;
+    if (down_w > f.max_stage_k) f.max_stage_k = down_w;
+    f.enabled = f.max_units <= FAST_MAX_UNITS && fplan.max_chunks <= FAST_MAX_CHUNKS;
+  }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete m;
@@ -320,11 +470,34 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->st_y = (int32_t*)(W + p.st_y);
   s->st_probs = (float*)(W + p.st_probs);
   s->st_uni = (float*)(W + p.st_uni);
+  s->hfix = (long long*)(W + p.hfix);
+  s->fpart = (float*)(W + p.fpart);
+  s->attn_counters = (int32_t*)(W + p.attn_counters);
+  s->flags = (uint32_t*)(W + p.flags);
+  s->epoch_base = (uint32_t*)(W + p.epoch_base);
+  s->path = 0;
+  s->trace = nullptr;
+  s->trace_cap = 0;
   *out = s;
   return SSD_OK;
 }
 
 void ssd_streams_destroy(ssd_streams* s) { delete s; }
+
+int ssd_streams_set_path(ssd_streams* s, int32_t path) {
+  if (!s) return SSD_ERR_NULL;
+  if (path != 0 && path != 1) return SSD_ERR_BAD_PARAM;
+  s->path = path;
+  return SSD_OK;
+}
+
+int ssd_streams_set_trace(ssd_streams* s, int64_t* dev_trace, int32_t ctas, int32_t events_per_cta) {
+  if (!s) return SSD_ERR_NULL;
+  if (dev_trace && (ctas < FAST_MAX_CTAS || events_per_cta < 1)) return SSD_ERR_TOO_SMALL;
+  s->trace = (long long*)dev_trace;
+  s->trace_cap = dev_trace ? events_per_cta : 0;
+  return SSD_OK;
+}
 
 int ssd_kv_truncate(ssd_streams* s, const int32_t* host_len, const int32_t* host_pending,
                     void* stream) {
@@ -416,8 +589,13 @@ int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_token
   cudaStream_t st = (cudaStream_t)stream;
   const int gamma = params->gamma;
   float* logits = dev_logits_or_null ? dev_logits_or_null : s->logits;
-  launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
-  rc = forward(target, s, RowMap{0, s->B, gamma + 1}, logits, st);
+  const RowMap rm{0, s->B, gamma + 1};
+  if (use_fast(target, s, rm)) {
+    rc = forward_fast(target, s, rm, nullptr, dev_draft_tokens, logits, st);
+  } else {
+    launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
+    rc = forward(target, s, rm, logits, st);
+  }
   if (rc != SSD_OK) return rc;
   SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
                                  dev_uniforms, s->B, gamma, 1.0f / params->temperature,

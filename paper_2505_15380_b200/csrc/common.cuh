@@ -74,6 +74,17 @@ struct LayerW {
 
 }  // namespace ssd
 
+// Device-side view of the weights packed for the persistent small-batch kernel (fast.h).
+struct ssd_fast_model {
+  bool enabled = false;
+  const uint8_t* wstream = nullptr;
+  const uint64_t* stream_off = nullptr;
+  const uint8_t* chunks = nullptr;
+  const int32_t *chunk_cnt = nullptr, *unit_cnt = nullptr, *unit_off = nullptr, *unit_tile = nullptr;
+  const float *bias_qkv = nullptr, *gains = nullptr;
+  int n_cta = 0, max_units = 0, down_split = 1, max_stage_k = 0;
+};
+
 struct ssd_model {
   ssd_model_config cfg;
   int el;  // bytes per weight element
@@ -82,6 +93,7 @@ struct ssd_model {
   std::vector<ssd::LayerW> layers;
   const void *norm_f, *head;
   const double* inv_freq;  // [head_dim / 2]
+  ssd_fast_model fast;
 };
 
 struct ssd_streams {
@@ -98,4 +110,13 @@ struct ssd_streams {
   // staging for the host-buffer entry point
   int32_t *st_tokens, *st_k, *st_y;
   float *st_probs, *st_uni;
+  // persistent small-batch kernel: fixed-point residual stream, attention partials and counters,
+  // grid-barrier words
+  long long* hfix;
+  float* fpart;
+  int32_t* attn_counters;
+  uint32_t *flags, *epoch_base;
+  int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
+  long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)
+  int trace_cap;
 };
