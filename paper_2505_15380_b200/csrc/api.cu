@@ -119,7 +119,7 @@ struct WsPlan {
   size_t len, pending, status, counters, row_ids, accept_flags;
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
-  size_t hfix, fpart, attn_counters, flags, epoch_base;
+  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, ssq_a, ssq_b, tile_cnt;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -155,6 +155,14 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.st_probs = take((size_t)B * max_gamma * V * 4);
   p.st_uni = take(M * 2 * 4);
   p.hfix = take((size_t)FAST_MAX_T * d * 8);
+  // operand-layout activations: per 16 columns 32 lanes x 32 bytes (16 rows, bf16 hi + lo)
+  p.xa = take(d * 64);
+  p.xb = take(d * 64);
+  p.xo = take(qd * 64);
+  p.xd = take(F * 64);
+  p.ssq_a = take((d / 8 + 1) * FAST_MAX_T * 4);
+  p.ssq_b = take((d / 8 + 1) * FAST_MAX_T * 4);
+  p.tile_cnt = take((d / 8 + 1) * 4);
   p.fpart = take((size_t)FAST_MAX_T * c.n_q_heads * FAST_NSPLIT_CAP * (c.head_dim + 2) * 4);
   p.attn_counters = take((size_t)FAST_MAX_T * c.n_q_heads * 4);
   p.flags = take(64);
@@ -226,9 +234,14 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.draft_tokens = draft_tokens;
   p.hfix = s->hfix;
   p.qrot = s->qrot;
-  p.attn_out = s->attn_out;
-  p.act = s->act;
   p.rope_cs = s->rope_cs;
+  p.xa = s->xa;
+  p.xb = s->xb;
+  p.xo = s->xo;
+  p.xd = s->xd;
+  p.ssq_a = s->ssq_a;
+  p.ssq_b = s->ssq_b;
+  p.tile_cnt = s->tile_cnt;
   p.part = s->fpart;
   p.logits = logits_out;
   p.attn_counters = s->attn_counters;
@@ -471,6 +484,13 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->st_probs = (float*)(W + p.st_probs);
   s->st_uni = (float*)(W + p.st_uni);
   s->hfix = (long long*)(W + p.hfix);
+  s->xa = (uint32_t*)(W + p.xa);
+  s->xb = (uint32_t*)(W + p.xb);
+  s->xo = (uint32_t*)(W + p.xo);
+  s->xd = (uint32_t*)(W + p.xd);
+  s->ssq_a = (float*)(W + p.ssq_a);
+  s->ssq_b = (float*)(W + p.ssq_b);
+  s->tile_cnt = (int32_t*)(W + p.tile_cnt);
   s->fpart = (float*)(W + p.fpart);
   s->attn_counters = (int32_t*)(W + p.attn_counters);
   s->flags = (uint32_t*)(W + p.flags);

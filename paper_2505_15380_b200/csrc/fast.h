@@ -18,7 +18,10 @@
 
 namespace ssd {
 
-constexpr int FAST_WARPS = 8;         // warps per CTA; they split K of every projection
+#ifndef SSD_FAST_WARPS
+#define SSD_FAST_WARPS 8
+#endif
+constexpr int FAST_WARPS = SSD_FAST_WARPS;  // warps per CTA; they split K of every projection
 constexpr int FAST_THREADS = FAST_WARPS * 32;
 constexpr int FAST_TILE_BYTES = 256;  // one operand tile: 8 weight rows x 16 k, bf16
 constexpr int FAST_SLOT_TILES = 8;    // a ring slot holds one chunk of at most this many tiles
@@ -124,7 +127,14 @@ struct FastParams {
   const int32_t* draft_tokens;  // [B, gamma] when row_ids is null
   // workspace
   long long* hfix;  // residual stream [T][d] in 2^-32 fixed point (order-independent accumulation)
-  float *qrot, *attn_out, *act, *rope_cs, *part, *logits;  // logits null: skip the LM head
+  float *qrot, *rope_cs, *part, *logits;  // logits null: skip the LM head
+  // Inputs of the projections, written by their producers already in the tensor-core operand layout
+  // (bf16 leading part + remainder, see fast_verify.cu): the RMS-norm inputs x * gain of the QKV /
+  // LM-head projection (xa) and of gate/up (xb), the attention output (xo), SiLU(g) * u (xd); and
+  // per 8-column tile and row the sums of squares that go with xa / xb.
+  uint32_t *xa, *xb, *xo, *xd;
+  float *ssq_a, *ssq_b;   // [d / 8][FAST_MAX_T]
+  int32_t* tile_cnt;      // [d / 8] arrivals of the down projection's K slices per output tile
   int32_t* attn_counters;
   uint32_t* flags;       // [0] grid-barrier arrival counter, monotonic across launches
   uint32_t* epoch_base;  // [0] counter value at the start of the next launch, [1] nonzero after a failure

@@ -31,7 +31,7 @@ namespace ssd {
 namespace {
 
 constexpr unsigned long long FAST_WAIT_CYCLES = 3000000000ull;  // ~1.5 s at 2 GHz
-constexpr int FAST_KEYS_MIN = 64;                                // fewest keys worth a split of their own
+constexpr int FAST_KEYS_MIN = 32;                                // fewest keys worth a split of their own
 constexpr float FIX_SCALE = 4294967296.f;                        // residual stream: 2^-32 fixed point
 constexpr float FIX_INV_SCALE = 1.f / 4294967296.f;
 
@@ -175,6 +175,18 @@ __device__ __forceinline__ void ring_release(Ring& r, int lane) {
   }
 }
 
+#ifdef SSD_TRACE_FINE
+// debug build: every warp's clock at marked points of one layer, kept in shared memory
+__shared__ unsigned int g_wtr[FAST_WARPS][96];
+__shared__ int g_wtr_on;
+#define WMARK(i)                                                                         \
+  do {                                                                                   \
+    if (g_wtr_on && (threadIdx.x & 31) == 0) g_wtr[threadIdx.x >> 5][(i)] = (unsigned)clock64(); \
+  } while (0)
+#else
+#define WMARK(i) do {} while (0)
+#endif
+
 __device__ __forceinline__ void trace_mark(const FastParams& P, int& n_trace) {
   if (P.trace && threadIdx.x == 0 && n_trace < P.trace_cap)
     P.trace[(size_t)blockIdx.x * P.trace_cap + n_trace++] = clock64();
@@ -216,143 +228,94 @@ __device__ __noinline__ bool grid_sync(const FastParams& P, uint32_t target, boo
 
 // One projection of the layer: which weights, which input, which epilogue.
 struct PhaseDesc {
-  const void* in;     // input rows (fixed-point residual stream when in_fix, else fp32)
-  const float* gain;  // RMSNorm gain (in_fix only)
-  int op;             // FOP_*: whose tiles of this CTA
-  int epi;            // EPI_F_*
-  int in_fix;
-  int ld, kb, kc;     // input row stride; first column and number of columns this CTA covers
-  int n_rows;         // valid weight rows (the last tile of the LM head is padded)
+  const uint32_t* xin;  // operand-layout input, at this CTA's first k-step
+  const float* ssq_in;  // with in_fix: the per-tile sums of squares of the input rows
+  int op;               // FOP_*: whose tiles of this CTA
+  int epi;              // EPI_F_*
+  int in_fix;           // the input is x * gain of an RMS norm: scale the outputs by inv_rms[row]
+  int kc;               // input columns this CTA covers
+  int n_rows;           // valid weight rows (the last tile of the LM head is padded)
   int layer;
-  bf16* kv_layer;     // this layer's slice of the cache (QKV epilogue)
-  float qscale;       // 1 / sqrt(head_dim)
+  bf16* kv_layer;       // this layer's slice of the cache (QKV epilogue)
+  float qscale;         // 1 / sqrt(head_dim)
+  // residual epilogues: the operand the finished rows become for the next projection
+  uint32_t* xout;
+  float* ssq_out;
+  const float* gain_next;
+  int nsplit;           // K slices (CTAs) adding into the same output tile (1: a single writer)
 };
 
-// Shared-memory image of the A operand: for k-step s and lane l (g = l / 4, t = l % 4) 16 bytes
+// Operand layout of the activations (the A operand of the projections), in global memory where a
+// producer writes it and in shared memory where the consumers copy it: for k-step s and lane l
+// (g = l / 4, t = l % 4) 16 bytes
 //   { hi(x[g][16s+2t..]), hi(x[g][16s+8+2t..]), lo(same), lo(same) }
-// and, when more than 8 rows are in flight, 16 more bytes for row g + 8.
+// (hi = bf16 leading part, lo = bf16 of the remainder) and, when more than 8 rows are in flight,
+// 16 more bytes for row g + 8.  Every value is converted once, by the thread that produces it,
+// instead of once per consuming CTA.
 template <bool T16>
 __device__ __forceinline__ uint32_t afrag_word(int row, int kk) {  // kk = column pair index
   constexpr int W = T16 ? 8 : 4;
   const int s = kk >> 3, t = kk & 3, which = (kk >> 2) & 1;
   return (uint32_t)(((s * 32 + (row & 7) * 4 + t) * W) + (row >> 3) * 4 + which);
 }
+// Columns (k, k + 1), k even, of row `row`.
+template <bool T16>
+__device__ __forceinline__ void write_frag_pair(uint32_t* buf, int row, int k, float x0, float x1) {
+  uint32_t hi, lo;
+  split2(x0, x1, hi, lo);
+  const uint32_t wd = afrag_word<T16>(row, k >> 1);
+  buf[wd] = hi;
+  buf[wd + 2] = lo;
+}
+// One column of row `row` (two 2-byte stores).
+template <bool T16>
+__device__ __forceinline__ void write_frag_elem(uint32_t* buf, int row, int k, float x) {
+  const bf16 h = __float2bfloat16_rn(x);
+  const bf16 l = __float2bfloat16_rn(x - __bfloat162float(h));
+  bf16* w = reinterpret_cast<bf16*>(buf + afrag_word<T16>(row, k >> 1)) + (k & 1);
+  w[0] = h;
+  w[4] = l;  // two words on
+}
 
-// Residual-stream rows -> A operand of x * gain, and the rows' sums of squares, for inputs of at
-// most J * 2 * FAST_THREADS columns.  All loads of a batch of rows are in flight before the first
-// is used.
-template <int J, bool T16>
-__device__ __forceinline__ void stage_fix_rows(const longlong2* __restrict__ hin,
-                                               const float2* __restrict__ gain2, uint32_t* af,
-                                               FastMisc& M, int T, int half_k, int ld2, int tid) {
-  constexpr int RB = 16 / J;  // rows per batch
-  const int lane = tid & 31, warp = tid >> 5;
-  float2 gj[J];
+// Copies `nsteps` k-steps of an operand-layout input from global memory (written by other CTAs in
+// an earlier phase, hence read past L1) to shared memory.  All loads are in flight before the
+// first store.
+template <bool T16>
+__device__ __forceinline__ void stage_copy(const uint32_t* __restrict__ src, uint32_t* af, int nsteps) {
+  constexpr int LB = 8;
+  const int n16 = nsteps * (T16 ? 64 : 32);
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(af);
+  for (int i0 = threadIdx.x; i0 < n16; i0 += LB * FAST_THREADS) {
+    uint4 v[LB];
 #pragma unroll
-  for (int j = 0; j < J; ++j) {
-    const int kk = j * FAST_THREADS + tid;
-    gj[j] = kk < half_k ? __ldg(gain2 + kk) : make_float2(0.f, 0.f);
-  }
-  for (int r0 = 0; r0 < T; r0 += RB) {
-    longlong2 hv[RB][J];
+    for (int i = 0; i < LB; ++i)
+      if (i0 + i * FAST_THREADS < n16) v[i] = __ldcg(s4 + i0 + i * FAST_THREADS);
 #pragma unroll
-    for (int rr = 0; rr < RB; ++rr) {
-#pragma unroll
-      for (int j = 0; j < J; ++j) {
-        const int kk = j * FAST_THREADS + tid;
-        if (r0 + rr < T && kk < half_k) hv[rr][j] = __ldcg(hin + (r0 + rr) * ld2 + kk);
-      }
-    }
-#pragma unroll
-    for (int rr = 0; rr < RB; ++rr) {
-      const int row = r0 + rr;
-      if (row < T) {
-        float ss = 0.f;
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-          const int kk = j * FAST_THREADS + tid;
-          if (kk < half_k) {
-            const float x0 = fix_to_float(hv[rr][j].x), x1 = fix_to_float(hv[rr][j].y);
-            ss = fmaf(x0, x0, fmaf(x1, x1, ss));
-            uint32_t hi, lo;
-            split2(x0 * gj[j].x, x1 * gj[j].y, hi, lo);
-            const uint32_t wd = afrag_word<T16>(row, kk);
-            af[wd] = hi;
-            af[wd + 2] = lo;
-          }
-        }
-        ss = warp_sum(ss);
-        if (lane == 0) M.wred[warp][row] = ss;
-      }
-    }
+    for (int i = 0; i < LB; ++i)
+      if (i0 + i * FAST_THREADS < n16) d4[i0 + i * FAST_THREADS] = v[i];
   }
 }
 
-// Stages the input of a projection phase as the A operand in shared memory: columns
-// [kb, kb + kc) of an input with row stride `ld` (written by other CTAs in an earlier phase, hence
-// read past L1).  With in_fix the input is the fixed-point residual stream and the operand is
-// x * gain; the rows' sums of squares go to wred (the RMS scale is applied in the epilogue, which
-// is exact because it is one factor per token).
-template <bool T16>
-__device__ __noinline__ void stage_input(const FastParams& P, FastMisc& M, uint32_t* af,
-                                         const PhaseDesc& D) {
-  const int T = P.T, tid = threadIdx.x;
-  const int kc = D.kc, ld = D.ld;
-  if (D.in_fix) {
-    const longlong2* hin = static_cast<const longlong2*>(D.in);
-    const float2* gain2 = reinterpret_cast<const float2*>(D.gain);
-    const int half_k = kc >> 1, ld2 = ld >> 1;
-    if (half_k <= FAST_THREADS) stage_fix_rows<1, T16>(hin, gain2, af, M, T, half_k, ld2, tid);
-    else if (half_k <= 2 * FAST_THREADS) stage_fix_rows<2, T16>(hin, gain2, af, M, T, half_k, ld2, tid);
-    else if (half_k <= 4 * FAST_THREADS) stage_fix_rows<4, T16>(hin, gain2, af, M, T, half_k, ld2, tid);
-    else stage_fix_rows<16, T16>(hin, gain2, af, M, T, half_k, ld2, tid);
-  } else {
-    constexpr int LB = 8;
-    const float* fin = static_cast<const float*>(D.in) + D.kb;
-    const int c4 = kc >> 2;
-    // this thread's float4 elements: (row, col) advancing by FAST_THREADS columns with carry
-    int row_l = 0, col_l = tid;
-    while (col_l >= c4) { col_l -= c4; ++row_l; }
-    int row_u = row_l, col_u = col_l;
-    while (row_u < T) {
-      float4 v[LB];
-#pragma unroll
-      for (int i = 0; i < LB; ++i) {
-        if (row_l < T) v[i] = __ldcg(reinterpret_cast<const float4*>(fin + row_l * ld) + col_l);
-        col_l += FAST_THREADS;
-        while (col_l >= c4) { col_l -= c4; ++row_l; }
-      }
-#pragma unroll
-      for (int i = 0; i < LB; ++i) {
-        if (row_u < T) {
-          uint32_t h0, l0, h1, l1;
-          split2(v[i].x, v[i].y, h0, l0);
-          split2(v[i].z, v[i].w, h1, l1);
-          const uint32_t wd = afrag_word<T16>(row_u, 2 * col_u);  // pair 2c; pair 2c+1 is the next lane's
-          af[wd] = h0;
-          af[wd + 2] = l0;
-          af[wd + (T16 ? 8 : 4)] = h1;
-          af[wd + (T16 ? 8 : 4) + 2] = l1;
-        }
-        col_u += FAST_THREADS;
-        while (col_u >= c4) { col_u -= c4; ++row_u; }
-      }
-    }
+// inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
+// warp per row, fixed summation order.
+__device__ __forceinline__ void compute_inv_rms(const float* __restrict__ ssq, int ntiles, int T, int K,
+                                                float eps, FastMisc& M) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int row = warp; row < T; row += FAST_WARPS) {
+    float v = 0.f;
+    for (int tile = lane; tile < ntiles; tile += 32) v += __ldcg(ssq + tile * FAST_MAX_T + row);
+    v = warp_sum(v);
+    if (lane == 0) M.inv_rms[row] = rsqrtf(v / (float)K + eps);
   }
-  __syncthreads();
 }
 
 // One output element pair of a projection: token `tok`, packed weight rows n and n + 1.
+template <bool T16>
 __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDesc& D, const FastMisc& M,
                                               int tok, int n, float c0, float c1) {
-  if (D.epi == EPI_F_RESID) {
-    // 64-bit integer adds commute: the K slices of different CTAs may arrive in any order and the
-    // sum is still bit-reproducible
-    unsigned long long* dst = reinterpret_cast<unsigned long long*>(P.hfix + (size_t)tok * P.d + n);
-    atomicAdd(dst, (unsigned long long)__float2ll_rn(c0 * FIX_SCALE));
-    atomicAdd(dst + 1, (unsigned long long)__float2ll_rn(c1 * FIX_SCALE));
-  } else if (D.epi == EPI_F_SWIGLU) {
-    P.act[(size_t)tok * P.F + (n >> 1)] = c0 / (1.f + expf(-c0)) * c1;
+  if (D.epi == EPI_F_SWIGLU) {
+    write_frag_elem<T16>(P.xd, tok, n >> 1, __fdividef(c0, 1.f + __expf(-c0)) * c1);
   } else if (D.epi == EPI_F_LOGITS) {
     if (n < D.n_rows) P.logits[(size_t)tok * P.V + n] = c0;
     if (n + 1 < D.n_rows) P.logits[(size_t)tok * P.V + n + 1] = c1;
@@ -382,6 +345,80 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
       bf16* vdst = D.kv_layer + (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * hd + (size_t)pos * hd;
       *reinterpret_cast<__nv_bfloat162*>(vdst + jj) = __floats2bfloat162_rn(x1, x2);
     }
+  }
+}
+
+// Residual epilogue of one output tile (8 columns of h), collective over a warp: lane = (row g,
+// column pair t) adds its projection outputs to the fixed-point residual stream.  64-bit integer
+// adds commute, so the K slices of different CTAs may arrive in any order and the sum is still
+// bit-reproducible.  The warp that completes the tile (the only writer, or the last of the slices
+// to arrive) turns the finished rows into the operand of the next projection: x * gain as bf16
+// hi / lo in operand layout, plus the tile's sums of squares for the RMS norm.
+template <bool T16>
+__device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
+                                           const float* c) {
+  constexpr int NACC = T16 ? 4 : 2;
+  const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
+  const bool v0 = gg < T, v1 = T16 && gg + 8 < T;
+  long long* h0 = P.hfix + (size_t)gg * P.d + n;
+  long long* h1 = h0 + (size_t)8 * P.d;
+  longlong2 a = make_longlong2(0, 0), b = make_longlong2(0, 0);
+  if (D.nsplit > 1) {
+    if (v0) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(h0), (unsigned long long)__float2ll_rn(c[0] * FIX_SCALE));
+      atomicAdd(reinterpret_cast<unsigned long long*>(h0) + 1, (unsigned long long)__float2ll_rn(c[1] * FIX_SCALE));
+    }
+    if (v1) {
+      atomicAdd(reinterpret_cast<unsigned long long*>(h1), (unsigned long long)__float2ll_rn(c[NACC - 2] * FIX_SCALE));
+      atomicAdd(reinterpret_cast<unsigned long long*>(h1) + 1, (unsigned long long)__float2ll_rn(c[NACC - 1] * FIX_SCALE));
+    }
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) {
+      __threadfence();
+      last = atomicAdd(&P.tile_cnt[tile], 1) == D.nsplit - 1;
+      if (last) P.tile_cnt[tile] = 0;
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    __threadfence();
+    if (v0) a = __ldcg(reinterpret_cast<const longlong2*>(h0));
+    if (v1) b = __ldcg(reinterpret_cast<const longlong2*>(h1));
+  } else {
+    if (v0) {
+      a = __ldcg(reinterpret_cast<const longlong2*>(h0));
+      a.x += __float2ll_rn(c[0] * FIX_SCALE);
+      a.y += __float2ll_rn(c[1] * FIX_SCALE);
+      *reinterpret_cast<longlong2*>(h0) = a;
+    }
+    if (v1) {
+      b = __ldcg(reinterpret_cast<const longlong2*>(h1));
+      b.x += __float2ll_rn(c[NACC - 2] * FIX_SCALE);
+      b.y += __float2ll_rn(c[NACC - 1] * FIX_SCALE);
+      *reinterpret_cast<longlong2*>(h1) = b;
+    }
+  }
+  const float2 gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));
+  float s0 = 0.f, s1 = 0.f;
+  if (v0) {
+    const float x0 = fix_to_float(a.x), x1 = fix_to_float(a.y);
+    s0 = fmaf(x0, x0, x1 * x1);
+    write_frag_pair<T16>(D.xout, gg, n, x0 * gn.x, x1 * gn.y);
+  }
+  if (v1) {
+    const float x0 = fix_to_float(b.x), x1 = fix_to_float(b.y);
+    s1 = fmaf(x0, x0, x1 * x1);
+    write_frag_pair<T16>(D.xout, gg + 8, n, x0 * gn.x, x1 * gn.y);
+  }
+  s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
+  s0 += __shfl_xor_sync(0xffffffffu, s0, 2);
+  if (T16) {
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 2);
+  }
+  if (tt == 0) {
+    if (v0) D.ssq_out[tile * FAST_MAX_T + gg] = s0;
+    if (v1) D.ssq_out[tile * FAST_MAX_T + gg + 8] = s1;
   }
 }
 
@@ -433,8 +470,8 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
   }
 }
 
-// One projection phase: stage the input, run this CTA's tiles (the warps split K), add the warps'
-// partial sums in shared memory and apply the epilogue.
+// One projection phase: copy the input operand to shared memory, run this CTA's tiles (the warps
+// split K), add the warps' partial sums in shared memory and apply the epilogue.
 template <bool T16>
 __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
                                            const PhaseDesc& D) {
@@ -445,13 +482,12 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   const int KS = D.kc >> 4;
   uint32_t* af = reinterpret_cast<uint32_t*>(uni);                             // A operand, KS steps
   float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
-  stage_input<T16>(P, M, af, D);
-  if (D.in_fix && tid < T) {
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < FAST_WARPS; ++w) tot += M.wred[w][tid];
-    M.inv_rms[tid] = rsqrtf(tot / (float)D.kc + P.eps);
-  }
+  WMARK(D.op * 10 + 0);
+  stage_copy<T16>(D.xin, af, KS);
+  if (D.in_fix) compute_inv_rms(D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
+  WMARK(90);
+  __syncthreads();
+  WMARK(D.op * 10 + 2);
   const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
   const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
   const bool row0 = g < T, row1 = T16 && g + 8 < T;
@@ -469,8 +505,10 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
       case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
       default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
     }
+    WMARK(D.op * 10 + 3);
     __syncthreads();
-    for (int idx = tid; idx < cnt * 32; idx += FAST_THREADS) {
+    WMARK(D.op * 10 + 4);
+    for (int idx = tid; idx < cnt * 32; idx += FAST_THREADS) {  // whole warps: one tile per warp pass
       const int u = idx >> 5, l = idx & 31, gg = l >> 2, tt = l & 3;
       float c[NACC];
 #pragma unroll
@@ -481,16 +519,22 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
 #pragma unroll
         for (int i = 0; i < NACC; ++i) c[i] += src[i];
       }
-      const int n = M.utile[D.op][u0 + u] * 8 + 2 * tt;
-      if (gg < T) {
-        const float inv = D.in_fix ? M.inv_rms[gg] : 1.f;
-        epilogue_pair(P, D, M, gg, n, c[0] * inv, c[1] * inv);
-      }
-      if (T16 && gg + 8 < T) {
-        const float inv = D.in_fix ? M.inv_rms[gg + 8] : 1.f;
-        epilogue_pair(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv);
+      const int tile = M.utile[D.op][u0 + u];
+      if (D.epi == EPI_F_RESID) {
+        resid_tile<T16>(P, D, tile, l, c);
+      } else {
+        const int n = tile * 8 + 2 * tt;
+        if (gg < T) {
+          const float inv = D.in_fix ? M.inv_rms[gg] : 1.f;
+          epilogue_pair<T16>(P, D, M, gg, n, c[0] * inv, c[1] * inv);
+        }
+        if (T16 && gg + 8 < T) {
+          const float inv = D.in_fix ? M.inv_rms[gg + 8] : 1.f;
+          epilogue_pair<T16>(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv);
+        }
       }
     }
+    WMARK(D.op * 10 + 5);
     if (u0 + FAST_MAXU < cnt_total) __syncthreads();
   }
 }
@@ -502,7 +546,7 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
 // causal inside the draft block), keeps a running max / sum per row and accumulates P * V in
 // shared memory.  With more than one split the partials go to global memory and the CTA that
 // arrives last for a (stream, head) merges them in split order.
-template <int HD>
+template <int HD, bool T16>
 __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_t* uni, int layer) {
   constexpr int KT = 8192 / HD;         // keys per tile (a power of two >= 64)
   constexpr int KROW = HD * 2 + 16;     // padded K row in bytes (conflict-free 16-byte reads)
@@ -637,7 +681,7 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
     for (int idx = tid; idx < R * HD; idx += FAST_THREADS) {
       const int r = idx / HD, dd = idx % HD, tok = bi * R + r;
       if (nsplit == 1) {
-        P.attn_out[((size_t)tok * Hq + hq) * HD + dd] = acc_s[idx] / M.row_l[r];
+        write_frag_elem<T16>(P.xo, tok, hq * HD + dd, acc_s[idx] / M.row_l[r]);
       } else {
         float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
         dst[dd] = acc_s[idx];
@@ -684,7 +728,7 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
               }
             }
           }
-          P.attn_out[((size_t)tok * Hq + hq) * HD + dd] = o / denom;
+          write_frag_elem<T16>(P.xo, tok, hq * HD + dd, o / denom);
         }
       }
     }
@@ -760,9 +804,23 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       if (tid == 0) atomicOr(P.status, SSD_STATUS_BAD_TOKEN);
       id = min(max(id, 0), P.vocab_in - 1);
     }
-    const bf16* src = P.embed + (size_t)id * d;
-    for (int j = tid; j < d; j += FAST_THREADS)
-      P.hfix[(size_t)tok * d + j] = __float2ll_rn(__bfloat162float(src[j]) * FIX_SCALE);
+    const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(P.embed + (size_t)id * d);
+    const float2* g0 = reinterpret_cast<const float2*>(P.m.gains);  // first layer's input norm
+    for (int kk0 = 0; kk0 < (d >> 1); kk0 += FAST_THREADS) {         // column pairs; whole warps
+      const int kk = kk0 + tid;
+      float ss = 0.f;
+      if (kk < (d >> 1)) {
+        const float2 x = __bfloat1622float2(src[kk]);
+        const float2 gn = __ldg(g0 + kk);
+        *reinterpret_cast<longlong2*>(P.hfix + (size_t)tok * d + 2 * kk) =
+            make_longlong2(__float2ll_rn(x.x * FIX_SCALE), __float2ll_rn(x.y * FIX_SCALE));
+        write_frag_pair<T16>(P.xa, tok, 2 * kk, x.x * gn.x, x.y * gn.y);
+        ss = fmaf(x.x, x.x, x.y * x.y);
+      }
+      ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+      ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+      if (kk < (d >> 1) && (kk & 3) == 0) P.ssq_a[(kk >> 2) * FAST_MAX_T + tok] = ss;
+    }
     const double pos = (double)M.tok_pos[tok];
     for (int j = tid; j < half; j += FAST_THREADS) {
       double sn, cs;
@@ -790,36 +848,56 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
 #pragma unroll 1
   for (int it = 0; it < n_phase && ok; ++it) {
     if (it == 5 * P.L) ph = 5;
+#ifdef SSD_TRACE_FINE
+    if (tid == 0) g_wtr_on = (l == 5 && ph < 5);
+    __syncthreads();
+    WMARK(50 + ph * 2);
+#endif
     if (ph == 1) {
-      if (P.hd == 64) attn_phase<64>(P, M, uni, l);
-      else if (P.hd == 128) attn_phase<128>(P, M, uni, l);
-      else attn_phase<32>(P, M, uni, l);
+      if (P.hd == 64) attn_phase<64, T16>(P, M, uni, l);
+      else if (P.hd == 128) attn_phase<128, T16>(P, M, uni, l);
+      else attn_phase<32, T16>(P, M, uni, l);
     } else {
       PhaseDesc D;
       D.layer = l;
-      D.gain = nullptr;
-      D.kb = 0;
       D.qscale = qscale;
       D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
+      D.ssq_in = nullptr;
+      D.xout = nullptr;
+      D.ssq_out = nullptr;
+      D.gain_next = nullptr;
+      D.nsplit = 1;
       if (ph == 0) {
-        D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.in = P.hfix;
-        D.gain = P.m.gains + (size_t)l * 2 * d; D.ld = d; D.kc = d; D.n_rows = qd + 2 * P.Hkv * P.hd;
+        D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
+        D.kc = d; D.n_rows = qd + 2 * P.Hkv * P.hd;
       } else if (ph == 2) {
-        D.op = FOP_O; D.epi = EPI_F_RESID; D.in_fix = 0; D.in = P.attn_out;
-        D.ld = qd; D.kc = qd; D.n_rows = d;
+        D.op = FOP_O; D.epi = EPI_F_RESID; D.in_fix = 0; D.xin = P.xo; D.kc = qd; D.n_rows = d;
+        D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
       } else if (ph == 3) {
-        D.op = FOP_GU; D.epi = EPI_F_SWIGLU; D.in_fix = 1; D.in = P.hfix;
-        D.gain = P.m.gains + (size_t)l * 2 * d + d; D.ld = d; D.kc = d; D.n_rows = 2 * P.F;
+        D.op = FOP_GU; D.epi = EPI_F_SWIGLU; D.in_fix = 1; D.xin = P.xb; D.ssq_in = P.ssq_b;
+        D.kc = d; D.n_rows = 2 * P.F;
       } else if (ph == 4) {
-        D.op = FOP_DOWN; D.epi = EPI_F_RESID; D.in_fix = 0; D.in = P.act;
-        D.ld = P.F; D.kb = dk0; D.kc = dk1 - dk0; D.n_rows = d;
+        D.op = FOP_DOWN; D.epi = EPI_F_RESID; D.in_fix = 0;
+        D.xin = P.xd + (size_t)(dk0 >> 4) * (T16 ? 256 : 128); D.kc = dk1 - dk0; D.n_rows = d;
+        D.xout = P.xa; D.ssq_out = P.ssq_a; D.nsplit = P.m.down_split;
+        D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
       } else {
-        D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.in = P.hfix; D.layer = 0;
-        D.gain = P.m.gains + (size_t)P.L * 2 * d; D.ld = d; D.kc = d; D.n_rows = P.V;
+        D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
+        D.layer = 0; D.kc = d; D.n_rows = P.V;
       }
       gemm_phase<T16>(P, M, uni, ring, D);
     }
     trace_mark(P, n_trace);
+#ifdef SSD_TRACE_FINE
+    WMARK(51 + ph * 2);
+    if (g_wtr_on && ph < 5 && P.trace) {   // dump this phase's marks: trace[cta][100 + ph*8*16 + warp*16 + k]
+      __syncthreads();
+      if (lane < 16) {
+        int src = lane < 6 ? (ph == 1 ? 90 : (ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 6 ? 90 : lane == 7 ? 50 + ph * 2 : lane == 8 ? 51 + ph * 2 : 95);
+        P.trace[(size_t)blockIdx.x * P.trace_cap + 400 + (ph * FAST_WARPS + warp) * 16 + lane] = g_wtr[warp][src];
+      }
+    }
+#endif
     if (ph < 5) {
       ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
       trace_mark(P, n_trace);
