@@ -119,7 +119,7 @@ struct WsPlan {
   size_t len, pending, status, counters, row_ids, accept_flags;
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
-  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, ssq_a, ssq_b, tile_cnt;
+  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, xq, ssq_a, ssq_b, tile_cnt;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -159,6 +159,7 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.xa = take(d * 64);
   p.xb = take(d * 64);
   p.xo = take(qd * 64);
+  p.xq = take(qd * 64);
   p.xd = take(F * 64);
   p.ssq_a = take((d / 8 + 1) * FAST_MAX_T * 4);
   p.ssq_b = take((d / 8 + 1) * FAST_MAX_T * 4);
@@ -233,11 +234,11 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.row_ids = row_ids;
   p.draft_tokens = draft_tokens;
   p.hfix = s->hfix;
-  p.qrot = s->qrot;
   p.rope_cs = s->rope_cs;
   p.xa = s->xa;
   p.xb = s->xb;
   p.xo = s->xo;
+  p.xq = s->xq;
   p.xd = s->xd;
   p.ssq_a = s->ssq_a;
   p.ssq_b = s->ssq_b;
@@ -487,6 +488,7 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->xa = (uint32_t*)(W + p.xa);
   s->xb = (uint32_t*)(W + p.xb);
   s->xo = (uint32_t*)(W + p.xo);
+  s->xq = (uint32_t*)(W + p.xq);
   s->xd = (uint32_t*)(W + p.xd);
   s->ssq_a = (float*)(W + p.ssq_a);
   s->ssq_b = (float*)(W + p.ssq_b);

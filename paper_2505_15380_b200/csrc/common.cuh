@@ -113,7 +113,7 @@ struct ssd_streams {
   // persistent small-batch kernel: fixed-point residual stream, attention partials and counters,
   // grid-barrier words
   long long* hfix;
-  uint32_t *xa, *xb, *xo, *xd;  // projection inputs in tensor-core operand layout
+  uint32_t *xa, *xb, *xo, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
   float *ssq_a, *ssq_b;
   int32_t* tile_cnt;
   float* fpart;

@@ -127,12 +127,12 @@ struct FastParams {
   const int32_t* draft_tokens;  // [B, gamma] when row_ids is null
   // workspace
   long long* hfix;  // residual stream [T][d] in 2^-32 fixed point (order-independent accumulation)
-  float *qrot, *rope_cs, *part, *logits;  // logits null: skip the LM head
+  float *rope_cs, *part, *logits;  // logits null: skip the LM head
   // Inputs of the projections, written by their producers already in the tensor-core operand layout
   // (bf16 leading part + remainder, see fast_verify.cu): the RMS-norm inputs x * gain of the QKV /
   // LM-head projection (xa) and of gate/up (xb), the attention output (xo), SiLU(g) * u (xd); and
   // per 8-column tile and row the sums of squares that go with xa / xb.
-  uint32_t *xa, *xb, *xo, *xd;
+  uint32_t *xa, *xb, *xo, *xd, *xq;  // xq: the rotated, scaled queries
   float *ssq_a, *ssq_b;   // [d / 8][FAST_MAX_T]
   int32_t* tile_cnt;      // [d / 8] arrivals of the down projection's K slices per output tile
   int32_t* attn_counters;

@@ -31,7 +31,7 @@ namespace ssd {
 namespace {
 
 constexpr unsigned long long FAST_WAIT_CYCLES = 3000000000ull;  // ~1.5 s at 2 GHz
-constexpr int FAST_KEYS_MIN = 32;                                // fewest keys worth a split of their own
+constexpr int FAST_KEYS_MIN = 128;                               // fewest keys worth a split of their own
 constexpr float FIX_SCALE = 4294967296.f;                        // residual stream: 2^-32 fixed point
 constexpr float FIX_INV_SCALE = 1.f / 4294967296.f;
 
@@ -298,15 +298,38 @@ __device__ __forceinline__ void stage_copy(const uint32_t* __restrict__ src, uin
 }
 
 // inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
-// warp per row, fixed summation order.
-__device__ __forceinline__ void compute_inv_rms(const float* __restrict__ ssq, int ntiles, int T, int K,
-                                                float eps, FastMisc& M) {
+// warp per row, fixed summation order.  The loads are issued at the start of the phase and
+// summed after the tensor-core work, so their latency stays off the critical path.
+constexpr int SSQ_REGS = 8;  // covers d <= 2048 in one go
+struct SsqLoads {
+  float v[2][SSQ_REGS];  // rows warp and warp + FAST_WARPS
+};
+__device__ __forceinline__ void ssq_issue(SsqLoads& q, const float* __restrict__ ssq, int ntiles, int T) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int row = warp; row < T; row += FAST_WARPS) {
-    float v = 0.f;
-    for (int tile = lane; tile < ntiles; tile += 32) v += __ldcg(ssq + tile * FAST_MAX_T + row);
-    v = warp_sum(v);
-    if (lane == 0) M.inv_rms[row] = rsqrtf(v / (float)K + eps);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int row = warp + h * FAST_WARPS;
+#pragma unroll
+    for (int i = 0; i < SSQ_REGS; ++i) {
+      const int tile = lane + 32 * i;
+      q.v[h][i] = (row < T && tile < ntiles) ? __ldcg(ssq + tile * FAST_MAX_T + row) : 0.f;
+    }
+  }
+}
+__device__ __forceinline__ void ssq_finish(const SsqLoads& q, const float* __restrict__ ssq, int ntiles, int T,
+                                           int K, float eps, FastMisc& M) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int row = warp + h * FAST_WARPS;
+    if (row < T) {  // uniform per warp
+      float v = 0.f;
+#pragma unroll
+      for (int i = 0; i < SSQ_REGS; ++i) v += q.v[h][i];
+      for (int tile = lane + 32 * SSQ_REGS; tile < ntiles; tile += 32) v += __ldcg(ssq + tile * FAST_MAX_T + row);
+      v = warp_sum(v);
+      if (lane == 0) M.inv_rms[row] = rsqrtf(v / (float)K + eps);
+    }
   }
 }
 
@@ -329,9 +352,9 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
       const float2 cs = __ldcg(reinterpret_cast<const float2*>(P.rope_cs + ((size_t)tok * half + j) * 2));
       const float o1 = x1 * cs.x - x2 * cs.y, o2 = x2 * cs.x + x1 * cs.y;
       if (n < qd) {
-        float* q = P.qrot + tok * qd + (n & ~(hd - 1));
-        q[j] = o1 * D.qscale;
-        q[j + half] = o2 * D.qscale;
+        const int col = (n & ~(hd - 1)) + j;  // q, pre-scaled, as the operand of the score contraction
+        write_frag_elem<T16>(P.xq, tok, col, o1 * D.qscale);
+        write_frag_elem<T16>(P.xq, tok, col + half, o2 * D.qscale);
       } else if (pos < P.cap) {
         const int gk = (n - qd) >> hs;
         bf16* kdst = D.kv_layer + (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * hd + (size_t)pos * hd;
@@ -363,6 +386,7 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
   long long* h0 = P.hfix + (size_t)gg * P.d + n;
   long long* h1 = h0 + (size_t)8 * P.d;
   longlong2 a = make_longlong2(0, 0), b = make_longlong2(0, 0);
+  const float2 gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
   if (D.nsplit > 1) {
     if (v0) {
       atomicAdd(reinterpret_cast<unsigned long long*>(h0), (unsigned long long)__float2ll_rn(c[0] * FIX_SCALE));
@@ -398,7 +422,6 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
       *reinterpret_cast<longlong2*>(h1) = b;
     }
   }
-  const float2 gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));
   float s0 = 0.f, s1 = 0.f;
   if (v0) {
     const float x0 = fix_to_float(a.x), x1 = fix_to_float(a.y);
@@ -430,9 +453,12 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
   constexpr int SPC = FAST_SLOT_TILES / CNT;
   constexpr uint32_t STEP = T16 ? 1024u : 512u;
   constexpr int NACC = T16 ? 4 : 2;
-  float acc[CNT][4];
+  constexpr bool TWO = CNT <= 4;  // few tiles: keep the hi and lo terms in separate accumulators
+  float acc[CNT][4], acl[TWO ? CNT : 1][4];
 #pragma unroll
   for (int u = 0; u < CNT; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
+#pragma unroll
+  for (int u = 0; u < (TWO ? CNT : 1); ++u) acl[u][0] = acl[u][1] = acl[u][2] = acl[u][3] = 0.f;
 #pragma unroll 1
   for (int s = s0; s < s1; s += SPC) {
     ring_acquire(r);
@@ -457,10 +483,17 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 #pragma unroll
         for (int u = 0; u < CNT; ++u) mma_bf16(acc[u], ahi, b[u].x, b[u].y);
 #pragma unroll
-        for (int u = 0; u < CNT; ++u) mma_bf16(acc[u], alo, b[u].x, b[u].y);
+        for (int u = 0; u < CNT; ++u) mma_bf16(TWO ? acl[u] : acc[u], alo, b[u].x, b[u].y);
       }
     }
     ring_release(r, lane);
+  }
+  if (TWO) {
+#pragma unroll
+    for (int u = 0; u < CNT; ++u) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[u][i] += acl[u][i];
+    }
   }
 #pragma unroll
   for (int u = 0; u < CNT; ++u) {
@@ -483,8 +516,9 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   uint32_t* af = reinterpret_cast<uint32_t*>(uni);                             // A operand, KS steps
   float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
   WMARK(D.op * 10 + 0);
+  SsqLoads ssq;
+  if (D.in_fix) ssq_issue(ssq, D.ssq_in, P.d >> 3, T);
   stage_copy<T16>(D.xin, af, KS);
-  if (D.in_fix) compute_inv_rms(D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
   WMARK(90);
   __syncthreads();
   WMARK(D.op * 10 + 2);
@@ -505,6 +539,7 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
       case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
       default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
     }
+    if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
     WMARK(D.op * 10 + 3);
     __syncthreads();
     WMARK(D.op * 10 + 4);
@@ -541,73 +576,87 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
 
 // ---- attention ---------------------------------------------------------------------------------
 
-// Work item = (stream, query head, key split).  The item's CTA stages KT keys / values at a time
-// in shared memory, computes the scores of the stream's R rows (row r sees keys 0..len + r:
-// causal inside the draft block), keeps a running max / sum per row and accumulates P * V in
-// shared memory.  With more than one split the partials go to global memory and the CTA that
-// arrives last for a (stream, head) merges them in split order.
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+
+// Work item = (stream, query head, key split).  Per pass of up to 16 keys per warp the item's CTA
+// stages the keys / values (bf16, as cached) in shared memory and runs both contractions on the
+// tensor cores: scores S[key, row] = K[key, :] . q[row, :] (q arrives pre-split in operand layout
+// from the QKV epilogue) and O[row, :] += P[row, key] V[key, :] (P split into bf16 hi + lo, V read
+// with a transposing matrix load), with a running max / sum per row in between.  Row r of a stream
+// sees keys 0..len + r: causal inside the draft block.  The operand rows are the forward's rows
+// (all streams); rows of other streams are masked out.  With more than one split the partials go
+// to global memory and the CTA that arrives last for a (stream, head) merges them in split order.
 template <int HD, bool T16>
 __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_t* uni, int layer) {
-  constexpr int KT = 8192 / HD;         // keys per tile (a power of two >= 64)
-  constexpr int KROW = HD * 2 + 16;     // padded K row in bytes (conflict-free 16-byte reads)
+  constexpr int KT = 16 * FAST_WARPS;     // keys per pass
+  constexpr int ROWB = HD * 2 + 16;       // padded K / V row in bytes (conflict-free fragment loads)
+  constexpr int NT = T16 ? 2 : 1;         // 8-row tiles of the forward's rows
+  constexpr int W = T16 ? 8 : 4;          // words per (k-step, lane) of an operand
+  constexpr int KSTEPS = HD / 16;
+  constexpr int DT = HD / 8;              // 8-dim tiles of the output
+  constexpr int DPW = (DT + FAST_WARPS - 1) / FAST_WARPS;
+  constexpr int CH = HD / 8;              // 16-byte chunks per row
   const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   int max_total = 0;
   for (int bi = 0; bi < nb; ++bi) max_total = max(max_total, min(M.tok_pos[bi * R] + R, P.cap));
   int nsplit = (max_total + FAST_KEYS_MIN - 1) / FAST_KEYS_MIN;
   nsplit = max(1, min(nsplit, min(FAST_NSPLIT_CAP, max(1, P.m.n_cta / (nb * Hq)))));
   const int items = nb * Hq * nsplit;
 
-  float* qs = reinterpret_cast<float*>(uni);                     // [R][HD]
-  uint8_t* Ks = reinterpret_cast<uint8_t*>(qs + R * HD);          // [KT][KROW]
-  bf16* Vs = reinterpret_cast<bf16*>(Ks + KT * KROW);             // [KT][HD]
-  float* ps = reinterpret_cast<float*>(Vs + KT * HD);             // [R][KT] scores, then weights
-  float* acc_s = ps + R * KT;                                     // [R][HD] running P * V
+  uint8_t* Ks = uni;                                             // [KT][ROWB]
+  uint8_t* Vs = Ks + KT * ROWB;                                  // [KT][ROWB]
+  uint32_t* ps = reinterpret_cast<uint32_t*>(Vs + KT * ROWB);    // weights P, operand layout, KT / 16 steps
+  const uint32_t ks_lane = smem_u32(Ks) + (16 * warp + g) * ROWB + t * 4;
+  const uint32_t vs_lane = smem_u32(Vs) + (lane & 15) * ROWB;
+  const uint32_t ps_lane = smem_u32(ps) + lane * (W * 4);
   const bf16* kvl = P.kv + (size_t)layer * P.kv_layer_elems;
 
   for (int item = blockIdx.x; item < items; item += P.m.n_cta) {
     const int c = item % nsplit, hq = (item / nsplit) % Hq, bi = item / (nsplit * Hq);
-    const int stream = P.b0 + bi, gk = hq / G;
-    const int L = M.tok_pos[bi * R], total = min(L + R, P.cap);
-    const int per = (((total + nsplit - 1) / nsplit) + 7) & ~7;
+    const int stream = P.b0 + bi, gk = hq / G, t_lo = bi * R, t_hi = t_lo + R;
+    const int L = M.tok_pos[t_lo], total = min(L + R, P.cap);
+    const int per = (((total + nsplit - 1) / nsplit) + 15) & ~15;
     const int k0 = c * per, k1 = min(k0 + per, total);
     __syncthreads();
-    {
-      constexpr int QB = FAST_MAX_T * HD / FAST_THREADS;  // covers R * HD <= 16 * HD values
-      float qv[QB];
-#pragma unroll
-      for (int i = 0; i < QB; ++i) {
-        const int idx = tid + i * FAST_THREADS;
-        if (idx < R * HD) qv[i] = __ldcg(P.qrot + ((size_t)(bi * R + idx / HD) * Hq + hq) * HD + idx % HD);
-      }
-#pragma unroll
-      for (int i = 0; i < QB; ++i) {
-        const int idx = tid + i * FAST_THREADS;
-        if (idx < R * HD) {
-          qs[idx] = qv[i];
-          acc_s[idx] = 0.f;
-        }
-      }
-    }
-    if (tid < R) {
+    if (tid < FAST_MAX_T) {
       M.row_m[tid] = -CUDART_INF_F;
       M.row_l[tid] = 0.f;
     }
+    // q of this head: B operand of the score contraction, bf16 hi / lo as the QKV epilogue left it
+    uint4 qf[KSTEPS][NT];
+#pragma unroll
+    for (int s = 0; s < KSTEPS; ++s) {
+      const uint4* src = reinterpret_cast<const uint4*>(P.xq + ((size_t)(hq * KSTEPS + s) * 32 + lane) * W);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) qf[s][nt] = __ldcg(src + nt);
+    }
+    float o[DPW][4];
+#pragma unroll
+    for (int dp = 0; dp < DPW; ++dp) o[dp][0] = o[dp][1] = o[dp][2] = o[dp][3] = 0.f;
     const size_t kbase = (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * HD;
     const size_t vbase = (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD;
 
     for (int kt0 = k0; kt0 < k1; kt0 += KT) {
-      const int nk = min(KT, k1 - kt0);
+      const int nk = min(KT, k1 - kt0), nk16 = (nk + 15) & ~15;
       __syncthreads();
-      {
+      {  // keys and values of this pass -> shared memory; rows up to the next multiple of 16 are zeroed
         const uint4* ksrc = reinterpret_cast<const uint4*>(kvl + kbase + (size_t)kt0 * HD);
         const uint4* vsrc = reinterpret_cast<const uint4*>(kvl + vbase + (size_t)kt0 * HD);
-        constexpr int CB = KT * (HD / 8) / FAST_THREADS;  // 16-byte chunks per thread of a full tile
+        constexpr int CB = KT * CH / FAST_THREADS;
         uint4 kq[CB], vq[CB];
 #pragma unroll
         for (int i = 0; i < CB; ++i) {
           const int idx = tid + i * FAST_THREADS;
-          if (idx < nk * (HD / 8)) {
+          kq[i] = vq[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (idx < nk * CH) {
             kq[i] = __ldcg(ksrc + idx);
             vq[i] = __ldcg(vsrc + idx);
           }
@@ -615,79 +664,128 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
 #pragma unroll
         for (int i = 0; i < CB; ++i) {
           const int idx = tid + i * FAST_THREADS;
-          if (idx < nk * (HD / 8)) {
-            *reinterpret_cast<uint4*>(Ks + (idx / (HD / 8)) * KROW + (idx % (HD / 8)) * 16) = kq[i];
-            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(Vs) + (size_t)idx * 16) = vq[i];
+          if (idx < nk16 * CH) {
+            *reinterpret_cast<uint4*>(Ks + (idx / CH) * ROWB + (idx % CH) * 16) = kq[i];
+            *reinterpret_cast<uint4*>(Vs + (idx / CH) * ROWB + (idx % CH) * 16) = vq[i];
           }
         }
       }
       __syncthreads();
-      // scores of (row, key) pairs; a warp works on 32 consecutive keys of one row
-      for (int idx = tid; idx < R * KT; idx += FAST_THREADS) {
-        const int r = idx / KT, key = idx % KT;
-        float sc = -CUDART_INF_F;
-        if (key < nk && kt0 + key <= L + r) {
-          const float* q = qs + r * HD;
-          const uint8_t* krow = Ks + key * KROW;
-          sc = 0.f;
-#pragma unroll 2
-          for (int ch = 0; ch < HD / 8; ++ch) {
-            float kx[8];
-            unpack8(*reinterpret_cast<const uint4*>(krow + ch * 16), kx);
-            const float4 q0 = *reinterpret_cast<const float4*>(q + ch * 8);
-            const float4 q1 = *reinterpret_cast<const float4*>(q + ch * 8 + 4);
-            sc = fmaf(kx[0], q0.x, sc); sc = fmaf(kx[1], q0.y, sc);
-            sc = fmaf(kx[2], q0.z, sc); sc = fmaf(kx[3], q0.w, sc);
-            sc = fmaf(kx[4], q1.x, sc); sc = fmaf(kx[5], q1.y, sc);
-            sc = fmaf(kx[6], q1.z, sc); sc = fmaf(kx[7], q1.w, sc);
+      // scores of this warp's 16 keys against all rows; thread: keys g, g + 8 x rows 2t, 2t + 1 (+ 8)
+      const bool active = 16 * warp < nk;
+      float sc[NT][4];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+      if (active) {
+#pragma unroll
+        for (int s = 0; s < KSTEPS; ++s) {
+          uint32_t a[4];
+          a[0] = lds_u32(ks_lane + s * 32);
+          a[1] = lds_u32(ks_lane + s * 32 + 8 * ROWB);
+          a[2] = lds_u32(ks_lane + s * 32 + 16);
+          a[3] = lds_u32(ks_lane + s * 32 + 8 * ROWB + 16);
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            mma_bf16(sc[nt], a, qf[s][nt].x, qf[s][nt].y);
+            mma_bf16(sc[nt], a, qf[s][nt].z, qf[s][nt].w);
           }
         }
-        ps[idx] = sc;
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int key = 16 * warp + g + (i >> 1) * 8, tok = nt * 8 + 2 * t + (i & 1);
+          const bool valid = active && key < nk && tok >= t_lo && tok < t_hi && kt0 + key <= L + (tok - t_lo);
+          if (!valid) sc[nt][i] = -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          float v = fmaxf(sc[nt][j], sc[nt][j + 2]);
+          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
+          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
+          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
+          if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
+        }
       }
       __syncthreads();
-      // running max / sum per row (one warp per row), scores -> weights in place
-      for (int r = warp; r < R; r += FAST_WARPS) {
-        float mt = -CUDART_INF_F;
-        for (int key = lane; key < nk; key += 32) mt = fmaxf(mt, ps[r * KT + key]);
-        mt = warp_max(mt);
-        const float m_old = M.row_m[r], m_new = fmaxf(m_old, mt);
+      if (tid < 8 * NT) {
+        float mt = M.wred[0][tid];
+#pragma unroll
+        for (int w = 1; w < FAST_WARPS; ++w) mt = fmaxf(mt, M.wred[w][tid]);
+        const float m_old = M.row_m[tid], m_new = fmaxf(m_old, mt);
+        M.row_corr[tid] = m_new == -CUDART_INF_F ? 0.f : __expf(m_old - m_new);
+        M.row_m[tid] = m_new;
+      }
+      __syncthreads();
+      // weights, their row sums, and P in operand layout for the second contraction
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float pw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float m = M.row_m[nt * 8 + 2 * t + (i & 1)];
+          pw[i] = sc[nt][i] == -CUDART_INF_F ? 0.f : __expf(sc[nt][i] - m);
+          if (active) write_frag_elem<T16>(ps, nt * 8 + 2 * t + (i & 1), 16 * warp + g + (i >> 1) * 8, pw[i]);
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          float v = pw[j] + pw[j + 2];
+          v += __shfl_xor_sync(0xffffffffu, v, 4);
+          v += __shfl_xor_sync(0xffffffffu, v, 8);
+          v += __shfl_xor_sync(0xffffffffu, v, 16);
+          if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
+        }
+      }
+      __syncthreads();
+      if (tid < 8 * NT) {
         float lt = 0.f;
-        for (int key = lane; key < nk; key += 32) {
-          const float sc = ps[r * KT + key];
-          const float pw = sc == -CUDART_INF_F ? 0.f : expf(sc - m_new);
-          ps[r * KT + key] = pw;
-          lt += pw;
-        }
-        lt = warp_sum(lt);
-        if (lane == 0) {
-          const float corr = m_new == -CUDART_INF_F ? 0.f : expf(m_old - m_new);
-          M.row_corr[r] = corr;
-          M.row_m[r] = m_new;
-          M.row_l[r] = M.row_l[r] * corr + lt;
-        }
+#pragma unroll
+        for (int w = 0; w < FAST_WARPS; ++w) lt += M.wred[w][tid];
+        M.row_l[tid] = M.row_l[tid] * M.row_corr[tid] + lt;
       }
-      __syncthreads();
-      // P * V for (row, dim) pairs
-      for (int idx = tid; idx < R * HD; idx += FAST_THREADS) {
-        const int r = idx / HD, dd = idx % HD;
-        float a = acc_s[idx] * M.row_corr[r];
-        const float* pr = ps + r * KT;
-#pragma unroll 4
-        for (int key = 0; key < nk; ++key) a = fmaf(pr[key], __bfloat162float(Vs[key * HD + dd]), a);
-        acc_s[idx] = a;
+      // O += P V: this warp owns 8-dim tiles of the output
+      const float c0 = M.row_corr[g], c1 = T16 ? M.row_corr[g + 8] : 0.f;
+#pragma unroll
+      for (int dp = 0; dp < DPW; ++dp) {
+        const int dtile = warp + dp * FAST_WARPS;
+        if (dtile < DT) {
+          o[dp][0] *= c0; o[dp][1] *= c0; o[dp][2] *= c1; o[dp][3] *= c1;
+          for (int ks = 0; ks < (nk16 >> 4); ++ks) {
+            const uint4 pa = lds_v4(ps_lane + ks * (32 * W * 4));
+            uint32_t ahi[4] = {pa.x, 0u, pa.y, 0u}, alo[4] = {pa.z, 0u, pa.w, 0u};
+            if (T16) {
+              const uint4 pb = lds_v4(ps_lane + ks * (32 * W * 4) + 16);
+              ahi[1] = pb.x; ahi[3] = pb.y; alo[1] = pb.z; alo[3] = pb.w;
+            }
+            uint32_t b0, b1;
+            ldmatrix_x2_trans(vs_lane + ks * 16 * ROWB + dtile * 16, b0, b1);
+            mma_bf16(o[dp], ahi, b0, b1);
+            mma_bf16(o[dp], alo, b0, b1);
+          }
+        }
       }
     }
     __syncthreads();
-    for (int idx = tid; idx < R * HD; idx += FAST_THREADS) {
-      const int r = idx / HD, dd = idx % HD, tok = bi * R + r;
-      if (nsplit == 1) {
-        write_frag_elem<T16>(P.xo, tok, hq * HD + dd, acc_s[idx] / M.row_l[r]);
-      } else {
-        float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
-        dst[dd] = acc_s[idx];
-        if (dd == 0) {
-          dst[HD] = M.row_m[r];
-          dst[HD + 1] = M.row_l[r];
+    // output: thread holds rows g (and g + 8) x dims 2t, 2t + 1 of its tiles
+#pragma unroll
+    for (int dp = 0; dp < DPW; ++dp) {
+      const int dtile = warp + dp * FAST_WARPS;
+      if (dtile < DT) {
+#pragma unroll
+        for (int h = 0; h < NT; ++h) {
+          const int tok = g + 8 * h, dd = dtile * 8 + 2 * t;
+          if (tok >= t_lo && tok < t_hi) {
+            const float o0 = o[dp][2 * h], o1 = o[dp][2 * h + 1];
+            if (nsplit == 1) {
+              const float il = 1.f / M.row_l[tok];
+              write_frag_pair<T16>(P.xo, tok, hq * HD + dd, o0 * il, o1 * il);
+            } else {
+              float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
+              *reinterpret_cast<float2*>(dst + dd) = make_float2(o0, o1);
+              if (dd == 0) *reinterpret_cast<float2*>(dst + HD) = make_float2(M.row_m[tok], M.row_l[tok]);
+            }
+          }
         }
       }
     }
@@ -703,9 +801,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
       if (M.last) {
         __threadfence();
         for (int idx = tid; idx < R * HD; idx += FAST_THREADS) {
-          const int r = idx / HD, dd = idx % HD, tok = bi * R + r;
+          const int r = idx / HD, dd = idx % HD, tok = t_lo + r;
           const float* src = P.part + ((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP * (HD + 2);
-          float m_tot = -CUDART_INF_F, denom = 0.f, o = 0.f;
+          float m_tot = -CUDART_INF_F, denom = 0.f, ov = 0.f;
           constexpr int MB = 8;  // splits loaded together
           for (int sp0 = 0; sp0 < nsplit; sp0 += MB) {
             float ms[MB], ls[MB], os[MB];
@@ -721,14 +819,14 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
             for (int i = 0; i < MB; ++i) {
               if (sp0 + i < nsplit && ms[i] != -CUDART_INF_F) {  // running merge in split order
                 const float m_new = fmaxf(m_tot, ms[i]);
-                const float ca = expf(m_tot - m_new), cb = expf(ms[i] - m_new);
+                const float ca = __expf(m_tot - m_new), cb = __expf(ms[i] - m_new);
                 denom = denom * ca + ls[i] * cb;
-                o = o * ca + os[i] * cb;
+                ov = ov * ca + os[i] * cb;
                 m_tot = m_new;
               }
             }
           }
-          write_frag_elem<T16>(P.xo, tok, hq * HD + dd, o / denom);
+          write_frag_elem<T16>(P.xo, tok, hq * HD + dd, ov / denom);
         }
       }
     }
@@ -932,9 +1030,9 @@ size_t fast_union_bytes(int stage_k, int hd, int T, int R) {
   const bool t16 = T > 8;
   size_t af = (size_t)(stage_k / 16) * (t16 ? 1024 : 512);
   size_t red = (size_t)FAST_WARPS * FAST_MAXU * 32 * (t16 ? 16 : 8);
-  const int KT = 8192 / hd;
-  size_t attn = (size_t)R * hd * 4 + (size_t)KT * (hd * 2 + 16) + (size_t)KT * hd * 2 +
-                (size_t)R * KT * 4 + (size_t)R * hd * 4;
+  const int KT = 16 * FAST_WARPS;
+  size_t attn = (size_t)2 * KT * (hd * 2 + 16) + (size_t)(KT / 16) * 32 * (t16 ? 32 : 16);
+  (void)R;
   size_t u = af + red > attn ? af + red : attn;
   return (u + 127) / 128 * 128;
 }
