@@ -144,6 +144,7 @@ struct FastParams {
   int trace_cap;
   // shared-memory carve-up (bytes)
   int nslot, ring_warp_bytes, union_off, misc_off;
+  int keys_min;  // fewest keys worth an attention split of their own
 };
 
 size_t fast_union_bytes(int stage_k, int head_dim, int T, int R);

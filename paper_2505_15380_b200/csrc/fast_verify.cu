@@ -110,8 +110,14 @@ struct FastMisc {
   float wred[FAST_WARPS][FAST_MAX_T];
   int32_t tok_stream[FAST_MAX_T];  // stream of each row of this forward
   int32_t tok_pos[FAST_MAX_T];     // its position len + r
+  int32_t attn_nsplit;             // key splits per (stream, head): the same in every layer
+  int32_t attn_item[6];            // this CTA's first work item: c, hq, bi, k0, k1, valid
   int32_t last;
 };
+
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 
 // A warp's private weight stream and shared-memory ring; every lane keeps an identical copy in
 // registers.  One chunk (whole k-steps of a round, at most FAST_SLOT_TILES tiles) fills one slot.
@@ -605,11 +611,7 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
   constexpr int CH = HD / 8;              // 16-byte chunks per row
   const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  int max_total = 0;
-  for (int bi = 0; bi < nb; ++bi) max_total = max(max_total, min(M.tok_pos[bi * R] + R, P.cap));
-  int nsplit = (max_total + FAST_KEYS_MIN - 1) / FAST_KEYS_MIN;
-  nsplit = max(1, min(nsplit, min(FAST_NSPLIT_CAP, max(1, P.m.n_cta / (nb * Hq)))));
-  const int items = nb * Hq * nsplit;
+  const int nsplit = M.attn_nsplit, items = nb * Hq * nsplit;
 
   uint8_t* Ks = uni;                                             // [KT][ROWB]
   uint8_t* Vs = Ks + KT * ROWB;                                  // [KT][ROWB]
@@ -620,16 +622,23 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
   const bf16* kvl = P.kv + (size_t)layer * P.kv_layer_elems;
 
   for (int item = blockIdx.x; item < items; item += P.m.n_cta) {
-    const int c = item % nsplit, hq = (item / nsplit) % Hq, bi = item / (nsplit * Hq);
+    int c, hq, bi, k0, k1;
+    if (item == (int)blockIdx.x) {  // the usual case: one item per CTA, worked out once per launch
+      c = M.attn_item[0]; hq = M.attn_item[1]; bi = M.attn_item[2]; k0 = M.attn_item[3]; k1 = M.attn_item[4];
+    } else {
+      c = item % nsplit; hq = (item / nsplit) % Hq; bi = item / (nsplit * Hq);
+      const int tot = min(M.tok_pos[bi * R] + R, P.cap);
+      const int per = (((tot + nsplit - 1) / nsplit) + 15) & ~15;
+      k0 = c * per; k1 = min(k0 + per, tot);
+    }
     const int stream = P.b0 + bi, gk = hq / G, t_lo = bi * R, t_hi = t_lo + R;
-    const int L = M.tok_pos[t_lo], total = min(L + R, P.cap);
-    const int per = (((total + nsplit - 1) / nsplit) + 15) & ~15;
-    const int k0 = c * per, k1 = min(k0 + per, total);
+    const int L = M.tok_pos[t_lo];
     __syncthreads();
     if (tid < FAST_MAX_T) {
       M.row_m[tid] = -CUDART_INF_F;
       M.row_l[tid] = 0.f;
     }
+    WMARK(60);
     // q of this head: B operand of the score contraction, bf16 hi / lo as the QKV epilogue left it
     uint4 qf[KSTEPS][NT];
 #pragma unroll
@@ -643,10 +652,22 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
     for (int dp = 0; dp < DPW; ++dp) o[dp][0] = o[dp][1] = o[dp][2] = o[dp][3] = 0.f;
     const size_t kbase = (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * HD;
     const size_t vbase = (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD;
+    if (layer + 1 < P.L) {
+      // the same keys and values of the next layer (the cached prefix does not change during the
+      // forward): pull them into L2 now, one 128-byte line per thread and pass
+      const uint8_t* nk_ = reinterpret_cast<const uint8_t*>(kvl + P.kv_layer_elems + kbase + (size_t)k0 * HD);
+      const uint8_t* nv_ = reinterpret_cast<const uint8_t*>(kvl + P.kv_layer_elems + vbase + (size_t)k0 * HD);
+      const int lines = ((k1 - k0) * HD * 2 + 127) >> 7;
+      for (int i = tid; i < lines; i += FAST_THREADS) {
+        prefetch_l2(nk_ + (size_t)i * 128);
+        prefetch_l2(nv_ + (size_t)i * 128);
+      }
+    }
 
     for (int kt0 = k0; kt0 < k1; kt0 += KT) {
       const int nk = min(KT, k1 - kt0), nk16 = (nk + 15) & ~15;
       __syncthreads();
+      WMARK(61);
       {  // keys and values of this pass -> shared memory; rows up to the next multiple of 16 are zeroed
         const uint4* ksrc = reinterpret_cast<const uint4*>(kvl + kbase + (size_t)kt0 * HD);
         const uint4* vsrc = reinterpret_cast<const uint4*>(kvl + vbase + (size_t)kt0 * HD);
@@ -670,7 +691,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
           }
         }
       }
+      WMARK(62);
       __syncthreads();
+      WMARK(63);
       // scores of this warp's 16 keys against all rows; thread: keys g, g + 8 x rows 2t, 2t + 1 (+ 8)
       const bool active = 16 * warp < nk;
       float sc[NT][4];
@@ -708,7 +731,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
           if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
         }
       }
+      WMARK(64);
       __syncthreads();
+      WMARK(65);
       if (tid < 8 * NT) {
         float mt = M.wred[0][tid];
 #pragma unroll
@@ -717,7 +742,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
         M.row_corr[tid] = m_new == -CUDART_INF_F ? 0.f : __expf(m_old - m_new);
         M.row_m[tid] = m_new;
       }
+      WMARK(66);
       __syncthreads();
+      WMARK(67);
       // weights, their row sums, and P in operand layout for the second contraction
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
@@ -737,7 +764,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
           if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
         }
       }
+      WMARK(68);
       __syncthreads();
+      WMARK(69);
       if (tid < 8 * NT) {
         float lt = 0.f;
 #pragma unroll
@@ -766,7 +795,9 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
         }
       }
     }
+    WMARK(70);
     __syncthreads();
+    WMARK(71);
     // output: thread holds rows g (and g + 8) x dims 2t, 2t + 1 of its tiles
 #pragma unroll
     for (int dp = 0; dp < DPW; ++dp) {
@@ -789,9 +820,11 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
         }
       }
     }
+    WMARK(72);
     if (nsplit > 1) {
       __threadfence();
       __syncthreads();
+      WMARK(73);
       if (tid == 0) {
         int prev = atomicAdd(&P.attn_counters[bi * Hq + hq], 1);
         M.last = prev == nsplit - 1;
@@ -864,6 +897,23 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     const int bi = tid / P.R, r = tid % P.R;
     M.tok_stream[tid] = P.b0 + bi;
     M.tok_pos[tid] = P.len[P.b0 + bi] + r;
+  }
+
+  if (tid == 0) {
+    const int R = P.R, nb = P.nb, Hq = P.Hq;
+    int max_total = 0;
+    for (int bi = 0; bi < nb; ++bi) max_total = max(max_total, min(P.len[P.b0 + bi] + R, P.cap));
+    int nsplit = (max_total + P.keys_min - 1) / P.keys_min;
+    nsplit = max(1, min(nsplit, min(FAST_NSPLIT_CAP, max(1, P.m.n_cta / (nb * Hq)))));
+    M.attn_nsplit = nsplit;
+    const int item = cta;
+    if (item < nb * Hq * nsplit) {
+      const int c = item % nsplit, hq = (item / nsplit) % Hq, bi = item / (nsplit * Hq);
+      const int tot = min(P.len[P.b0 + bi] + R, P.cap);
+      const int per = (((tot + nsplit - 1) / nsplit) + 15) & ~15;
+      M.attn_item[0] = c; M.attn_item[1] = hq; M.attn_item[2] = bi;
+      M.attn_item[3] = c * per; M.attn_item[4] = min(c * per + per, tot);
+    }
   }
 
   // this warp's ring: barriers, then the first copies
@@ -951,6 +1001,15 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     __syncthreads();
     WMARK(50 + ph * 2);
 #endif
+    if (ph == 0 && cta == (l % P.m.n_cta) + 0 && l + 1 < P.L) {
+      // the small per-layer constants are read once per forward, so they would miss all the way
+      // to HBM in the middle of an epilogue: one CTA pulls the next layer's into L2 ahead of time
+      const int nq = (P.Hq + 2 * P.Hkv) * P.hd;
+      const uint8_t* bq = reinterpret_cast<const uint8_t*>(P.m.bias_qkv + (size_t)(l + 1) * nq);
+      const uint8_t* gq = reinterpret_cast<const uint8_t*>(P.m.gains + (size_t)(l + 1) * 2 * d);
+      for (int i = tid; i < ((nq * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(bq + (size_t)i * 128);
+      for (int i = tid; i < ((3 * d * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(gq + (size_t)i * 128);
+    }
     if (ph == 1) {
       if (P.hd == 64) attn_phase<64, T16>(P, M, uni, l);
       else if (P.hd == 128) attn_phase<128, T16>(P, M, uni, l);
@@ -991,7 +1050,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     if (g_wtr_on && ph < 5 && P.trace) {   // dump this phase's marks: trace[cta][100 + ph*8*16 + warp*16 + k]
       __syncthreads();
       if (lane < 16) {
-        int src = lane < 6 ? (ph == 1 ? 90 : (ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 6 ? 90 : lane == 7 ? 50 + ph * 2 : lane == 8 ? 51 + ph * 2 : 95);
+        int src = ph == 1 ? (lane < 14 ? 60 + lane : (lane == 14 ? 50 + ph * 2 : 51 + ph * 2)) : lane < 6 ? ((ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 6 ? 90 : lane == 7 ? 50 + ph * 2 : lane == 8 ? 51 + ph * 2 : 95);
         P.trace[(size_t)blockIdx.x * P.trace_cap + 400 + (ph * FAST_WARPS + warp) * 16 + lane] = g_wtr[warp][src];
       }
     }
@@ -1050,6 +1109,7 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   int nslot = (int)((max_smem - uni - misc) / ((size_t)FAST_WARPS * FAST_SLOT_BYTES));
   if (nslot > FAST_RING_SLOTS) nslot = FAST_RING_SLOTS;
   p.nslot = nslot;
+  p.keys_min = getenv("SSD_KEYS_MIN") ? atoi(getenv("SSD_KEYS_MIN")) : FAST_KEYS_MIN;
   p.ring_warp_bytes = nslot * FAST_SLOT_BYTES;
   p.union_off = FAST_WARPS * p.ring_warp_bytes;
   p.misc_off = p.union_off + (int)uni;
