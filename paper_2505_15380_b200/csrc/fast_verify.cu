@@ -283,24 +283,27 @@ __device__ __forceinline__ void write_frag_elem(uint32_t* buf, int row, int k, f
   w[4] = l;  // two words on
 }
 
-// Copies `nsteps` k-steps of an operand-layout input from global memory (written by other CTAs in
-// an earlier phase, hence read past L1) to shared memory.  All loads are in flight before the
-// first store.
+// Copies this warp's k-steps [s0, s1) of an operand-layout input from global memory (written by
+// other CTAs in an earlier phase, hence read past L1) to the same place in the shared-memory image.
+// A warp only ever multiplies with its own K slice, so the staging needs no CTA-wide barrier.
+// All loads are in flight before the first store.
 template <bool T16>
-__device__ __forceinline__ void stage_copy(const uint32_t* __restrict__ src, uint32_t* af, int nsteps) {
-  constexpr int LB = 8;
-  const int n16 = nsteps * (T16 ? 64 : 32);
-  const uint4* s4 = reinterpret_cast<const uint4*>(src);
-  uint4* d4 = reinterpret_cast<uint4*>(af);
-  for (int i0 = threadIdx.x; i0 < n16; i0 += LB * FAST_THREADS) {
+__device__ __forceinline__ void stage_copy_warp(const uint32_t* __restrict__ src, uint32_t* af, int s0,
+                                                int s1, int lane) {
+  constexpr int LB = 8, V = T16 ? 2 : 1;  // 16-byte vectors per lane and step
+  const uint4* s4 = reinterpret_cast<const uint4*>(src) + (size_t)s0 * 32 * V;
+  uint4* d4 = reinterpret_cast<uint4*>(af) + (size_t)s0 * 32 * V;
+  const int n16 = (s1 - s0) * 32 * V;
+  for (int i0 = lane; i0 < n16; i0 += LB * 32) {
     uint4 v[LB];
 #pragma unroll
     for (int i = 0; i < LB; ++i)
-      if (i0 + i * FAST_THREADS < n16) v[i] = __ldcg(s4 + i0 + i * FAST_THREADS);
+      if (i0 + i * 32 < n16) v[i] = __ldcg(s4 + i0 + i * 32);
 #pragma unroll
     for (int i = 0; i < LB; ++i)
-      if (i0 + i * FAST_THREADS < n16) d4[i0 + i * FAST_THREADS] = v[i];
+      if (i0 + i * 32 < n16) d4[i0 + i * 32] = v[i];
   }
+  __syncwarp();
 }
 
 // inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
@@ -315,10 +318,12 @@ __device__ __forceinline__ void ssq_issue(SsqLoads& q, const float* __restrict__
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const int row = warp + h * FAST_WARPS;
+    if (row < T) {  // uniform per warp
 #pragma unroll
-    for (int i = 0; i < SSQ_REGS; ++i) {
-      const int tile = lane + 32 * i;
-      q.v[h][i] = (row < T && tile < ntiles) ? __ldcg(ssq + tile * FAST_MAX_T + row) : 0.f;
+      for (int i = 0; i < SSQ_REGS; ++i) {
+        const int tile = lane + 32 * i;
+        q.v[h][i] = tile < ntiles ? __ldcg(ssq + tile * FAST_MAX_T + row) : 0.f;
+      }
     }
   }
 }
@@ -455,7 +460,7 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
 // per chunk (one ring slot = SPC whole k-steps), partial sums to shared memory at the end.
 template <int CNT, bool T16>
 __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, int s0, int s1, bool row0,
-                                          bool row1, float* red_dst) {
+                                          bool row1, float* red_dst, int mark = 0) {
   constexpr int SPC = FAST_SLOT_TILES / CNT;
   constexpr uint32_t STEP = T16 ? 1024u : 512u;
   constexpr int NACC = T16 ? 4 : 2;
@@ -468,6 +473,7 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 #pragma unroll 1
   for (int s = s0; s < s1; s += SPC) {
     ring_acquire(r);
+    if (s == s0) WMARK(mark + 6);
     const uint32_t wb = r.ring + r.slot * FAST_SLOT_BYTES + lane * 8;
 #pragma unroll
     for (int i = 0; i < SPC; ++i) {
@@ -492,7 +498,9 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
         for (int u = 0; u < CNT; ++u) mma_bf16(TWO ? acl[u] : acc[u], alo, b[u].x, b[u].y);
       }
     }
+    if (s == s0) WMARK(mark + 7);
     ring_release(r, lane);
+    if (s == s0) WMARK(mark + 8);
   }
   if (TWO) {
 #pragma unroll
@@ -522,28 +530,26 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   uint32_t* af = reinterpret_cast<uint32_t*>(uni);                             // A operand, KS steps
   float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
   WMARK(D.op * 10 + 0);
+  const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
   SsqLoads ssq;
   if (D.in_fix) ssq_issue(ssq, D.ssq_in, P.d >> 3, T);
-  stage_copy<T16>(D.xin, af, KS);
-  WMARK(90);
-  __syncthreads();
-  WMARK(D.op * 10 + 2);
-  const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
-  const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
   const bool row0 = g < T, row1 = T16 && g + 8 < T;
+  stage_copy_warp<T16>(D.xin, af, s0, s1, lane);
+  WMARK(D.op * 10 + 2);
+  const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
   float* red_dst = red + ((size_t)warp * FAST_MAXU * 32 + lane) * NACC;
 
   for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
     const int cnt = min(FAST_MAXU, cnt_total - u0);
     switch (cnt) {
-      case 1: mma_round<1, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 2: mma_round<2, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 3: mma_round<3, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 4: mma_round<4, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 1: mma_round<1, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 2: mma_round<2, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 3: mma_round<3, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 4: mma_round<4, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
     }
     if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
     WMARK(D.op * 10 + 3);
@@ -1050,7 +1056,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     if (g_wtr_on && ph < 5 && P.trace) {   // dump this phase's marks: trace[cta][100 + ph*8*16 + warp*16 + k]
       __syncthreads();
       if (lane < 16) {
-        int src = ph == 1 ? (lane < 14 ? 60 + lane : (lane == 14 ? 50 + ph * 2 : 51 + ph * 2)) : lane < 6 ? ((ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 6 ? 90 : lane == 7 ? 50 + ph * 2 : lane == 8 ? 51 + ph * 2 : 95);
+        int src = ph == 1 ? (lane < 14 ? 60 + lane : (lane == 14 ? 50 + ph * 2 : 51 + ph * 2)) : lane < 9 ? ((ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 9 ? 50 + ph * 2 : lane == 10 ? 51 + ph * 2 : 95);
         P.trace[(size_t)blockIdx.x * P.trace_cap + 400 + (ph * FAST_WARPS + warp) * 16 + lane] = g_wtr[warp][src];
       }
     }
