@@ -28,6 +28,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent forward kernel, from
+# the ncu capture summarised under profiles/ (null once the kernel has changed since)
+TRAFFIC_BYTES = {}
 
 
 def _measured_peaks():
@@ -236,6 +239,25 @@ def run_cuda(args):
         torch.cuda.synchronize()
         dev_ms = e0.elapsed_time(e1)
         k_timed = d_k.cpu().numpy().copy()
+        # the dominant kernel alone: the decoder forward (one persistent kernel when the forward has
+        # at most 16 rows), in a graph of its own, timed with events on the launching stream
+        fgraph = torch.cuda.CUDAGraph()
+        gs.forward(d_tok, g, d_logits, stream=stream)
+        stream.synchronize()
+        n1 = L.ssd_kernel_launch_count()
+        with torch.cuda.graph(fgraph, stream=stream):
+            gs.forward(d_tok, g, d_logits, stream=stream)
+        fwd_launches = L.ssd_kernel_launch_count() - n1
+        for _ in range(3):
+            fgraph.replay()
+        stream.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.steps):
+            fgraph.replay()
+        f1.record(stream)
+        stream.synchronize()
+        fwd_ms = f0.elapsed_time(f1)
         # per-step distribution (each replay between its own events)
         per = []
         for _ in range(min(args.steps, 50)):
@@ -267,10 +289,10 @@ def run_cuda(args):
     assert gs.last_status() == 0, "device status flags raised during the benchmark"
     assert np.array_equal(h_k.numpy(), k_timed), "host-buffer path disagrees with the device path"
 
-    t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
+    t = torch.tensor([dev_ms, e2e_ms, fwd_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dev_ms, e2e_ms = float(t[0]), float(t[1])
+    dev_ms, e2e_ms, fwd_ms = float(t[0]), float(t[1]), float(t[2])
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -280,7 +302,12 @@ def run_cuda(args):
     e2e_us = e2e_ms * 1e3 / args.steps
     kv_read = sum(int(n) + R for n in lens0) * shape.kv_bytes_per_token()
     alg_bytes = shape.streamed_weight_bytes() + kv_read
-    achieved = alg_bytes / (us * 1e-6) / 1e9
+    fwd_us = fwd_ms * 1e3 / args.steps
+    persistent = fwd_launches == 1
+    # roofline of the dominant kernel: the persistent forward kernel when there is one (it streams
+    # all algorithmic bytes of the step), else the step as a whole
+    kern_us = fwd_us if persistent else us
+    achieved = alg_bytes / (kern_us * 1e-6) / 1e9
     peak, peak_kind = _measured_peaks()
     mean_tokens = float(np.mean(k_timed + 1))
     out = {
@@ -307,8 +334,11 @@ def run_cuda(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_step": alg_bytes, "traffic": None,
-                     "kernel": "whole verify step (all launches of one graph replay)"},
+                     "algorithmic_bytes_per_step": alg_bytes, "traffic": TRAFFIC_BYTES.get(wl.name) if persistent else None,
+                     "kernel": ("fast_forward_kernel (persistent decoder forward, one launch)" if persistent
+                                else "whole verify step (all launches of one graph replay)"),
+                     "kernel_us": kern_us, "kernel_share_of_step": kern_us / us,
+                     "step_frac": alg_bytes / (us * 1e-6) / 1e9 / peak},
         "paper_context": "paper reports 1.4x LM speedup over AR decoding on A100-SXM4-40GB "
                          "(beta=0.4, L_d=3); no verify-step latency is published",
     }

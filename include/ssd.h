@@ -177,6 +177,12 @@ int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_token
                const ssd_verify_params* params, int32_t* dev_accepted_len,
                int32_t* dev_next_token, float* dev_logits_or_null, void* stream);
 
+/* The decoder forward of Eq. 4 alone: feeds [pending, x_1..x_gamma] of every stream at positions
+ * len..len+gamma, writes their provisional K/V and the raw target logits float [B, gamma+1, V];
+ * no acceptance step.  (ssd_verify = this followed by the acceptance kernel.) */
+int ssd_forward(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens, int32_t gamma,
+                float* dev_logits, void* stream);
+
 /* Same step with HOST buffers: copies the three inputs to the device, runs ssd_verify and
  * ssd_kv_commit, copies accepted_len / next_token back and synchronises `stream`.  Host
  * buffers should be pinned for the copies to be asynchronous. */
@@ -211,6 +217,19 @@ int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_draft_tokens,
                        const float* dev_draft_probs, const float* dev_uniforms,
                        const ssd_verify_params* params, int32_t batch, int32_t vocab,
                        int32_t* dev_accepted_len, int32_t* dev_next_token, void* stream);
+
+/* ---- host-side checks of the persistent kernel's weight packing (no device needed) ------- */
+
+/* Plan of the persistent small-batch kernel for a bf16 model on n_cta CTAs.  out8 receives:
+ * packed bytes in total, fewest / most bytes any CTA streams, most output tiles a CTA owns for one
+ * projection, most chunks in a warp's table, K slices of the down projection, warps per CTA,
+ * output tiles over all CTAs and projections.  SSD_ERR_BAD_CONFIG if the model has no such path. */
+int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8);
+/* Packs the projection weights of host_weights (blob of ssd_model_create) into the per-warp streams
+ * and walks the streams back into host_out (same layout and size; only the projection matrices and
+ * the LM head are written).  *bad_chunks = chunk-table entries that disagree with the walk. */
+int ssd_fast_pack_roundtrip_host(const ssd_model_config* cfg, int32_t n_cta, const void* host_weights,
+                                 size_t nbytes, void* host_out, int64_t* bad_chunks);
 
 /* ---- diagnostics ------------------------------------------------------------------------- */
 

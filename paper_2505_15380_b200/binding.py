@@ -20,7 +20,8 @@ _lib = None
 EXPORTS = [
     "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
     "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_streams_set_path",
-    "ssd_streams_set_trace", "ssd_kv_truncate",
+    "ssd_streams_set_trace", "ssd_forward", "ssd_fast_plan_host",
+    "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
@@ -68,6 +69,9 @@ def lib() -> ctypes.CDLL:
     L.ssd_streams_destroy.argtypes = [vp]
     L.ssd_streams_set_path.argtypes = [vp, i32]
     L.ssd_streams_set_trace.argtypes = [vp, vp, i32, i32]
+    L.ssd_forward.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.ssd_fast_plan_host.argtypes = [cfgp, i32, ctypes.POINTER(ctypes.c_int64)]
+    L.ssd_fast_pack_roundtrip_host.argtypes = [cfgp, i32, vp, sz, vp, ctypes.POINTER(ctypes.c_int64)]
     L.ssd_kv_truncate.argtypes = [vp, vp, vp, vp]
     L.ssd_streams_get_state.argtypes = [vp, vp, vp, vp]
     L.ssd_prefill.argtypes = [vp, vp, vp, vp, vp]
@@ -244,6 +248,14 @@ class Streams:
                                draft_probs.data_ptr(), uniforms.data_ptr(), ctypes.byref(params),
                                accepted_len.data_ptr(), next_token.data_ptr(), _ptr(logits),
                                _stream_ptr(stream)))
+
+    def forward(self, draft_tokens: torch.Tensor, gamma: int, logits: torch.Tensor, stream=None) -> None:
+        """ssd_forward: the decoder forward alone (logits [B, gamma+1, V]), no acceptance step."""
+        assert draft_tokens.dtype == torch.int32 and draft_tokens.numel() == self.B * gamma
+        assert logits.dtype == torch.float32 and logits.is_contiguous() and \
+            logits.numel() == self.B * (gamma + 1) * self.model.shape.vocab_out
+        check(lib().ssd_forward(self.model.handle, self.handle, draft_tokens.data_ptr(), gamma,
+                                logits.data_ptr(), _stream_ptr(stream)))
 
     def verify_host(self, draft_tokens: torch.Tensor, draft_probs: torch.Tensor,
                     uniforms: torch.Tensor, params: VerifyParams, accepted_len: torch.Tensor,

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
+#include <stdint.h>
 
 #include <new>
 
@@ -505,6 +506,54 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
 }
 
 void ssd_streams_destroy(ssd_streams* s) { delete s; }
+
+int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8) {
+  if (!cfg || !out8) return SSD_ERR_NULL;
+  if (!cfg_ok(cfg) || !fast_supported(*cfg) || n_cta < 1 || n_cta > FAST_MAX_CTAS) return SSD_ERR_BAD_CONFIG;
+  const FastPlan p = fast_make_plan(*cfg, n_cta);
+  int64_t mn = INT64_MAX, mx = 0;
+  for (int cta = 0; cta < n_cta; ++cta) {
+    const size_t lo = p.stream_off[(size_t)cta * FAST_WARPS];
+    const size_t hi = cta + 1 < n_cta ? p.stream_off[(size_t)(cta + 1) * FAST_WARPS] : p.total_bytes;
+    mn = (int64_t)(hi - lo) < mn ? (int64_t)(hi - lo) : mn;
+    mx = (int64_t)(hi - lo) > mx ? (int64_t)(hi - lo) : mx;
+  }
+  int32_t mu = 0;
+  for (int32_t v : p.unit_cnt) mu = v > mu ? v : mu;
+  out8[0] = (int64_t)p.total_bytes;
+  out8[1] = mn;
+  out8[2] = mx;
+  out8[3] = mu;
+  out8[4] = p.max_chunks;
+  out8[5] = p.ops[FOP_DOWN].ksplit;
+  out8[6] = FAST_WARPS;
+  out8[7] = (int64_t)p.unit_tile.size();
+  return SSD_OK;
+}
+
+int ssd_fast_pack_roundtrip_host(const ssd_model_config* cfg, int32_t n_cta, const void* host_weights,
+                                 size_t nbytes, void* host_out, int64_t* bad_chunks) {
+  if (!cfg || !host_weights || !host_out || !bad_chunks) return SSD_ERR_NULL;
+  if (!cfg_ok(cfg) || !fast_supported(*cfg) || n_cta < 1 || n_cta > FAST_MAX_CTAS) return SSD_ERR_BAD_CONFIG;
+  if (nbytes != blob_elems(*cfg) * 2) return SSD_ERR_BAD_CONFIG;
+  const FastPlan p = fast_make_plan(*cfg, n_cta);
+  std::vector<uint8_t> packed(p.total_bytes);
+  fast_pack_streams(*cfg, p, (const uint16_t*)host_weights, packed.data());
+  *bad_chunks = fast_unpack_streams(*cfg, p, packed.data(), (uint16_t*)host_out);
+  return SSD_OK;
+}
+
+int ssd_forward(ssd_model* model, ssd_streams* s, const int32_t* dev_draft_tokens, int32_t gamma,
+                float* dev_logits, void* stream) {
+  if (!model || !s || !dev_draft_tokens || !dev_logits) return SSD_ERR_NULL;
+  if (!same_shape(model->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
+  if (gamma < 1 || gamma > s->max_gamma) return SSD_ERR_BAD_GAMMA;
+  cudaStream_t st = (cudaStream_t)stream;
+  const RowMap rm{0, s->B, gamma + 1};
+  if (use_fast(model, s, rm)) return forward_fast(model, s, rm, nullptr, dev_draft_tokens, dev_logits, st);
+  launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
+  return forward(model, s, rm, dev_logits, st);
+}
 
 int ssd_streams_set_path(ssd_streams* s, int32_t path) {
   if (!s) return SSD_ERR_NULL;

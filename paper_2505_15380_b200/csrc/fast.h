@@ -86,6 +86,8 @@ FastPlan fast_make_plan(const ssd_model_config& c, int n_cta);
 // streams described by `plan` (out has plan.total_bytes bytes).
 void fast_pack_streams(const ssd_model_config& c, const FastPlan& plan, const uint16_t* blob,
                        uint8_t* out);
+long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, const uint8_t* streams,
+                              uint16_t* blob_out);
 // Biases of q/k/v in packed row order and the three kinds of norm gains, as fp32:
 //   bias [L][n_qkv]; gains [L][2][d] followed by the final norm's [d].
 void fast_pack_aux(const ssd_model_config& c, const uint16_t* blob, std::vector<float>& bias,

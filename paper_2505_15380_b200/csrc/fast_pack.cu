@@ -236,6 +236,57 @@ void fast_pack_streams(const ssd_model_config& c, const FastPlan& plan, const ui
     }
 }
 
+// Inverse of fast_pack_streams, written as a consumer would walk the streams (chunk by chunk, a
+// chunk being whole k-steps of one round): scatters every tile back into a flat blob of the
+// ssd_model_create layout.  Returns the number of chunks whose size disagrees with the walk.
+long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, const uint8_t* streams,
+                              uint16_t* blob_out) {
+  const BlobView v = view_blob(c);
+  long long bad = 0;
+  for (int cta = 0; cta < plan.n_cta; ++cta)
+    for (int w = 0; w < FAST_WARPS; ++w) {
+      const size_t wi = (size_t)cta * FAST_WARPS + w;
+      const uint8_t* tab = plan.chunks.data() + wi * FAST_MAX_CHUNKS;
+      const int ncl = plan.chunk_cnt[wi * 2], nch = plan.chunk_cnt[wi * 2 + 1];
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(streams + plan.stream_off[wi]);
+      for (int l = 0; l <= c.n_layers; ++l) {
+        int ci = l < c.n_layers ? 0 : ncl;  // chunk cursor in the table
+        const int op_begin = l < c.n_layers ? 0 : FOP_HEAD, op_end = l < c.n_layers ? FOP_HEAD : FOP_COUNT;
+        for (int op = op_begin; op < op_end; ++op) {
+          const FastOpShape& s = plan.ops[op];
+          const int cnt_total = plan.unit_cnt[(size_t)cta * FOP_COUNT + op];
+          const int32_t* tiles = plan.unit_tile.data() + plan.unit_off[(size_t)cta * FOP_COUNT + op];
+          const int sk0 = fast_slice_k0(s, cta), steps = fast_slice_k1(s, cta) - sk0;
+          const int s0 = sk0 + fast_warp_k0(w, steps), s1 = sk0 + fast_warp_k1(w, steps);
+          for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
+            const int cnt = std::min(FAST_MAXU, cnt_total - u0), spc = fast_steps_per_chunk(cnt);
+            for (int sb = s0; sb < s1; sb += spc) {
+              const int nst = std::min(spc, s1 - sb);
+              if (tab[ci++] != nst * cnt) ++bad;
+              for (int i = 0; i < nst; ++i)
+                for (int u = 0; u < cnt; ++u) {
+                  for (int g = 0; g < 8; ++g) {
+                    uint16_t* row = const_cast<uint16_t*>(
+                        packed_row(c, v, blob_out, op, l < c.n_layers ? l : 0, tiles[u0 + u] * 8 + g));
+                    for (int t = 0; t < 4; ++t) {
+                      const uint32_t lo = src[(g * 4 + t) * 2], hi = src[(g * 4 + t) * 2 + 1];
+                      if (!row) continue;
+                      uint16_t* a = row + (size_t)(sb + i) * 16 + 2 * t;
+                      a[0] = (uint16_t)lo; a[1] = (uint16_t)(lo >> 16);
+                      a[8] = (uint16_t)hi; a[9] = (uint16_t)(hi >> 16);
+                    }
+                  }
+                  src += FAST_TILE_BYTES / 4;
+                }
+            }
+          }
+        }
+        if (l < c.n_layers ? ci != ncl : ci != ncl + nch) ++bad;
+      }
+    }
+  return bad;
+}
+
 void fast_pack_aux(const ssd_model_config& c, const uint16_t* blob, std::vector<float>& bias,
                    std::vector<float>& gains) {
   const BlobView v = view_blob(c);

@@ -168,3 +168,92 @@ def test_device_status_flags_and_host_errors():
                                 gs.ws.data_ptr(), gs.ws.numel(), ctypes.byref(h)) == -6
     assert L.ssd_streams_create(model.handle, 1, 16, 4, gs.kv_raw.data_ptr() + 2, 1 << 30,
                                 gs.ws.data_ptr(), gs.ws.numel(), ctypes.byref(h)) == -5
+
+
+# ---- the persistent small-batch kernel (forwards of <= 16 rows over a bf16 model) ---------------
+
+def _fast_shape(hd, hq=4, hkv=2, d=128, f=256, v=300, layers=2):
+    return synth.ModelShape(layers, d, hq, hkv, hd, f, v, 8, 1e4, weight_dtype=synth.BF16)
+
+
+@pytest.mark.parametrize("hd,batch,gamma,lens", [
+    (64, 1, 4, [20]), (64, 2, 2, [70, 129]), (32, 1, 8, [300]), (128, 3, 4, [1, 64, 700]),
+    (64, 1, 15, [33]), (64, 4, 3, [5, 127, 128, 129])])
+def test_persistent_kernel_against_oracle(hd, batch, gamma, lens):
+    """Rows <= 8 and <= 16, several streams in one forward, prefixes around the 16-key tiles and
+    the 128-key passes of the attention phase, all three head sizes."""
+    shape = _fast_shape(hd, hq=14 if hd == 64 else 4, hkv=2)
+    wl = _wl(shape, batch, gamma, lens)
+    _case(wl, beta=0.0, sigma=0.5, path=0)
+    _case(wl, beta=0.4, sigma=2.0, commit_and_repeat=True, path=0)
+
+
+def test_generic_kernels_still_cover_small_bf16_forwards():
+    shape = _fast_shape(64, hq=14, hkv=2)
+    _case(_wl(shape, 2, 4, [70, 129]), beta=0.0, sigma=0.5, path=1)
+
+
+def test_both_paths_agree_and_forward_only_matches():
+    from paper_2505_15380_b200 import binding
+    shape = _fast_shape(64, hq=14, hkv=2, d=256, f=1408, v=700, layers=3)   # FFN > 1280: K-split down
+    w = synth.make_weights(shape, 7)
+    model = binding.Model(shape, synth.weights_blob(shape, w))
+    dev = model.device
+    B, g, V = 2, 5, shape.vocab_out
+    lens = [140, 9]
+    p = torch.from_numpy(synth.random_prob_rows(B * g, V, 1).reshape(B, g, V)).to(dev)
+    x = torch.from_numpy(synth.sample_from_rows(p.reshape(-1, V).cpu().numpy(), 2).reshape(B, g)
+                         .astype(np.int32)).to(dev)
+    u = torch.from_numpy(synth.verify_uniforms(5, B, g + 1)).to(dev)
+    par = binding.VerifyParams(g, 0.9, 20, 0.2)
+    res = []
+    for path in (0, 1):
+        gs = binding.Streams(model, B, 200, g)
+        gs.set_path(path)
+        synth.fill_synthetic_kv(gs.kv, lens, seed=5)
+        gs.kv_truncate(lens, [3, 4])
+        k = torch.zeros(B, dtype=torch.int32, device=dev)
+        y = torch.zeros(B, dtype=torch.int32, device=dev)
+        lg = torch.zeros((B, g + 1, V), dtype=torch.float32, device=dev)
+        gs.verify(x, p, u, par, k, y, lg)
+        lf = torch.zeros_like(lg)
+        gs.forward(x, g, lf)                                  # the forward alone: same logits
+        torch.cuda.synchronize()
+        assert gs.last_status() == 0
+        assert torch.equal(lf, lg)
+        res.append((lg.cpu(), k.cpu(), y.cpu(), gs.kv[:, :, :, :, :150].float().cpu()))
+    assert (res[0][0] - res[1][0]).abs().max() < 2e-3
+    assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+    # the appended K/V rows agree up to the storage rounding of values that differ in the last bits
+    n0 = lens[0]
+    assert (res[0][3][:, 0, :, :, n0:n0 + g + 1] - res[1][3][:, 0, :, :, n0:n0 + g + 1]).abs().max() < 2e-2
+
+
+def test_phase_trace_of_the_persistent_kernel():
+    from paper_2505_15380_b200 import binding
+    shape = _fast_shape(64)
+    w = synth.make_weights(shape, 3)
+    model = binding.Model(shape, synth.weights_blob(shape, w))
+    dev = model.device
+    gs = binding.Streams(model, 1, 64, 4)
+    gs.kv_truncate([0], [3])
+    V = shape.vocab_out
+    x = torch.zeros((1, 4), dtype=torch.int32, device=dev)
+    lg = torch.zeros((1, 5, V), dtype=torch.float32, device=dev)
+    buf = torch.zeros((256, 64), dtype=torch.int64, device=dev)
+    gs.set_trace(buf)
+    gs.forward(x, 4, lg)
+    torch.cuda.synchronize()
+    t = buf.cpu().numpy()
+    n_events = 3 + 2 * 5 * shape.n_layers + 1               # set-up, embedding + barrier, phases, head
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    for cta in (0, sms - 1):
+        row = t[cta]
+        assert np.count_nonzero(row) == n_events
+        assert np.all(np.diff(row[:n_events]) > 0)           # one SM's clock only moves forward
+    assert not t[sms:].any()
+    gs.set_trace(None)
+    buf.zero_()
+    gs.forward(x, 4, lg)
+    torch.cuda.synchronize()
+    assert not buf.any()
