@@ -31,7 +31,7 @@ namespace ssd {
 namespace {
 
 constexpr unsigned long long FAST_WAIT_CYCLES = 3000000000ull;  // ~1.5 s at 2 GHz
-constexpr int FAST_KEYS_MIN = 128;                               // fewest keys worth a split of their own
+constexpr int FAST_KEYS_MIN = 384;                               // fewest keys worth a split of their own
 constexpr float FIX_SCALE = 4294967296.f;                        // residual stream: 2^-32 fixed point
 constexpr float FIX_INV_SCALE = 1.f / 4294967296.f;
 
@@ -309,7 +309,7 @@ __device__ __forceinline__ void stage_copy_warp(const uint32_t* __restrict__ src
 // inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
 // warp per row, fixed summation order.  The loads are issued at the start of the phase and
 // summed after the tensor-core work, so their latency stays off the critical path.
-constexpr int SSQ_REGS = 8;  // covers d <= 2048 in one go
+constexpr int SSQ_REGS = 4;  // covers d <= 1024 in one go
 struct SsqLoads {
   float v[2][SSQ_REGS];  // rows warp and warp + FAST_WARPS
 };
@@ -597,34 +597,39 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   return v;
 }
 
-// Work item = (stream, query head, key split).  Per pass of up to 16 keys per warp the item's CTA
-// stages the keys / values (bf16, as cached) in shared memory and runs both contractions on the
-// tensor cores: scores S[key, row] = K[key, :] . q[row, :] (q arrives pre-split in operand layout
-// from the QKV epilogue) and O[row, :] += P[row, key] V[key, :] (P split into bf16 hi + lo, V read
-// with a transposing matrix load), with a running max / sum per row in between.  Row r of a stream
-// sees keys 0..len + r: causal inside the draft block.  The operand rows are the forward's rows
-// (all streams); rows of other streams are masked out.  With more than one split the partials go
-// to global memory and the CTA that arrives last for a (stream, head) merges them in split order.
+// Work item = (stream, query head, key split).  Every warp of the item's CTA works through its
+// own 16-key tiles from start to end (keys 16 w, 16 w + 128, ... of the split): it stages the
+// tile's keys / values (bf16, as cached) in its private part of shared memory, computes the scores
+// S[row, key] = q[row, :] . K[key, :] on the tensor cores (q arrives pre-split in operand layout
+// from the QKV epilogue), keeps a running max / sum per row in registers, and accumulates
+// O[row, :] += P[row, key] V[key, :] with P taken straight from the score registers (split into
+// bf16 hi + lo) and V read with a transposing matrix load.  One CTA barrier later the eight warps'
+// partials are combined.  Row r of a stream sees keys 0..len + r: causal inside the draft block.
+// The operand rows are the forward's rows (all streams); rows of other streams are masked out.
+// With more than one split the partials go to global memory and the CTA that arrives last for a
+// (stream, head) merges them in split order.
 template <int HD, bool T16>
-__device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_t* uni, int layer) {
-  constexpr int KT = 16 * FAST_WARPS;     // keys per pass
+__device__ __forceinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_t* uni, int layer) {
   constexpr int ROWB = HD * 2 + 16;       // padded K / V row in bytes (conflict-free fragment loads)
-  constexpr int NT = T16 ? 2 : 1;         // 8-row tiles of the forward's rows
+  constexpr int NH = T16 ? 2 : 1;         // row halves: rows g and g + 8
   constexpr int W = T16 ? 8 : 4;          // words per (k-step, lane) of an operand
   constexpr int KSTEPS = HD / 16;
   constexpr int DT = HD / 8;              // 8-dim tiles of the output
-  constexpr int DPW = (DT + FAST_WARPS - 1) / FAST_WARPS;
   constexpr int CH = HD / 8;              // 16-byte chunks per row
+  constexpr int LPL = 16 * CH / 32;       // 16-byte loads per lane for 16 rows
+  constexpr int NROW = 8 * NH;            // rows held
   const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   const int nsplit = M.attn_nsplit, items = nb * Hq * nsplit;
 
-  uint8_t* Ks = uni;                                             // [KT][ROWB]
-  uint8_t* Vs = Ks + KT * ROWB;                                  // [KT][ROWB]
-  uint32_t* ps = reinterpret_cast<uint32_t*>(Vs + KT * ROWB);    // weights P, operand layout, KT / 16 steps
-  const uint32_t ks_lane = smem_u32(Ks) + (16 * warp + g) * ROWB + t * 4;
-  const uint32_t vs_lane = smem_u32(Vs) + (lane & 15) * ROWB;
-  const uint32_t ps_lane = smem_u32(ps) + lane * (W * 4);
+  uint32_t* qsm = reinterpret_cast<uint32_t*>(uni);                       // q operand, KSTEPS steps
+  uint8_t* kv_w = uni + KSTEPS * 32 * W * 4 + warp * (2 * 16 * ROWB);     // this warp's K then V tile
+  float* cm = reinterpret_cast<float*>(uni + KSTEPS * 32 * W * 4 + FAST_WARPS * 2 * 16 * ROWB);  // [warp][NROW]
+  float* cl = cm + FAST_WARPS * NROW;
+  float* co = cl + FAST_WARPS * NROW;                                      // [warp][NROW][HD]
+  const uint32_t q_lane = smem_u32(qsm) + lane * (W * 4);
+  const uint32_t k_lane = smem_u32(kv_w) + g * ROWB + t * 4;
+  const uint32_t v_lane = smem_u32(kv_w) + 16 * ROWB + (lane & 15) * ROWB;
   const bf16* kvl = P.kv + (size_t)layer * P.kv_layer_elems;
 
   for (int item = blockIdx.x; item < items; item += P.m.n_cta) {
@@ -639,198 +644,177 @@ __device__ __noinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_
     }
     const int stream = P.b0 + bi, gk = hq / G, t_lo = bi * R, t_hi = t_lo + R;
     const int L = M.tok_pos[t_lo];
-    __syncthreads();
-    if (tid < FAST_MAX_T) {
-      M.row_m[tid] = -CUDART_INF_F;
-      M.row_l[tid] = 0.f;
+    const uint4* kg = reinterpret_cast<const uint4*>(kvl + (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * HD);
+    const uint4* vg = reinterpret_cast<const uint4*>(kvl + (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD);
+
+    // first tile of this warp: loads in flight before anything else
+    int key0 = k0 + 16 * warp;
+    uint4 kq[LPL], vq[LPL];
+#pragma unroll
+    for (int i = 0; i < LPL; ++i) {
+      const int idx = lane + 32 * i, key = key0 + idx / CH;
+      kq[i] = vq[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (key < k1) {
+        kq[i] = __ldcg(kg + (size_t)key * CH + idx % CH);
+        vq[i] = __ldcg(vg + (size_t)key * CH + idx % CH);
+      }
     }
-    WMARK(60);
-    // q of this head: B operand of the score contraction, bf16 hi / lo as the QKV epilogue left it
-    uint4 qf[KSTEPS][NT];
-#pragma unroll
-    for (int s = 0; s < KSTEPS; ++s) {
-      const uint4* src = reinterpret_cast<const uint4*>(P.xq + ((size_t)(hq * KSTEPS + s) * 32 + lane) * W);
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) qf[s][nt] = __ldcg(src + nt);
+    __syncthreads();  // the previous user of the shared memory (projection phase or item) is done
+    {                 // q of this head (operand layout, bf16 hi / lo as the QKV epilogue left it)
+      const uint4* src = reinterpret_cast<const uint4*>(P.xq + (size_t)hq * KSTEPS * 32 * W);
+      for (int i = tid; i < KSTEPS * 32 * W / 4; i += FAST_THREADS) reinterpret_cast<uint4*>(qsm)[i] = __ldcg(src + i);
     }
-    float o[DPW][4];
-#pragma unroll
-    for (int dp = 0; dp < DPW; ++dp) o[dp][0] = o[dp][1] = o[dp][2] = o[dp][3] = 0.f;
-    const size_t kbase = (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * HD;
-    const size_t vbase = (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD;
     if (layer + 1 < P.L) {
       // the same keys and values of the next layer (the cached prefix does not change during the
       // forward): pull them into L2 now, one 128-byte line per thread and pass
-      const uint8_t* nk_ = reinterpret_cast<const uint8_t*>(kvl + P.kv_layer_elems + kbase + (size_t)k0 * HD);
-      const uint8_t* nv_ = reinterpret_cast<const uint8_t*>(kvl + P.kv_layer_elems + vbase + (size_t)k0 * HD);
+      const uint8_t* nk_ = reinterpret_cast<const uint8_t*>(kg) + P.kv_layer_elems * 2 + (size_t)k0 * HD * 2;
+      const uint8_t* nv_ = reinterpret_cast<const uint8_t*>(vg) + P.kv_layer_elems * 2 + (size_t)k0 * HD * 2;
       const int lines = ((k1 - k0) * HD * 2 + 127) >> 7;
       for (int i = tid; i < lines; i += FAST_THREADS) {
         prefetch_l2(nk_ + (size_t)i * 128);
         prefetch_l2(nv_ + (size_t)i * 128);
       }
     }
-
-    for (int kt0 = k0; kt0 < k1; kt0 += KT) {
-      const int nk = min(KT, k1 - kt0), nk16 = (nk + 15) & ~15;
-      __syncthreads();
-      WMARK(61);
-      {  // keys and values of this pass -> shared memory; rows up to the next multiple of 16 are zeroed
-        const uint4* ksrc = reinterpret_cast<const uint4*>(kvl + kbase + (size_t)kt0 * HD);
-        const uint4* vsrc = reinterpret_cast<const uint4*>(kvl + vbase + (size_t)kt0 * HD);
-        constexpr int CB = KT * CH / FAST_THREADS;
-        uint4 kq[CB], vq[CB];
-#pragma unroll
-        for (int i = 0; i < CB; ++i) {
-          const int idx = tid + i * FAST_THREADS;
-          kq[i] = vq[i] = make_uint4(0u, 0u, 0u, 0u);
-          if (idx < nk * CH) {
-            kq[i] = __ldcg(ksrc + idx);
-            vq[i] = __ldcg(vsrc + idx);
-          }
-        }
-#pragma unroll
-        for (int i = 0; i < CB; ++i) {
-          const int idx = tid + i * FAST_THREADS;
-          if (idx < nk16 * CH) {
-            *reinterpret_cast<uint4*>(Ks + (idx / CH) * ROWB + (idx % CH) * 16) = kq[i];
-            *reinterpret_cast<uint4*>(Vs + (idx / CH) * ROWB + (idx % CH) * 16) = vq[i];
-          }
-        }
-      }
-      WMARK(62);
-      __syncthreads();
-      WMARK(63);
-      // scores of this warp's 16 keys against all rows; thread: keys g, g + 8 x rows 2t, 2t + 1 (+ 8)
-      const bool active = 16 * warp < nk;
-      float sc[NT][4];
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-      if (active) {
-#pragma unroll
-        for (int s = 0; s < KSTEPS; ++s) {
-          uint32_t a[4];
-          a[0] = lds_u32(ks_lane + s * 32);
-          a[1] = lds_u32(ks_lane + s * 32 + 8 * ROWB);
-          a[2] = lds_u32(ks_lane + s * 32 + 16);
-          a[3] = lds_u32(ks_lane + s * 32 + 8 * ROWB + 16);
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt) {
-            mma_bf16(sc[nt], a, qf[s][nt].x, qf[s][nt].y);
-            mma_bf16(sc[nt], a, qf[s][nt].z, qf[s][nt].w);
-          }
-        }
-      }
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int key = 16 * warp + g + (i >> 1) * 8, tok = nt * 8 + 2 * t + (i & 1);
-          const bool valid = active && key < nk && tok >= t_lo && tok < t_hi && kt0 + key <= L + (tok - t_lo);
-          if (!valid) sc[nt][i] = -CUDART_INF_F;
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          float v = fmaxf(sc[nt][j], sc[nt][j + 2]);
-          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
-          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
-          v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
-          if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
-        }
-      }
-      WMARK(64);
-      __syncthreads();
-      WMARK(65);
-      if (tid < 8 * NT) {
-        float mt = M.wred[0][tid];
-#pragma unroll
-        for (int w = 1; w < FAST_WARPS; ++w) mt = fmaxf(mt, M.wred[w][tid]);
-        const float m_old = M.row_m[tid], m_new = fmaxf(m_old, mt);
-        M.row_corr[tid] = m_new == -CUDART_INF_F ? 0.f : __expf(m_old - m_new);
-        M.row_m[tid] = m_new;
-      }
-      WMARK(66);
-      __syncthreads();
-      WMARK(67);
-      // weights, their row sums, and P in operand layout for the second contraction
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        float pw[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float m = M.row_m[nt * 8 + 2 * t + (i & 1)];
-          pw[i] = sc[nt][i] == -CUDART_INF_F ? 0.f : __expf(sc[nt][i] - m);
-          if (active) write_frag_elem<T16>(ps, nt * 8 + 2 * t + (i & 1), 16 * warp + g + (i >> 1) * 8, pw[i]);
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          float v = pw[j] + pw[j + 2];
-          v += __shfl_xor_sync(0xffffffffu, v, 4);
-          v += __shfl_xor_sync(0xffffffffu, v, 8);
-          v += __shfl_xor_sync(0xffffffffu, v, 16);
-          if (g == 0) M.wred[warp][nt * 8 + 2 * t + j] = v;
-        }
-      }
-      WMARK(68);
-      __syncthreads();
-      WMARK(69);
-      if (tid < 8 * NT) {
-        float lt = 0.f;
-#pragma unroll
-        for (int w = 0; w < FAST_WARPS; ++w) lt += M.wred[w][tid];
-        M.row_l[tid] = M.row_l[tid] * M.row_corr[tid] + lt;
-      }
-      // O += P V: this warp owns 8-dim tiles of the output
-      const float c0 = M.row_corr[g], c1 = T16 ? M.row_corr[g + 8] : 0.f;
-#pragma unroll
-      for (int dp = 0; dp < DPW; ++dp) {
-        const int dtile = warp + dp * FAST_WARPS;
-        if (dtile < DT) {
-          o[dp][0] *= c0; o[dp][1] *= c0; o[dp][2] *= c1; o[dp][3] *= c1;
-          for (int ks = 0; ks < (nk16 >> 4); ++ks) {
-            const uint4 pa = lds_v4(ps_lane + ks * (32 * W * 4));
-            uint32_t ahi[4] = {pa.x, 0u, pa.y, 0u}, alo[4] = {pa.z, 0u, pa.w, 0u};
-            if (T16) {
-              const uint4 pb = lds_v4(ps_lane + ks * (32 * W * 4) + 16);
-              ahi[1] = pb.x; ahi[3] = pb.y; alo[1] = pb.z; alo[3] = pb.w;
-            }
-            uint32_t b0, b1;
-            ldmatrix_x2_trans(vs_lane + ks * 16 * ROWB + dtile * 16, b0, b1);
-            mma_bf16(o[dp], ahi, b0, b1);
-            mma_bf16(o[dp], alo, b0, b1);
-          }
-        }
-      }
-    }
-    WMARK(70);
     __syncthreads();
-    WMARK(71);
-    // output: thread holds rows g (and g + 8) x dims 2t, 2t + 1 of its tiles
+
+    float m_run[NH], l_run[NH], o[DT][4];
 #pragma unroll
-    for (int dp = 0; dp < DPW; ++dp) {
-      const int dtile = warp + dp * FAST_WARPS;
-      if (dtile < DT) {
+    for (int h = 0; h < NH; ++h) { m_run[h] = -CUDART_INF_F; l_run[h] = 0.f; }
 #pragma unroll
-        for (int h = 0; h < NT; ++h) {
-          const int tok = g + 8 * h, dd = dtile * 8 + 2 * t;
-          if (tok >= t_lo && tok < t_hi) {
-            const float o0 = o[dp][2 * h], o1 = o[dp][2 * h + 1];
-            if (nsplit == 1) {
-              const float il = 1.f / M.row_l[tok];
-              write_frag_pair<T16>(P.xo, tok, hq * HD + dd, o0 * il, o1 * il);
-            } else {
-              float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
-              *reinterpret_cast<float2*>(dst + dd) = make_float2(o0, o1);
-              if (dd == 0) *reinterpret_cast<float2*>(dst + HD) = make_float2(M.row_m[tok], M.row_l[tok]);
-            }
+    for (int dt = 0; dt < DT; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
+
+    for (; key0 < k1; key0 += 16 * FAST_WARPS) {
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < LPL; ++i) {
+        const int idx = lane + 32 * i;
+        *reinterpret_cast<uint4*>(kv_w + (idx / CH) * ROWB + (idx % CH) * 16) = kq[i];
+        *reinterpret_cast<uint4*>(kv_w + 16 * ROWB + (idx / CH) * ROWB + (idx % CH) * 16) = vq[i];
+      }
+      __syncwarp();
+      {  // the next tile's loads, in flight during this tile's arithmetic
+        const int nkey0 = key0 + 16 * FAST_WARPS;
+#pragma unroll
+        for (int i = 0; i < LPL; ++i) {
+          const int idx = lane + 32 * i, key = nkey0 + idx / CH;
+          kq[i] = vq[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (key < k1) {
+            kq[i] = __ldcg(kg + (size_t)key * CH + idx % CH);
+            vq[i] = __ldcg(vg + (size_t)key * CH + idx % CH);
           }
         }
       }
+      // scores: thread holds rows g (and g + 8) x keys 8j + 2t, 8j + 2t + 1 of the tile
+      float sc[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+      for (int s = 0; s < KSTEPS; ++s) {
+        const uint4 qa = lds_v4(q_lane + s * (32 * W * 4));
+        uint32_t ahi[4] = {qa.x, 0u, qa.y, 0u}, alo[4] = {qa.z, 0u, qa.w, 0u};
+        if (T16) {
+          const uint4 qb = lds_v4(q_lane + s * (32 * W * 4) + 16);
+          ahi[1] = qb.x; ahi[3] = qb.y; alo[1] = qb.z; alo[3] = qb.w;
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const uint32_t b0 = lds_u32(k_lane + j * 8 * ROWB + s * 32), b1 = lds_u32(k_lane + j * 8 * ROWB + s * 32 + 16);
+          mma_bf16(sc[j], ahi, b0, b1);
+          mma_bf16(sc[j], alo, b0, b1);
+        }
+      }
+      // mask, running max / sum, weights as the A operand of the second contraction
+      uint32_t phi[4], plo[4];
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const int tok = g + 8 * h;
+        const bool rowok = tok >= t_lo && tok < t_hi;
+        float mt = -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int key = key0 + 8 * j + 2 * t + i;
+            if (!(rowok && key < k1 && key <= L + (tok - t_lo))) sc[j][2 * h + i] = -CUDART_INF_F;
+            mt = fmaxf(mt, sc[j][2 * h + i]);
+          }
+        }
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+        const float m_new = fmaxf(m_run[h], mt);
+        const float corr = m_new == -CUDART_INF_F ? 0.f : __expf(m_run[h] - m_new);
+        float pw[2][2], ls = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            pw[j][i] = sc[j][2 * h + i] == -CUDART_INF_F ? 0.f : __expf(sc[j][2 * h + i] - m_new);
+            ls += pw[j][i];
+          }
+        }
+        ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+        ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+        l_run[h] = l_run[h] * corr + ls;
+        m_run[h] = m_new;
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt) { o[dt][2 * h] *= corr; o[dt][2 * h + 1] *= corr; }
+        split2(pw[0][0], pw[0][1], phi[h], plo[h]);          // keys 2t, 2t + 1
+        split2(pw[1][0], pw[1][1], phi[2 + h], plo[2 + h]);  // keys 8 + 2t, 8 + 2t + 1
+      }
+      if (!T16) phi[1] = phi[3] = plo[1] = plo[3] = 0u;
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        uint32_t b0, b1;
+        ldmatrix_x2_trans(v_lane + dt * 16, b0, b1);
+        mma_bf16(o[dt], phi, b0, b1);
+        mma_bf16(o[dt], plo, b0, b1);
+      }
     }
-    WMARK(72);
+    // this warp's partial -> shared memory; then all warps combine
+    if (t == 0) {
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        cm[warp * NROW + g + 8 * h] = m_run[h];
+        cl[warp * NROW + g + 8 * h] = l_run[h];
+      }
+    }
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) {
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+        *reinterpret_cast<float2*>(co + ((size_t)warp * NROW + g + 8 * h) * HD + dt * 8 + 2 * t) =
+            make_float2(o[dt][2 * h], o[dt][2 * h + 1]);
+    }
+    __syncthreads();
+    for (int idx = tid; idx < R * (HD / 2); idx += FAST_THREADS) {  // (row of the stream, dim pair)
+      const int r = idx / (HD / 2), dd = (idx % (HD / 2)) * 2, tok = t_lo + r;
+      float mw[FAST_WARPS], m = -CUDART_INF_F;
+#pragma unroll
+      for (int w = 0; w < FAST_WARPS; ++w) {
+        mw[w] = cm[w * NROW + tok];
+        m = fmaxf(m, mw[w]);
+      }
+      float l = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+      for (int w = 0; w < FAST_WARPS; ++w) {  // fixed order: bit-reproducible
+        const float e = mw[w] == -CUDART_INF_F ? 0.f : __expf(mw[w] - m);
+        const float2 ov = *reinterpret_cast<const float2*>(co + ((size_t)w * NROW + tok) * HD + dd);
+        l = fmaf(cl[w * NROW + tok], e, l);
+        o0 = fmaf(ov.x, e, o0);
+        o1 = fmaf(ov.y, e, o1);
+      }
+      if (nsplit == 1) {
+        const float il = 1.f / l;
+        write_frag_pair<T16>(P.xo, tok, hq * HD + dd, o0 * il, o1 * il);
+      } else {
+        float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
+        *reinterpret_cast<float2*>(dst + dd) = make_float2(o0, o1);
+        if (dd == 0) *reinterpret_cast<float2*>(dst + HD) = make_float2(m, l);
+      }
+    }
     if (nsplit > 1) {
       __threadfence();
       __syncthreads();
-      WMARK(73);
       if (tid == 0) {
         int prev = atomicAdd(&P.attn_counters[bi * Hq + hq], 1);
         M.last = prev == nsplit - 1;
@@ -1095,8 +1079,9 @@ size_t fast_union_bytes(int stage_k, int hd, int T, int R) {
   const bool t16 = T > 8;
   size_t af = (size_t)(stage_k / 16) * (t16 ? 1024 : 512);
   size_t red = (size_t)FAST_WARPS * FAST_MAXU * 32 * (t16 ? 16 : 8);
-  const int KT = 16 * FAST_WARPS;
-  size_t attn = (size_t)2 * KT * (hd * 2 + 16) + (size_t)(KT / 16) * 32 * (t16 ? 32 : 16);
+  const int nrow = t16 ? 16 : 8;  // q operand, per-warp K / V tiles, per-warp partials (m, l, O)
+  size_t attn = (size_t)(hd / 16) * 32 * (t16 ? 32 : 16) + (size_t)FAST_WARPS * 2 * 16 * (hd * 2 + 16) +
+                (size_t)FAST_WARPS * nrow * (hd + 2) * 4;
   (void)R;
   size_t u = af + red > attn ? af + red : attn;
   return (u + 127) / 128 * 128;
