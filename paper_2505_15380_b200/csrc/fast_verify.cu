@@ -102,6 +102,7 @@ __device__ __forceinline__ float fix_to_float(long long v) {
 // Per-CTA bookkeeping in shared memory.
 struct FastMisc {
   unsigned long long bars[FAST_WARPS][FAST_MAX_SLOTS];
+  unsigned long long sbar[FAST_WARPS];          // per warp: arrival of its slice of the A operand
   uint8_t chunks[FAST_WARPS][FAST_MAX_CHUNKS];  // chunk sizes (tiles) of each warp's stream
   int32_t ucnt[FOP_COUNT];
   int32_t utile[FOP_COUNT][FAST_MAX_UNITS];
@@ -521,7 +522,7 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 // split K), add the warps' partial sums in shared memory and apply the epilogue.
 template <bool T16>
 __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
-                                           const PhaseDesc& D) {
+                                           const PhaseDesc& D, uint32_t& stage_parity) {
   constexpr int NACC = T16 ? 4 : 2;
   const int cnt_total = M.ucnt[D.op];
   if (cnt_total == 0) return;
@@ -534,7 +535,20 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   SsqLoads ssq;
   if (D.in_fix) ssq_issue(ssq, D.ssq_in, P.d >> 3, T);
   const bool row0 = g < T, row1 = T16 && g + 8 < T;
-  stage_copy_warp<T16>(D.xin, af, s0, s1, lane);
+  // this warp's k-steps of the operand: one bulk copy from L2 (the producers' stores were made
+  // visible by the grid barrier; the proxy fence orders that observation before the async read)
+  const uint32_t sbar = smem_u32(&M.sbar[warp]);
+  const uint32_t stage_bytes = (uint32_t)(s1 - s0) * (T16 ? 1024u : 512u);
+  if (stage_bytes && lane == 0) {
+    asm volatile("fence.proxy.async;" ::: "memory");
+    mbar_expect_tx(sbar, stage_bytes);
+    bulk_g2s(smem_u32(af) + (uint32_t)s0 * (T16 ? 1024u : 512u),
+             reinterpret_cast<const uint8_t*>(D.xin) + (size_t)s0 * (T16 ? 1024 : 512), stage_bytes, sbar);
+  }
+  if (stage_bytes) {
+    if (!mbar_try_wait(sbar, stage_parity) && !bounded_mbar_wait(sbar, stage_parity)) ring.dead = true;
+    stage_parity ^= 1u;
+  }
   WMARK(D.op * 10 + 2);
   const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
   float* red_dst = red + ((size_t)warp * FAST_MAXU * 32 + lane) * NACC;
@@ -920,7 +934,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   ring.nslot = (uint32_t)P.nslot;
   ring.outstanding = 0;
   ring.dead = false;
+  uint32_t stage_parity = 0;
   if (lane == 0) {
+    mbar_init(smem_u32(&M.sbar[warp]), 1);
     for (int s = 0; s < P.nslot; ++s) mbar_init(ring.bars + s * 8, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1032,7 +1048,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
         D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
         D.layer = 0; D.kc = d; D.n_rows = P.V;
       }
-      gemm_phase<T16>(P, M, uni, ring, D);
+      gemm_phase<T16>(P, M, uni, ring, D, stage_parity);
     }
     trace_mark(P, n_trace);
 #ifdef SSD_TRACE_FINE
