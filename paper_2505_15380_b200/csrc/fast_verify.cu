@@ -9,11 +9,13 @@
 // The phases of a layer (QKV projection, attention, O projection, gate/up, down) are separated by
 // grid barriers on one monotonic arrival counter, with bounded waits.
 //
-// The forward is a chain of ~5 dependent phases per layer, each far shorter than a microsecond of
-// memory time, so what bounds it is the number of instructions a warp executes per phase (eight
-// warps per SM hide little latency).  Hence: activations are converted once per phase into the
-// tensor-core operand layout, the weight stream is pre-cut into chunks of whole k-steps so the
-// inner loop is straight-line for each tile count, and everything rare is out of line.
+// The forward is a chain of 5 dependent phases per layer, each far shorter than a microsecond of
+// memory time, so what bounds it is latency: the instructions a warp executes per phase (eight
+// warps per SM hide little) and the round trips through L2 between phases.  Hence: every activation
+// is converted to the tensor-core operand layout (bf16 hi + lo) once, by the thread that produces
+// it, and consumers fetch their slice with one bulk copy; the weight stream is pre-cut into chunks
+// of whole k-steps so the inner loop is straight-line for each tile count; everything rare is out
+// of line; attention keeps its weights in registers between its two contractions.
 //
 // Projections: D[token, weight row] = sum_k X[token, k] * W[row, k] on mma.m16n8k16 (bf16 inputs,
 // fp32 accumulate): the 16-row A operand holds the tokens, the B operand one packed tile of 8 weight
@@ -21,7 +23,6 @@
 // products are exact to ~2^-17 relative; weights are exactly their stored bf16 values.  The warps
 // of a CTA split K; their partial sums are added in a fixed order in shared memory.
 #include <math_constants.h>
-#include <stdlib.h>
 
 #include "fast.h"
 #include "kernels.h"
@@ -182,18 +183,6 @@ __device__ __forceinline__ void ring_release(Ring& r, int lane) {
   }
 }
 
-#ifdef SSD_TRACE_FINE
-// debug build: every warp's clock at marked points of one layer, kept in shared memory
-__shared__ unsigned int g_wtr[FAST_WARPS][96];
-__shared__ int g_wtr_on;
-#define WMARK(i)                                                                         \
-  do {                                                                                   \
-    if (g_wtr_on && (threadIdx.x & 31) == 0) g_wtr[threadIdx.x >> 5][(i)] = (unsigned)clock64(); \
-  } while (0)
-#else
-#define WMARK(i) do {} while (0)
-#endif
-
 __device__ __forceinline__ void trace_mark(const FastParams& P, int& n_trace) {
   if (P.trace && threadIdx.x == 0 && n_trace < P.trace_cap)
     P.trace[(size_t)blockIdx.x * P.trace_cap + n_trace++] = clock64();
@@ -282,29 +271,6 @@ __device__ __forceinline__ void write_frag_elem(uint32_t* buf, int row, int k, f
   bf16* w = reinterpret_cast<bf16*>(buf + afrag_word<T16>(row, k >> 1)) + (k & 1);
   w[0] = h;
   w[4] = l;  // two words on
-}
-
-// Copies this warp's k-steps [s0, s1) of an operand-layout input from global memory (written by
-// other CTAs in an earlier phase, hence read past L1) to the same place in the shared-memory image.
-// A warp only ever multiplies with its own K slice, so the staging needs no CTA-wide barrier.
-// All loads are in flight before the first store.
-template <bool T16>
-__device__ __forceinline__ void stage_copy_warp(const uint32_t* __restrict__ src, uint32_t* af, int s0,
-                                                int s1, int lane) {
-  constexpr int LB = 8, V = T16 ? 2 : 1;  // 16-byte vectors per lane and step
-  const uint4* s4 = reinterpret_cast<const uint4*>(src) + (size_t)s0 * 32 * V;
-  uint4* d4 = reinterpret_cast<uint4*>(af) + (size_t)s0 * 32 * V;
-  const int n16 = (s1 - s0) * 32 * V;
-  for (int i0 = lane; i0 < n16; i0 += LB * 32) {
-    uint4 v[LB];
-#pragma unroll
-    for (int i = 0; i < LB; ++i)
-      if (i0 + i * 32 < n16) v[i] = __ldcg(s4 + i0 + i * 32);
-#pragma unroll
-    for (int i = 0; i < LB; ++i)
-      if (i0 + i * 32 < n16) d4[i0 + i * 32] = v[i];
-  }
-  __syncwarp();
 }
 
 // inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
@@ -461,7 +427,7 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
 // per chunk (one ring slot = SPC whole k-steps), partial sums to shared memory at the end.
 template <int CNT, bool T16>
 __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, int s0, int s1, bool row0,
-                                          bool row1, float* red_dst, int mark = 0) {
+                                          bool row1, float* red_dst) {
   constexpr int SPC = FAST_SLOT_TILES / CNT;
   constexpr uint32_t STEP = T16 ? 1024u : 512u;
   constexpr int NACC = T16 ? 4 : 2;
@@ -474,7 +440,6 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 #pragma unroll 1
   for (int s = s0; s < s1; s += SPC) {
     ring_acquire(r);
-    if (s == s0) WMARK(mark + 6);
     const uint32_t wb = r.ring + r.slot * FAST_SLOT_BYTES + lane * 8;
 #pragma unroll
     for (int i = 0; i < SPC; ++i) {
@@ -499,9 +464,7 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
         for (int u = 0; u < CNT; ++u) mma_bf16(TWO ? acl[u] : acc[u], alo, b[u].x, b[u].y);
       }
     }
-    if (s == s0) WMARK(mark + 7);
     ring_release(r, lane);
-    if (s == s0) WMARK(mark + 8);
   }
   if (TWO) {
 #pragma unroll
@@ -530,7 +493,6 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   const int KS = D.kc >> 4;
   uint32_t* af = reinterpret_cast<uint32_t*>(uni);                             // A operand, KS steps
   float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
-  WMARK(D.op * 10 + 0);
   const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
   SsqLoads ssq;
   if (D.in_fix) ssq_issue(ssq, D.ssq_in, P.d >> 3, T);
@@ -549,26 +511,23 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
     if (!mbar_try_wait(sbar, stage_parity) && !bounded_mbar_wait(sbar, stage_parity)) ring.dead = true;
     stage_parity ^= 1u;
   }
-  WMARK(D.op * 10 + 2);
   const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
   float* red_dst = red + ((size_t)warp * FAST_MAXU * 32 + lane) * NACC;
 
   for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
     const int cnt = min(FAST_MAXU, cnt_total - u0);
     switch (cnt) {
-      case 1: mma_round<1, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 2: mma_round<2, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 3: mma_round<3, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 4: mma_round<4, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
-      default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst, D.op * 10); break;
+      case 1: mma_round<1, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 2: mma_round<2, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 3: mma_round<3, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 4: mma_round<4, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
     }
     if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
-    WMARK(D.op * 10 + 3);
     __syncthreads();
-    WMARK(D.op * 10 + 4);
     for (int idx = tid; idx < cnt * 32; idx += FAST_THREADS) {  // whole warps: one tile per warp pass
       const int u = idx >> 5, l = idx & 31, gg = l >> 2, tt = l & 3;
       float c[NACC];
@@ -595,7 +554,6 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
         }
       }
     }
-    WMARK(D.op * 10 + 5);
     if (u0 + FAST_MAXU < cnt_total) __syncthreads();
   }
 }
@@ -1002,11 +960,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
 #pragma unroll 1
   for (int it = 0; it < n_phase && ok; ++it) {
     if (it == 5 * P.L) ph = 5;
-#ifdef SSD_TRACE_FINE
-    if (tid == 0) g_wtr_on = (l == 5 && ph < 5);
-    __syncthreads();
-    WMARK(50 + ph * 2);
-#endif
     if (ph == 0 && cta == (l % P.m.n_cta) + 0 && l + 1 < P.L) {
       // the small per-layer constants are read once per forward, so they would miss all the way
       // to HBM in the middle of an epilogue: one CTA pulls the next layer's into L2 ahead of time
@@ -1051,16 +1004,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       gemm_phase<T16>(P, M, uni, ring, D, stage_parity);
     }
     trace_mark(P, n_trace);
-#ifdef SSD_TRACE_FINE
-    WMARK(51 + ph * 2);
-    if (g_wtr_on && ph < 5 && P.trace) {   // dump this phase's marks: trace[cta][100 + ph*8*16 + warp*16 + k]
-      __syncthreads();
-      if (lane < 16) {
-        int src = ph == 1 ? (lane < 14 ? 60 + lane : (lane == 14 ? 50 + ph * 2 : 51 + ph * 2)) : lane < 9 ? ((ph == 0 ? 0 : ph == 2 ? 10 : ph == 3 ? 20 : 30) + lane) : (lane == 9 ? 50 + ph * 2 : lane == 10 ? 51 + ph * 2 : 95);
-        P.trace[(size_t)blockIdx.x * P.trace_cap + 400 + (ph * FAST_WARPS + warp) * 16 + lane] = g_wtr[warp][src];
-      }
-    }
-#endif
     if (ph < 5) {
       ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
       trace_mark(P, n_trace);
@@ -1117,7 +1060,7 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   int nslot = (int)((max_smem - uni - misc) / ((size_t)FAST_WARPS * FAST_SLOT_BYTES));
   if (nslot > FAST_RING_SLOTS) nslot = FAST_RING_SLOTS;
   p.nslot = nslot;
-  p.keys_min = getenv("SSD_KEYS_MIN") ? atoi(getenv("SSD_KEYS_MIN")) : FAST_KEYS_MIN;
+  p.keys_min = FAST_KEYS_MIN;
   p.ring_warp_bytes = nslot * FAST_SLOT_BYTES;
   p.union_off = FAST_WARPS * p.ring_warp_bytes;
   p.misc_off = p.union_off + (int)uni;
