@@ -120,7 +120,7 @@ struct WsPlan {
   size_t len, pending, status, counters, row_ids, accept_flags;
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
-  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, xq, ssq_a, ssq_b, tile_cnt;
+  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, xq, ssq_a, ssq_b;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -162,9 +162,8 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.xo = take(qd * 64);
   p.xq = take(qd * 64);
   p.xd = take(F * 64);
-  p.ssq_a = take((d / 8 + 1) * FAST_MAX_T * 4);
-  p.ssq_b = take((d / 8 + 1) * FAST_MAX_T * 4);
-  p.tile_cnt = take((d / 8 + 1) * 4);
+  p.ssq_a = take((d / 64 + 1) * FAST_MAX_T * 8);
+  p.ssq_b = take((d / 64 + 1) * FAST_MAX_T * 8);
   p.fpart = take((size_t)FAST_MAX_T * c.n_q_heads * FAST_NSPLIT_CAP * (c.head_dim + 2) * 4);
   p.attn_counters = take((size_t)FAST_MAX_T * c.n_q_heads * 4);
   p.flags = take(64);
@@ -243,7 +242,6 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.xd = s->xd;
   p.ssq_a = s->ssq_a;
   p.ssq_b = s->ssq_b;
-  p.tile_cnt = s->tile_cnt;
   p.part = s->fpart;
   p.logits = logits_out;
   p.attn_counters = s->attn_counters;
@@ -491,9 +489,8 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->xo = (uint32_t*)(W + p.xo);
   s->xq = (uint32_t*)(W + p.xq);
   s->xd = (uint32_t*)(W + p.xd);
-  s->ssq_a = (float*)(W + p.ssq_a);
-  s->ssq_b = (float*)(W + p.ssq_b);
-  s->tile_cnt = (int32_t*)(W + p.tile_cnt);
+  s->ssq_a = (long long*)(W + p.ssq_a);
+  s->ssq_b = (long long*)(W + p.ssq_b);
   s->fpart = (float*)(W + p.fpart);
   s->attn_counters = (int32_t*)(W + p.attn_counters);
   s->flags = (uint32_t*)(W + p.flags);

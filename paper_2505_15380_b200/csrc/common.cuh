@@ -114,8 +114,7 @@ struct ssd_streams {
   // grid-barrier words
   long long* hfix;
   uint32_t *xa, *xb, *xo, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
-  float *ssq_a, *ssq_b;
-  int32_t* tile_cnt;
+  long long *ssq_a, *ssq_b;
   float* fpart;
   int32_t* attn_counters;
   uint32_t *flags, *epoch_base;

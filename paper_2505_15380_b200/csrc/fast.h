@@ -34,7 +34,7 @@ constexpr int FAST_MAX_SLOTS = 8;     // most ring slots per warp (barrier stora
 #define SSD_FAST_RING_SLOTS 3
 #endif
 constexpr int FAST_RING_SLOTS = SSD_FAST_RING_SLOTS;  // ring slots per warp actually used
-constexpr int FAST_MAXU = 8;          // output tiles a CTA accumulates at once (one "round")
+constexpr int FAST_MAXU = 10;         // output tiles a CTA accumulates at once (one "round")
 constexpr int FAST_MAX_UNITS = 64;    // output tiles per CTA and op (table size in shared memory)
 constexpr int FAST_MAX_CHUNKS = 128;  // chunks per warp: one layer's plus the LM head's
 constexpr int FAST_MAX_T = 16;        // rows per forward
@@ -134,15 +134,14 @@ struct FastParams {
   const int32_t* row_ids;       // explicit ids [nb * R], or null: row 0 = pending, rows 1.. = draft
   const int32_t* draft_tokens;  // [B, gamma] when row_ids is null
   // workspace
-  long long* hfix;  // residual stream [T][d] in 2^-32 fixed point (order-independent accumulation)
+  long long* hfix;  // residual stream [T][d]: 2^-32 fixed point above a 4-bit arrival count
   float *rope_cs, *part, *logits;  // logits null: skip the LM head
   // Inputs of the projections, written by their producers already in the tensor-core operand layout
   // (bf16 leading part + remainder, see fast_verify.cu): the RMS-norm inputs x * gain of the QKV /
   // LM-head projection (xa) and of gate/up (xb), the attention output (xo), SiLU(g) * u (xd); and
-  // per 8-column tile and row the sums of squares that go with xa / xb.
+  // per 64 columns and row the sums of squares that go with xa / xb.
   uint32_t *xa, *xb, *xo, *xd, *xq;  // xq: the rotated, scaled queries
-  float *ssq_a, *ssq_b;   // [d / 8][FAST_MAX_T]
-  int32_t* tile_cnt;      // [d / 8] arrivals of the down projection's K slices per output tile
+  long long *ssq_a, *ssq_b;  // [ceil(d / 64)][FAST_MAX_T], 2^-32 fixed point
   int32_t* attn_counters;
   uint32_t* flags;       // [0] grid-barrier arrival counter, monotonic across launches
   uint32_t* epoch_base;  // [0] counter value at the start of the next launch, [1] nonzero after a failure

@@ -225,7 +225,7 @@ __device__ __noinline__ bool grid_sync(const FastParams& P, uint32_t target, boo
 // One projection of the layer: which weights, which input, which epilogue.
 struct PhaseDesc {
   const uint32_t* xin;  // operand-layout input, at this CTA's first k-step
-  const float* ssq_in;  // with in_fix: the per-tile sums of squares of the input rows
+  const long long* ssq_in;  // with in_fix: the sums of squares of the input rows
   int op;               // FOP_*: whose tiles of this CTA
   int epi;              // EPI_F_*
   int in_fix;           // the input is x * gain of an RMS norm: scale the outputs by inv_rms[row]
@@ -236,9 +236,9 @@ struct PhaseDesc {
   float qscale;         // 1 / sqrt(head_dim)
   // residual epilogues: the operand the finished rows become for the next projection
   uint32_t* xout;
-  float* ssq_out;
+  long long* ssq_out;
   const float* gain_next;
-  int nsplit;           // K slices (CTAs) adding into the same output tile (1: a single writer)
+  int cinc;             // this CTA's increment of an element's arrival count (see resid_tile)
 };
 
 // Operand layout of the activations (the A operand of the projections), in global memory where a
@@ -273,40 +273,35 @@ __device__ __forceinline__ void write_frag_elem(uint32_t* buf, int row, int k, f
   w[4] = l;  // two words on
 }
 
-// inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the per-tile sums of squares a producer left; one
-// warp per row, fixed summation order.  The loads are issued at the start of the phase and
-// summed after the tensor-core work, so their latency stays off the critical path.
-constexpr int SSQ_REGS = 4;  // covers d <= 1024 in one go
+// inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the sums of squares the producers left, one 64-bit
+// fixed-point word (2^-32) per 64 columns and row; one warp per row.  The loads are issued at the
+// start of the phase and summed after the tensor-core work, so their latency stays off the
+// critical path.
+constexpr int SSQ_COLS = 64;  // columns per word
 struct SsqLoads {
-  float v[2][SSQ_REGS];  // rows warp and warp + FAST_WARPS
+  long long v[2];  // rows warp and warp + FAST_WARPS: word `lane`
 };
-__device__ __forceinline__ void ssq_issue(SsqLoads& q, const float* __restrict__ ssq, int ntiles, int T) {
+__device__ __forceinline__ void ssq_issue(SsqLoads& q, const long long* __restrict__ ssq, int nwords, int T) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const int row = warp + h * FAST_WARPS;
-    if (row < T) {  // uniform per warp
-#pragma unroll
-      for (int i = 0; i < SSQ_REGS; ++i) {
-        const int tile = lane + 32 * i;
-        q.v[h][i] = tile < ntiles ? __ldcg(ssq + tile * FAST_MAX_T + row) : 0.f;
-      }
-    }
+    q.v[h] = 0;
+    if (row < T && lane < nwords) q.v[h] = __ldcg(ssq + lane * FAST_MAX_T + row);
   }
 }
-__device__ __forceinline__ void ssq_finish(const SsqLoads& q, const float* __restrict__ ssq, int ntiles, int T,
+__device__ __forceinline__ void ssq_finish(const SsqLoads& q, const long long* __restrict__ ssq, int nwords, int T,
                                            int K, float eps, FastMisc& M) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const int row = warp + h * FAST_WARPS;
     if (row < T) {  // uniform per warp
-      float v = 0.f;
+      long long v = q.v[h];
+      for (int wd = lane + 32; wd < nwords; wd += 32) v += __ldcg(ssq + wd * FAST_MAX_T + row);
 #pragma unroll
-      for (int i = 0; i < SSQ_REGS; ++i) v += q.v[h][i];
-      for (int tile = lane + 32 * SSQ_REGS; tile < ntiles; tile += 32) v += __ldcg(ssq + tile * FAST_MAX_T + row);
-      v = warp_sum(v);
-      if (lane == 0) M.inv_rms[row] = rsqrtf(v / (float)K + eps);
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);  // integer: any order
+      if (lane == 0) M.inv_rms[row] = rsqrtf(fix_to_float(v) / (float)K + eps);
     }
   }
 }
@@ -349,77 +344,53 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
   }
 }
 
-// Residual epilogue of one output tile (8 columns of h), collective over a warp: lane = (row g,
-// column pair t) adds its projection outputs to the fixed-point residual stream.  64-bit integer
-// adds commute, so the K slices of different CTAs may arrive in any order and the sum is still
-// bit-reproducible.  The warp that completes the tile (the only writer, or the last of the slices
-// to arrive) turns the finished rows into the operand of the next projection: x * gain as bf16
-// hi / lo in operand layout, plus the tile's sums of squares for the RMS norm.
+// Residual epilogue of one output tile (8 columns of h), per lane = (row g, column pair t): the
+// projection outputs are added to the residual stream with 64-bit integer atomics.  A word holds
+// the value in 2^-32 fixed point above a 4-bit arrival count: integer adds commute, so the K
+// slices of different CTAs may arrive in any order and the sum is still bit-reproducible, and the
+// count tells the thread whose add completes an element that it holds the finished value (the
+// slices' count increments are +1, and 1 - nsplit for slice 0: they sum to zero, and no partial
+// sum is a multiple of 16).  That thread turns the element into the operand of the next
+// projection (x * gain as bf16 hi / lo in operand layout) and adds x^2 to the row's sums of
+// squares for the RMS norm, in fixed point as well.
 template <bool T16>
 __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
                                            const float* c) {
-  constexpr int NACC = T16 ? 4 : 2;
+  constexpr int NH = T16 ? 2 : 1;
   const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
-  const bool v0 = gg < T, v1 = T16 && gg + 8 < T;
-  long long* h0 = P.hfix + (size_t)gg * P.d + n;
-  long long* h1 = h0 + (size_t)8 * P.d;
-  longlong2 a = make_longlong2(0, 0), b = make_longlong2(0, 0);
   const float2 gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
-  if (D.nsplit > 1) {
-    if (v0) {
-      atomicAdd(reinterpret_cast<unsigned long long*>(h0), (unsigned long long)__float2ll_rn(c[0] * FIX_SCALE));
-      atomicAdd(reinterpret_cast<unsigned long long*>(h0) + 1, (unsigned long long)__float2ll_rn(c[1] * FIX_SCALE));
-    }
-    if (v1) {
-      atomicAdd(reinterpret_cast<unsigned long long*>(h1), (unsigned long long)__float2ll_rn(c[NACC - 2] * FIX_SCALE));
-      atomicAdd(reinterpret_cast<unsigned long long*>(h1) + 1, (unsigned long long)__float2ll_rn(c[NACC - 1] * FIX_SCALE));
-    }
-    __syncwarp();
-    int last = 0;
-    if (lane == 0) {
-      __threadfence();
-      last = atomicAdd(&P.tile_cnt[tile], 1) == D.nsplit - 1;
-      if (last) P.tile_cnt[tile] = 0;
-    }
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (!last) return;
-    __threadfence();
-    if (v0) a = __ldcg(reinterpret_cast<const longlong2*>(h0));
-    if (v1) b = __ldcg(reinterpret_cast<const longlong2*>(h1));
-  } else {
-    if (v0) {
-      a = __ldcg(reinterpret_cast<const longlong2*>(h0));
-      a.x += __float2ll_rn(c[0] * FIX_SCALE);
-      a.y += __float2ll_rn(c[1] * FIX_SCALE);
-      *reinterpret_cast<longlong2*>(h0) = a;
-    }
-    if (v1) {
-      b = __ldcg(reinterpret_cast<const longlong2*>(h1));
-      b.x += __float2ll_rn(c[NACC - 2] * FIX_SCALE);
-      b.y += __float2ll_rn(c[NACC - 1] * FIX_SCALE);
-      *reinterpret_cast<longlong2*>(h1) = b;
+  long long inc[NH][2], old[NH][2];
+#pragma unroll
+  for (int h = 0; h < NH; ++h) {
+    if (gg + 8 * h < T) {
+      unsigned long long* hp = reinterpret_cast<unsigned long long*>(P.hfix + (size_t)(gg + 8 * h) * P.d + n);
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        inc[h][j] = __float2ll_rn(c[2 * h + j] * FIX_SCALE) * 16 + D.cinc;
+        old[h][j] = (long long)atomicAdd(hp + j, (unsigned long long)inc[h][j]);
+      }
     }
   }
-  float s0 = 0.f, s1 = 0.f;
-  if (v0) {
-    const float x0 = fix_to_float(a.x), x1 = fix_to_float(a.y);
-    s0 = fmaf(x0, x0, x1 * x1);
-    write_frag_pair<T16>(D.xout, gg, n, x0 * gn.x, x1 * gn.y);
-  }
-  if (v1) {
-    const float x0 = fix_to_float(b.x), x1 = fix_to_float(b.y);
-    s1 = fmaf(x0, x0, x1 * x1);
-    write_frag_pair<T16>(D.xout, gg + 8, n, x0 * gn.x, x1 * gn.y);
-  }
-  s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
-  s0 += __shfl_xor_sync(0xffffffffu, s0, 2);
-  if (T16) {
-    s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
-    s1 += __shfl_xor_sync(0xffffffffu, s1, 2);
-  }
-  if (tt == 0) {
-    if (v0) D.ssq_out[tile * FAST_MAX_T + gg] = s0;
-    if (v1) D.ssq_out[tile * FAST_MAX_T + gg + 8] = s1;
+#pragma unroll
+  for (int h = 0; h < NH; ++h) {
+    const int row = gg + 8 * h;
+    if (row < T) {
+      long long sq = 0;
+      bool any = false;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const long long now = old[h][j] + inc[h][j];
+        if ((now & 15) == 0) {  // this add completed the element
+          const float x = fix_to_float(now >> 4);
+          write_frag_elem<T16>(D.xout, row, n + j, x * (j ? gn.y : gn.x));
+          sq += __float2ll_rn(x * x * FIX_SCALE);
+          any = true;
+        }
+      }
+      if (any)
+        atomicAdd(reinterpret_cast<unsigned long long*>(D.ssq_out + (n / SSQ_COLS) * FAST_MAX_T + row),
+                  (unsigned long long)sq);
+    }
   }
 }
 
@@ -495,7 +466,7 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
   const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
   SsqLoads ssq;
-  if (D.in_fix) ssq_issue(ssq, D.ssq_in, P.d >> 3, T);
+  if (D.in_fix) ssq_issue(ssq, D.ssq_in, (P.d + SSQ_COLS - 1) / SSQ_COLS, T);
   const bool row0 = g < T, row1 = T16 && g + 8 < T;
   // this warp's k-steps of the operand: one bulk copy from L2 (the producers' stores were made
   // visible by the grid barrier; the proxy fence orders that observation before the async read)
@@ -524,9 +495,11 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
       case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
       case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
       case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      default: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 8: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 9: mma_round<9, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      default: mma_round<10, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
     }
-    if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, P.d >> 3, T, D.kc, P.eps, M);
+    if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, (P.d + SSQ_COLS - 1) / SSQ_COLS, T, D.kc, P.eps, M);
     __syncthreads();
     for (int idx = tid; idx < cnt * 32; idx += FAST_THREADS) {  // whole warps: one tile per warp pass
       const int u = idx >> 5, l = idx & 31, gg = l >> 2, tt = l & 3;
@@ -918,20 +891,20 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     }
     const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(P.embed + (size_t)id * d);
     const float2* g0 = reinterpret_cast<const float2*>(P.m.gains);  // first layer's input norm
-    for (int kk0 = 0; kk0 < (d >> 1); kk0 += FAST_THREADS) {         // column pairs; whole warps
+    for (int kk0 = 0; kk0 < (d >> 1); kk0 += FAST_THREADS) {         // column pairs; a warp = 64 columns
       const int kk = kk0 + tid;
-      float ss = 0.f;
+      long long ss = 0;
       if (kk < (d >> 1)) {
         const float2 x = __bfloat1622float2(src[kk]);
         const float2 gn = __ldg(g0 + kk);
         *reinterpret_cast<longlong2*>(P.hfix + (size_t)tok * d + 2 * kk) =
-            make_longlong2(__float2ll_rn(x.x * FIX_SCALE), __float2ll_rn(x.y * FIX_SCALE));
+            make_longlong2(__float2ll_rn(x.x * FIX_SCALE) * 16, __float2ll_rn(x.y * FIX_SCALE) * 16);
         write_frag_pair<T16>(P.xa, tok, 2 * kk, x.x * gn.x, x.y * gn.y);
-        ss = fmaf(x.x, x.x, x.y * x.y);
+        ss = __float2ll_rn(x.x * x.x * FIX_SCALE) + __float2ll_rn(x.y * x.y * FIX_SCALE);
       }
-      ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-      ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-      if (kk < (d >> 1) && (kk & 3) == 0) P.ssq_a[(kk >> 2) * FAST_MAX_T + tok] = ss;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (lane == 0 && kk < (d >> 1)) P.ssq_a[(kk >> 5) * FAST_MAX_T + tok] = ss;
     }
     const double pos = (double)M.tok_pos[tok];
     for (int j = tid; j < half; j += FAST_THREADS) {
@@ -970,6 +943,12 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       for (int i = tid; i < ((3 * d * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(gq + (size_t)i * 128);
     }
     if (ph == 1) {
+      if (cta == P.m.n_cta - 1) {
+        // both sets of sums of squares are idle during this phase (the O projection adds to one
+        // after the next barrier, the down projection to the other two barriers on): clear them
+        const int nw = (d + SSQ_COLS - 1) / SSQ_COLS * FAST_MAX_T;
+        for (int i = tid; i < nw; i += FAST_THREADS) P.ssq_a[i] = P.ssq_b[i] = 0;
+      }
       if (P.hd == 64) attn_phase<64, T16>(P, M, uni, l);
       else if (P.hd == 128) attn_phase<128, T16>(P, M, uni, l);
       else attn_phase<32, T16>(P, M, uni, l);
@@ -982,7 +961,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       D.xout = nullptr;
       D.ssq_out = nullptr;
       D.gain_next = nullptr;
-      D.nsplit = 1;
+      D.cinc = 0;
       if (ph == 0) {
         D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
         D.kc = d; D.n_rows = qd + 2 * P.Hkv * P.hd;
@@ -995,7 +974,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       } else if (ph == 4) {
         D.op = FOP_DOWN; D.epi = EPI_F_RESID; D.in_fix = 0;
         D.xin = P.xd + (size_t)(dk0 >> 4) * (T16 ? 256 : 128); D.kc = dk1 - dk0; D.n_rows = d;
-        D.xout = P.xa; D.ssq_out = P.ssq_a; D.nsplit = P.m.down_split;
+        D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = dsl == 0 ? 1 - P.m.down_split : 1;
         D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
       } else {
         D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
