@@ -120,7 +120,7 @@ struct WsPlan {
   size_t len, pending, status, counters, row_ids, accept_flags;
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
-  size_t hfix, fpart, attn_counters, flags, epoch_base, xa, xb, xo, xd, xq, ssq_a, ssq_b;
+  size_t hfix, flags, epoch_base, xa, xb, xd, xq, ssq_a, ssq_b;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -159,13 +159,10 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   // operand-layout activations: per 16 columns 32 lanes x 32 bytes (16 rows, bf16 hi + lo)
   p.xa = take(d * 64);
   p.xb = take(d * 64);
-  p.xo = take(qd * 64);
   p.xq = take(qd * 64);
   p.xd = take(F * 64);
   p.ssq_a = take((d / 64 + 1) * FAST_MAX_T * 8);
   p.ssq_b = take((d / 64 + 1) * FAST_MAX_T * 8);
-  p.fpart = take((size_t)FAST_MAX_T * c.n_q_heads * FAST_NSPLIT_CAP * (c.head_dim + 2) * 4);
-  p.attn_counters = take((size_t)FAST_MAX_T * c.n_q_heads * 4);
   p.flags = take(64);
   p.epoch_base = take(2 * 4);
   p.total = off;
@@ -208,6 +205,7 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.m.n_cta = f.n_cta;
   p.m.max_units = f.max_units;
   p.m.down_split = f.down_split;
+  p.m.o_split = f.o_split;
   p.m.max_stage_k = f.max_stage_k;
   p.embed = (const bf16*)m->embed;
   p.inv_freq = m->inv_freq;
@@ -237,14 +235,11 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.rope_cs = s->rope_cs;
   p.xa = s->xa;
   p.xb = s->xb;
-  p.xo = s->xo;
   p.xq = s->xq;
   p.xd = s->xd;
   p.ssq_a = s->ssq_a;
   p.ssq_b = s->ssq_b;
-  p.part = s->fpart;
   p.logits = logits_out;
-  p.attn_counters = s->attn_counters;
   p.flags = s->flags;
   p.epoch_base = s->epoch_base;
   p.trace = s->trace;
@@ -401,6 +396,7 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
     f.gains = (const float*)(A + p.f_gains);
     f.n_cta = fplan.n_cta;
     f.down_split = fplan.ops[FOP_DOWN].ksplit;
+    f.o_split = fplan.ops[FOP_O].ksplit;
     f.max_units = 0;
     for (int32_t v : fplan.unit_cnt) f.max_units = v > f.max_units ? v : f.max_units;
     int down_w = 0;
@@ -486,13 +482,10 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->hfix = (long long*)(W + p.hfix);
   s->xa = (uint32_t*)(W + p.xa);
   s->xb = (uint32_t*)(W + p.xb);
-  s->xo = (uint32_t*)(W + p.xo);
   s->xq = (uint32_t*)(W + p.xq);
   s->xd = (uint32_t*)(W + p.xd);
   s->ssq_a = (long long*)(W + p.ssq_a);
   s->ssq_b = (long long*)(W + p.ssq_b);
-  s->fpart = (float*)(W + p.fpart);
-  s->attn_counters = (int32_t*)(W + p.attn_counters);
   s->flags = (uint32_t*)(W + p.flags);
   s->epoch_base = (uint32_t*)(W + p.epoch_base);
   s->path = 0;

@@ -82,7 +82,7 @@ struct ssd_fast_model {
   const uint8_t* chunks = nullptr;
   const int32_t *chunk_cnt = nullptr, *unit_cnt = nullptr, *unit_off = nullptr, *unit_tile = nullptr;
   const float *bias_qkv = nullptr, *gains = nullptr;
-  int n_cta = 0, max_units = 0, down_split = 1, max_stage_k = 0;
+  int n_cta = 0, max_units = 0, down_split = 1, o_split = 1, max_stage_k = 0;
 };
 
 struct ssd_model {
@@ -113,10 +113,8 @@ struct ssd_streams {
   // persistent small-batch kernel: fixed-point residual stream, attention partials and counters,
   // grid-barrier words
   long long* hfix;
-  uint32_t *xa, *xb, *xo, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
+  uint32_t *xa, *xb, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
   long long *ssq_a, *ssq_b;
-  float* fpart;
-  int32_t* attn_counters;
   uint32_t *flags, *epoch_base;
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)

@@ -38,7 +38,6 @@ constexpr int FAST_MAXU = 10;         // output tiles a CTA accumulates at once 
 constexpr int FAST_MAX_UNITS = 64;    // output tiles per CTA and op (table size in shared memory)
 constexpr int FAST_MAX_CHUNKS = 128;  // chunks per warp: one layer's plus the LM head's
 constexpr int FAST_MAX_T = 16;        // rows per forward
-constexpr int FAST_NSPLIT_CAP = 16;   // most key splits per (stream, head) in the attention phase
 constexpr int FAST_MAX_CTAS = 256;
 
 enum FastOpId { FOP_QKV = 0, FOP_O = 1, FOP_GU = 2, FOP_DOWN = 3, FOP_HEAD = 4, FOP_COUNT = 5 };
@@ -49,6 +48,8 @@ struct FastOpShape {
   int n_tiles;  // ceil(n_rows / 8)
   int ksteps;   // K / 16
   int ksplit;   // CTA c works on K slice c % ksplit (1: every CTA covers all of K)
+  int by_tile;  // 0: the warps of a CTA split the K slice; 1: they split the CTA's tiles (tile u goes
+                // to warp u % FAST_WARPS, which covers the whole K slice)
 };
 
 // K slice (in steps of 16 columns) of an op that CTA `cta` works on.
@@ -69,6 +70,11 @@ __host__ __device__ inline int fast_warp_k1(int w, int ksteps) {
 // k-steps per chunk for a round of `cnt` tiles (a chunk never holds more than FAST_SLOT_TILES).
 __host__ __device__ inline int fast_steps_per_chunk(int cnt) { return FAST_SLOT_TILES / cnt; }
 
+// Tiles of a CTA's `cnt` that warp w owns when the warps split the tiles.
+__host__ __device__ inline int fast_warp_tiles(int w, int cnt) {
+  return cnt > w ? (cnt - w + FAST_WARPS - 1) / FAST_WARPS : 0;
+}
+
 // Which output tiles each CTA owns for each op, and where each warp's byte stream lives.
 struct FastPlan {
   int n_cta = 0;
@@ -87,6 +93,9 @@ struct FastPlan {
 
 bool fast_supported(const ssd_model_config& c);
 int fast_down_split(const ssd_model_config& c);
+// K slices of the O projection = groups of query heads; a slice's CTAs compute the attention of
+// its heads themselves, so the O projection needs no exchange after the attention.
+int fast_o_split(const ssd_model_config& c, int n_cta);
 FastPlan fast_make_plan(const ssd_model_config& c, int n_cta);
 // Packs the bf16 weights of the flat host blob (layout of ssd_model_create) into the per-warp
 // streams described by `plan` (out has plan.total_bytes bytes).
@@ -113,6 +122,7 @@ struct FastModelDev {
   int n_cta;
   int max_units;    // most tiles any CTA owns for one op
   int down_split;   // K slices of the down projection
+  int o_split;      // K slices (groups of query heads) of the O projection
   int max_stage_k;  // widest input slice a CTA stages in shared memory
 };
 
@@ -135,14 +145,13 @@ struct FastParams {
   const int32_t* draft_tokens;  // [B, gamma] when row_ids is null
   // workspace
   long long* hfix;  // residual stream [T][d]: 2^-32 fixed point above a 4-bit arrival count
-  float *rope_cs, *part, *logits;  // logits null: skip the LM head
+  float *rope_cs, *logits;  // logits null: skip the LM head
   // Inputs of the projections, written by their producers already in the tensor-core operand layout
   // (bf16 leading part + remainder, see fast_verify.cu): the RMS-norm inputs x * gain of the QKV /
-  // LM-head projection (xa) and of gate/up (xb), the attention output (xo), SiLU(g) * u (xd); and
+  // LM-head projection (xa) and of gate/up (xb), SiLU(g) * u (xd); and
   // per 64 columns and row the sums of squares that go with xa / xb.
-  uint32_t *xa, *xb, *xo, *xd, *xq;  // xq: the rotated, scaled queries
+  uint32_t *xa, *xb, *xd, *xq;  // xq: the rotated, scaled queries
   long long *ssq_a, *ssq_b;  // [ceil(d / 64)][FAST_MAX_T], 2^-32 fixed point
-  int32_t* attn_counters;
   uint32_t* flags;       // [0] grid-barrier arrival counter, monotonic across launches
   uint32_t* epoch_base;  // [0] counter value at the start of the next launch, [1] nonzero after a failure
   // optional trace: thread 0 of CTA c stores clock64() at trace[c * trace_cap + i] for its i-th
@@ -151,10 +160,9 @@ struct FastParams {
   int trace_cap;
   // shared-memory carve-up (bytes)
   int nslot, ring_warp_bytes, union_off, misc_off;
-  int keys_min;  // fewest keys worth an attention split of their own
 };
 
-size_t fast_union_bytes(int stage_k, int head_dim, int T, int R);
+size_t fast_union_bytes(int stage_k, int head_dim, int T, int o_steps);
 cudaError_t launch_fast_forward(const FastParams& p, cudaStream_t st);
 
 }  // namespace ssd

@@ -13,7 +13,10 @@
 //
 // Order of a warp's stream: layers; ops (QKV, O, gate/up, down); rounds of FAST_MAXU of the CTA's
 // tiles; the warp's k-steps; the round's tiles.  The stream is cut into chunks of whole k-steps of
-// at most FAST_SLOT_TILES tiles: one chunk is one bulk copy into one ring slot.
+// at most FAST_SLOT_TILES tiles: one chunk is one bulk copy into one ring slot.  The O projection
+// is the exception: its K is split by groups of query heads over the CTAs, the warps of a CTA split
+// its tiles (warp w: tiles w, w + FAST_WARPS, ..), each tile with all k-steps of the slice in
+// order, and the chunks are simply runs of FAST_SLOT_TILES tiles of that sequence.
 #include <string.h>
 
 #include <algorithm>
@@ -111,6 +114,13 @@ bool fast_supported(const ssd_model_config& c) {
   return true;
 }
 
+int fast_o_split(const ssd_model_config& c, int n_cta) {
+  int s = 1;
+  for (int v = 1; v <= c.n_q_heads && v <= n_cta; ++v)
+    if (c.n_q_heads % v == 0) s = v;
+  return s;
+}
+
 int fast_down_split(const ssd_model_config& c) {
   // slices of at most 1280 input columns: a CTA stages its slice of the activations in shared memory
   int s = 1;
@@ -123,9 +133,10 @@ FastPlan fast_make_plan(const ssd_model_config& c, int n_cta) {
   p.n_cta = n_cta;
   p.n_layers = c.n_layers;
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn;
-  auto shape = [](int rows, int K, int split) { return FastOpShape{rows, K, (rows + 7) / 8, K / 16, split}; };
+  auto shape = [](int rows, int K, int split) { return FastOpShape{rows, K, (rows + 7) / 8, K / 16, split, 0}; };
   p.ops[FOP_QKV] = shape(qd + 2 * kvd, d, 1);
-  p.ops[FOP_O] = shape(d, qd, 1);
+  p.ops[FOP_O] = shape(d, qd, fast_o_split(c, n_cta));
+  p.ops[FOP_O].by_tile = 1;
   p.ops[FOP_GU] = shape(2 * F, d, 1);
   p.ops[FOP_DOWN] = shape(d, F, std::min(fast_down_split(c), n_cta));
   p.ops[FOP_HEAD] = shape(c.vocab_out, d, 1);
@@ -177,6 +188,12 @@ FastPlan fast_make_plan(const ssd_model_config& c, int n_cta) {
         const int ns = fast_warp_k1(w, slice_steps) - fast_warp_k0(w, slice_steps);
         const int cnt_total = (int)own[cta][op].size();
         std::vector<uint8_t>& ch = op == FOP_HEAD ? ch_head : ch_layer;
+        if (p.ops[op].by_tile) {
+          const int nt = fast_warp_tiles(w, cnt_total) * slice_steps;
+          for (int t0 = 0; t0 < nt; t0 += FAST_SLOT_TILES) ch.push_back((uint8_t)std::min(FAST_SLOT_TILES, nt - t0));
+          tiles_layer += (uint64_t)nt;
+          continue;
+        }
         for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
           const int cnt = std::min(FAST_MAXU, cnt_total - u0), spc = fast_steps_per_chunk(cnt);
           for (int s = 0; s < ns; s += spc) ch.push_back((uint8_t)(std::min(spc, ns - s) * cnt));
@@ -198,6 +215,41 @@ FastPlan fast_make_plan(const ssd_model_config& c, int n_cta) {
   return p;
 }
 
+namespace {
+
+// One operand tile (8 packed rows from row0, k-step ks) to / from 256 bytes of a stream.
+void emit_tile(const ssd_model_config& c, const BlobView& v, const uint16_t* blob, int op, int l, int row0,
+               int ks, uint32_t* dst) {
+  for (int g = 0; g < 8; ++g) {
+    const uint16_t* row = packed_row(c, v, blob, op, l, row0 + g);
+    for (int t = 0; t < 4; ++t) {
+      uint32_t lo = 0, hi = 0;
+      if (row) {
+        const uint16_t* a = row + (size_t)ks * 16 + 2 * t;
+        lo = (uint32_t)a[0] | ((uint32_t)a[1] << 16);
+        hi = (uint32_t)a[8] | ((uint32_t)a[9] << 16);
+      }
+      dst[(g * 4 + t) * 2 + 0] = lo;
+      dst[(g * 4 + t) * 2 + 1] = hi;
+    }
+  }
+}
+void scatter_tile(const ssd_model_config& c, const BlobView& v, uint16_t* blob_out, int op, int l, int row0,
+                  int ks, const uint32_t* src) {
+  for (int g = 0; g < 8; ++g) {
+    uint16_t* row = const_cast<uint16_t*>(packed_row(c, v, blob_out, op, l, row0 + g));
+    if (!row) continue;
+    for (int t = 0; t < 4; ++t) {
+      const uint32_t lo = src[(g * 4 + t) * 2], hi = src[(g * 4 + t) * 2 + 1];
+      uint16_t* a = row + (size_t)ks * 16 + 2 * t;
+      a[0] = (uint16_t)lo; a[1] = (uint16_t)(lo >> 16);
+      a[8] = (uint16_t)hi; a[9] = (uint16_t)(hi >> 16);
+    }
+  }
+}
+
+}  // namespace
+
 void fast_pack_streams(const ssd_model_config& c, const FastPlan& plan, const uint16_t* blob,
                        uint8_t* out) {
   const BlobView v = view_blob(c);
@@ -206,29 +258,25 @@ void fast_pack_streams(const ssd_model_config& c, const FastPlan& plan, const ui
       uint32_t* dst = reinterpret_cast<uint32_t*>(out + plan.stream_off[(size_t)cta * FAST_WARPS + w]);
       for (int l = 0; l <= c.n_layers; ++l) {
         const int op_begin = l < c.n_layers ? 0 : FOP_HEAD, op_end = l < c.n_layers ? FOP_HEAD : FOP_COUNT;
+        const int ll = l < c.n_layers ? l : 0;
         for (int op = op_begin; op < op_end; ++op) {
           const FastOpShape& s = plan.ops[op];
           const int cnt = plan.unit_cnt[(size_t)cta * FOP_COUNT + op];
           const int32_t* tiles = plan.unit_tile.data() + plan.unit_off[(size_t)cta * FOP_COUNT + op];
           const int sk0 = fast_slice_k0(s, cta), slice_steps = fast_slice_k1(s, cta) - sk0;
+          if (s.by_tile) {
+            for (int u = w; u < cnt; u += FAST_WARPS)
+              for (int ks = sk0; ks < sk0 + slice_steps; ++ks) {
+                emit_tile(c, v, blob, op, ll, tiles[u] * 8, ks, dst);
+                dst += FAST_TILE_BYTES / 4;
+              }
+            continue;
+          }
           const int k0 = sk0 + fast_warp_k0(w, slice_steps), k1 = sk0 + fast_warp_k1(w, slice_steps);
           for (int u0 = 0; u0 < cnt; u0 += FAST_MAXU)
             for (int ks = k0; ks < k1; ++ks)
               for (int u = u0; u < std::min(cnt, u0 + FAST_MAXU); ++u) {
-                const int row0 = tiles[u] * 8;
-                for (int g = 0; g < 8; ++g) {
-                  const uint16_t* row = packed_row(c, v, blob, op, l < c.n_layers ? l : 0, row0 + g);
-                  for (int t = 0; t < 4; ++t) {
-                    uint32_t lo = 0, hi = 0;
-                    if (row) {
-                      const uint16_t* a = row + (size_t)ks * 16 + 2 * t;
-                      lo = (uint32_t)a[0] | ((uint32_t)a[1] << 16);
-                      hi = (uint32_t)a[8] | ((uint32_t)a[9] << 16);
-                    }
-                    dst[(g * 4 + t) * 2 + 0] = lo;
-                    dst[(g * 4 + t) * 2 + 1] = hi;
-                  }
-                }
+                emit_tile(c, v, blob, op, ll, tiles[u] * 8, ks, dst);
                 dst += FAST_TILE_BYTES / 4;
               }
         }
@@ -237,8 +285,9 @@ void fast_pack_streams(const ssd_model_config& c, const FastPlan& plan, const ui
 }
 
 // Inverse of fast_pack_streams, written as a consumer would walk the streams (chunk by chunk, a
-// chunk being whole k-steps of one round): scatters every tile back into a flat blob of the
-// ssd_model_create layout.  Returns the number of chunks whose size disagrees with the walk.
+// chunk being whole k-steps of one round, or a run of a warp's own tiles): scatters every tile
+// back into a flat blob of the ssd_model_create layout.  Returns the number of chunks whose size
+// disagrees with the walk.
 long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, const uint8_t* streams,
                               uint16_t* blob_out) {
   const BlobView v = view_blob(c);
@@ -252,11 +301,30 @@ long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, c
       for (int l = 0; l <= c.n_layers; ++l) {
         int ci = l < c.n_layers ? 0 : ncl;  // chunk cursor in the table
         const int op_begin = l < c.n_layers ? 0 : FOP_HEAD, op_end = l < c.n_layers ? FOP_HEAD : FOP_COUNT;
+        const int ll = l < c.n_layers ? l : 0;
         for (int op = op_begin; op < op_end; ++op) {
           const FastOpShape& s = plan.ops[op];
           const int cnt_total = plan.unit_cnt[(size_t)cta * FOP_COUNT + op];
           const int32_t* tiles = plan.unit_tile.data() + plan.unit_off[(size_t)cta * FOP_COUNT + op];
           const int sk0 = fast_slice_k0(s, cta), steps = fast_slice_k1(s, cta) - sk0;
+          if (s.by_tile) {
+            int left = fast_warp_tiles(w, cnt_total) * steps, in_chunk = 0, u = w, ks = 0;
+            while (left > 0) {
+              if (in_chunk == 0) {
+                in_chunk = std::min(FAST_SLOT_TILES, left);
+                if (tab[ci++] != in_chunk) ++bad;
+              }
+              scatter_tile(c, v, blob_out, op, ll, tiles[u] * 8, sk0 + ks, src);
+              src += FAST_TILE_BYTES / 4;
+              --in_chunk;
+              --left;
+              if (++ks == steps) {
+                ks = 0;
+                u += FAST_WARPS;
+              }
+            }
+            continue;
+          }
           const int s0 = sk0 + fast_warp_k0(w, steps), s1 = sk0 + fast_warp_k1(w, steps);
           for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
             const int cnt = std::min(FAST_MAXU, cnt_total - u0), spc = fast_steps_per_chunk(cnt);
@@ -265,17 +333,7 @@ long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, c
               if (tab[ci++] != nst * cnt) ++bad;
               for (int i = 0; i < nst; ++i)
                 for (int u = 0; u < cnt; ++u) {
-                  for (int g = 0; g < 8; ++g) {
-                    uint16_t* row = const_cast<uint16_t*>(
-                        packed_row(c, v, blob_out, op, l < c.n_layers ? l : 0, tiles[u0 + u] * 8 + g));
-                    for (int t = 0; t < 4; ++t) {
-                      const uint32_t lo = src[(g * 4 + t) * 2], hi = src[(g * 4 + t) * 2 + 1];
-                      if (!row) continue;
-                      uint16_t* a = row + (size_t)(sb + i) * 16 + 2 * t;
-                      a[0] = (uint16_t)lo; a[1] = (uint16_t)(lo >> 16);
-                      a[8] = (uint16_t)hi; a[9] = (uint16_t)(hi >> 16);
-                    }
-                  }
+                  scatter_tile(c, v, blob_out, op, ll, tiles[u0 + u] * 8, sb + i, src);
                   src += FAST_TILE_BYTES / 4;
                 }
             }

@@ -32,7 +32,6 @@ namespace ssd {
 namespace {
 
 constexpr unsigned long long FAST_WAIT_CYCLES = 3000000000ull;  // ~1.5 s at 2 GHz
-constexpr int FAST_KEYS_MIN = 384;                               // fewest keys worth a split of their own
 constexpr float FIX_SCALE = 4294967296.f;                        // residual stream: 2^-32 fixed point
 constexpr float FIX_INV_SCALE = 1.f / 4294967296.f;
 
@@ -112,9 +111,6 @@ struct FastMisc {
   float wred[FAST_WARPS][FAST_MAX_T];
   int32_t tok_stream[FAST_MAX_T];  // stream of each row of this forward
   int32_t tok_pos[FAST_MAX_T];     // its position len + r
-  int32_t attn_nsplit;             // key splits per (stream, head): the same in every layer
-  int32_t attn_item[6];            // this CTA's first work item: c, hq, bi, k0, k1, valid
-  int32_t last;
 };
 
 __device__ __forceinline__ void prefetch_l2(const void* p) {
@@ -354,23 +350,33 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
 // projection (x * gain as bf16 hi / lo in operand layout) and adds x^2 to the row's sums of
 // squares for the RMS norm, in fixed point as well.
 template <bool T16>
-__device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
-                                           const float* c) {
+struct ResidAdds {
+  long long inc[T16 ? 2 : 1][2], old[T16 ? 2 : 1][2];
+  float2 gn;
+};
+template <bool T16>
+__device__ __forceinline__ void resid_issue(const FastParams& P, const PhaseDesc& D, int tile, int lane,
+                                            const float* c, ResidAdds<T16>& A) {
   constexpr int NH = T16 ? 2 : 1;
   const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
-  const float2 gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
-  long long inc[NH][2], old[NH][2];
+  A.gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
 #pragma unroll
   for (int h = 0; h < NH; ++h) {
     if (gg + 8 * h < T) {
       unsigned long long* hp = reinterpret_cast<unsigned long long*>(P.hfix + (size_t)(gg + 8 * h) * P.d + n);
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
-        inc[h][j] = __float2ll_rn(c[2 * h + j] * FIX_SCALE) * 16 + D.cinc;
-        old[h][j] = (long long)atomicAdd(hp + j, (unsigned long long)inc[h][j]);
+        A.inc[h][j] = __float2ll_rn(c[2 * h + j] * FIX_SCALE) * 16 + D.cinc;
+        A.old[h][j] = (long long)atomicAdd(hp + j, (unsigned long long)A.inc[h][j]);
       }
     }
   }
+}
+template <bool T16>
+__device__ __forceinline__ void resid_finish(const FastParams& P, const PhaseDesc& D, int tile, int lane,
+                                             const ResidAdds<T16>& A) {
+  constexpr int NH = T16 ? 2 : 1;
+  const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
 #pragma unroll
   for (int h = 0; h < NH; ++h) {
     const int row = gg + 8 * h;
@@ -379,10 +385,10 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
       bool any = false;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
-        const long long now = old[h][j] + inc[h][j];
+        const long long now = A.old[h][j] + A.inc[h][j];
         if ((now & 15) == 0) {  // this add completed the element
           const float x = fix_to_float(now >> 4);
-          write_frag_elem<T16>(D.xout, row, n + j, x * (j ? gn.y : gn.x));
+          write_frag_elem<T16>(D.xout, row, n + j, x * (j ? A.gn.y : A.gn.x));
           sq += __float2ll_rn(x * x * FIX_SCALE);
           any = true;
         }
@@ -392,6 +398,13 @@ __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc&
                   (unsigned long long)sq);
     }
   }
+}
+template <bool T16>
+__device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
+                                           const float* c) {
+  ResidAdds<T16> A;
+  resid_issue<T16>(P, D, tile, lane, c, A);
+  resid_finish<T16>(P, D, tile, lane, A);
 }
 
 // The tensor-core work of one round of CNT tiles over this warp's k-steps [s0, s1): straight-line
@@ -542,19 +555,27 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   return v;
 }
 
-// Work item = (stream, query head, key split).  Every warp of the item's CTA works through its
-// own 16-key tiles from start to end (keys 16 w, 16 w + 128, ... of the split): it stages the
-// tile's keys / values (bf16, as cached) in its private part of shared memory, computes the scores
-// S[row, key] = q[row, :] . K[key, :] on the tensor cores (q arrives pre-split in operand layout
-// from the QKV epilogue), keeps a running max / sum per row in registers, and accumulates
-// O[row, :] += P[row, key] V[key, :] with P taken straight from the score registers (split into
-// bf16 hi + lo) and V read with a transposing matrix load.  One CTA barrier later the eight warps'
-// partials are combined.  Row r of a stream sees keys 0..len + r: causal inside the draft block.
-// The operand rows are the forward's rows (all streams); rows of other streams are masked out.
-// With more than one split the partials go to global memory and the CTA that arrives last for a
-// (stream, head) merges them in split order.
+// Attention and O projection, one phase.  The K of the O projection is split over the CTAs by
+// groups of query heads (the slices of FOP_O), so a CTA needs the attention output of its own
+// heads only: every CTA of a slice computes that attention itself (the same work in each of
+// them), keeps the result in shared memory as the A operand, multiplies it with its tiles of W_o
+// and adds the products to the residual stream.  No exchange between attention and projection.
+//
+// Attention of one (stream, head): every warp works through its own 16-key tiles from start to
+// end (keys 16 w, 16 w + 128, ..): it stages the tile's keys / values (bf16, as cached) in its
+// private part of shared memory, computes the scores S[row, key] = q[row, :] . K[key, :] on the
+// tensor cores (q arrives pre-split in operand layout from the QKV epilogue), keeps a running max /
+// sum per row in registers, and accumulates O[row, :] += P[row, key] V[key, :] with P taken
+// straight from the score registers (split into bf16 hi + lo) and V read with a transposing
+// matrix load.  One CTA barrier later the eight warps' partials are combined.  Row r of a stream
+// sees keys 0..len + r: causal inside the draft block.  The operand rows are the forward's rows
+// (all streams); rows of other streams are masked out.
+//
+// O projection: the warps split the CTA's tiles (tile u: warp u % 8), two tiles at a time so that
+// the residual adds of both are in flight together.
 template <int HD, bool T16>
-__device__ __forceinline__ void attn_phase(const FastParams& P, FastMisc& M, uint8_t* uni, int layer) {
+__device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
+                                             const PhaseDesc& D, int layer) {
   constexpr int ROWB = HD * 2 + 16;       // padded K / V row in bytes (conflict-free fragment loads)
   constexpr int NH = T16 ? 2 : 1;         // row halves: rows g and g + 8
   constexpr int W = T16 ? 8 : 4;          // words per (k-step, lane) of an operand
@@ -563,37 +584,32 @@ __device__ __forceinline__ void attn_phase(const FastParams& P, FastMisc& M, uin
   constexpr int CH = HD / 8;              // 16-byte chunks per row
   constexpr int LPL = 16 * CH / 32;       // 16-byte loads per lane for 16 rows
   constexpr int NROW = 8 * NH;            // rows held
-  const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv;
+  const int cnt = M.ucnt[FOP_O];
+  if (cnt == 0) return;
+  const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv, T = P.T;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int nsplit = M.attn_nsplit, items = nb * Hq * nsplit;
+  const int hps = Hq / P.m.o_split, slice = (int)blockIdx.x % P.m.o_split, KS = hps * KSTEPS;
 
   uint32_t* qsm = reinterpret_cast<uint32_t*>(uni);                       // q operand, KSTEPS steps
   uint8_t* kv_w = uni + KSTEPS * 32 * W * 4 + warp * (2 * 16 * ROWB);     // this warp's K then V tile
   float* cm = reinterpret_cast<float*>(uni + KSTEPS * 32 * W * 4 + FAST_WARPS * 2 * 16 * ROWB);  // [warp][NROW]
   float* cl = cm + FAST_WARPS * NROW;
   float* co = cl + FAST_WARPS * NROW;                                      // [warp][NROW][HD]
+  uint32_t* osm = reinterpret_cast<uint32_t*>(co + FAST_WARPS * NROW * HD);  // attention output, KS steps
   const uint32_t q_lane = smem_u32(qsm) + lane * (W * 4);
   const uint32_t k_lane = smem_u32(kv_w) + g * ROWB + t * 4;
   const uint32_t v_lane = smem_u32(kv_w) + 16 * ROWB + (lane & 15) * ROWB;
   const bf16* kvl = P.kv + (size_t)layer * P.kv_layer_elems;
 
-  for (int item = blockIdx.x; item < items; item += P.m.n_cta) {
-    int c, hq, bi, k0, k1;
-    if (item == (int)blockIdx.x) {  // the usual case: one item per CTA, worked out once per launch
-      c = M.attn_item[0]; hq = M.attn_item[1]; bi = M.attn_item[2]; k0 = M.attn_item[3]; k1 = M.attn_item[4];
-    } else {
-      c = item % nsplit; hq = (item / nsplit) % Hq; bi = item / (nsplit * Hq);
-      const int tot = min(M.tok_pos[bi * R] + R, P.cap);
-      const int per = (((tot + nsplit - 1) / nsplit) + 15) & ~15;
-      k0 = c * per; k1 = min(k0 + per, tot);
-    }
+  for (int item = 0; item < hps * nb; ++item) {
+    const int hl = item / nb, bi = item % nb, hq = slice * hps + hl;
     const int stream = P.b0 + bi, gk = hq / G, t_lo = bi * R, t_hi = t_lo + R;
-    const int L = M.tok_pos[t_lo];
+    const int L = M.tok_pos[t_lo], k1 = min(L + R, P.cap);
     const uint4* kg = reinterpret_cast<const uint4*>(kvl + (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * HD);
     const uint4* vg = reinterpret_cast<const uint4*>(kvl + (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD);
 
     // first tile of this warp: loads in flight before anything else
-    int key0 = k0 + 16 * warp;
+    int key0 = 16 * warp;
     uint4 kq[LPL], vq[LPL];
 #pragma unroll
     for (int i = 0; i < LPL; ++i) {
@@ -609,12 +625,12 @@ __device__ __forceinline__ void attn_phase(const FastParams& P, FastMisc& M, uin
       const uint4* src = reinterpret_cast<const uint4*>(P.xq + (size_t)hq * KSTEPS * 32 * W);
       for (int i = tid; i < KSTEPS * 32 * W / 4; i += FAST_THREADS) reinterpret_cast<uint4*>(qsm)[i] = __ldcg(src + i);
     }
-    if (layer + 1 < P.L) {
+    if (layer + 1 < P.L && (int)blockIdx.x < P.m.o_split && hq % G == 0) {
       // the same keys and values of the next layer (the cached prefix does not change during the
-      // forward): pull them into L2 now, one 128-byte line per thread and pass
-      const uint8_t* nk_ = reinterpret_cast<const uint8_t*>(kg) + P.kv_layer_elems * 2 + (size_t)k0 * HD * 2;
-      const uint8_t* nv_ = reinterpret_cast<const uint8_t*>(vg) + P.kv_layer_elems * 2 + (size_t)k0 * HD * 2;
-      const int lines = ((k1 - k0) * HD * 2 + 127) >> 7;
+      // forward): one CTA per KV head pulls them into L2 now, one 128-byte line per thread and pass
+      const uint8_t* nk_ = reinterpret_cast<const uint8_t*>(kg) + P.kv_layer_elems * 2;
+      const uint8_t* nv_ = reinterpret_cast<const uint8_t*>(vg) + P.kv_layer_elems * 2;
+      const int lines = (k1 * HD * 2 + 127) >> 7;
       for (int i = tid; i < lines; i += FAST_THREADS) {
         prefetch_l2(nk_ + (size_t)i * 128);
         prefetch_l2(nv_ + (size_t)i * 128);
@@ -748,56 +764,63 @@ __device__ __forceinline__ void attn_phase(const FastParams& P, FastMisc& M, uin
         o0 = fmaf(ov.x, e, o0);
         o1 = fmaf(ov.y, e, o1);
       }
-      if (nsplit == 1) {
-        const float il = 1.f / l;
-        write_frag_pair<T16>(P.xo, tok, hq * HD + dd, o0 * il, o1 * il);
-      } else {
-        float* dst = P.part + (((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP + c) * (HD + 2);
-        *reinterpret_cast<float2*>(dst + dd) = make_float2(o0, o1);
-        if (dd == 0) *reinterpret_cast<float2*>(dst + HD) = make_float2(m, l);
-      }
+      const float il = 1.f / l;
+      write_frag_pair<T16>(osm, tok, hl * HD + dd, o0 * il, o1 * il);
     }
-    if (nsplit > 1) {
-      __threadfence();
-      __syncthreads();
-      if (tid == 0) {
-        int prev = atomicAdd(&P.attn_counters[bi * Hq + hq], 1);
-        M.last = prev == nsplit - 1;
-        if (M.last) P.attn_counters[bi * Hq + hq] = 0;
-      }
-      __syncthreads();
-      if (M.last) {
-        __threadfence();
-        for (int idx = tid; idx < R * HD; idx += FAST_THREADS) {
-          const int r = idx / HD, dd = idx % HD, tok = t_lo + r;
-          const float* src = P.part + ((size_t)tok * Hq + hq) * FAST_NSPLIT_CAP * (HD + 2);
-          float m_tot = -CUDART_INF_F, denom = 0.f, ov = 0.f;
-          constexpr int MB = 8;  // splits loaded together
-          for (int sp0 = 0; sp0 < nsplit; sp0 += MB) {
-            float ms[MB], ls[MB], os[MB];
+  }
+  __syncthreads();
+
+  // O projection of this CTA's tiles over the slice's KS k-steps
+  const uint32_t o_lane = smem_u32(osm) + lane * (W * 4);
+  const bool row0 = g < T, row1 = T16 && g + 8 < T;
+  int left = fast_warp_tiles(warp, cnt) * KS, in_chunk = 0;
+  uint32_t wb = 0;
+  for (int u = warp; u < cnt; u += 2 * FAST_WARPS) {
+    const int np = u + FAST_WARPS < cnt ? 2 : 1;
+    float acc[2][4], acl[2][4];
 #pragma unroll
-            for (int i = 0; i < MB; ++i) {
-              if (sp0 + i < nsplit) {
-                ms[i] = __ldcg(src + (sp0 + i) * (HD + 2) + HD);
-                ls[i] = __ldcg(src + (sp0 + i) * (HD + 2) + HD + 1);
-                os[i] = __ldcg(src + (sp0 + i) * (HD + 2) + dd);
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < MB; ++i) {
-              if (sp0 + i < nsplit && ms[i] != -CUDART_INF_F) {  // running merge in split order
-                const float m_new = fmaxf(m_tot, ms[i]);
-                const float ca = __expf(m_tot - m_new), cb = __expf(ms[i] - m_new);
-                denom = denom * ca + ls[i] * cb;
-                ov = ov * ca + os[i] * cb;
-                m_tot = m_new;
-              }
-            }
+    for (int p = 0; p < 2; ++p) {
+      acc[p][0] = acc[p][1] = acc[p][2] = acc[p][3] = 0.f;
+      acl[p][0] = acl[p][1] = acl[p][2] = acl[p][3] = 0.f;
+      if (p < np) {
+#pragma unroll 1
+        for (int s = 0; s < KS; ++s) {
+          if (in_chunk == 0) {
+            ring_acquire(ring);
+            in_chunk = min(FAST_SLOT_TILES, left);
+            left -= in_chunk;
+            wb = ring.ring + ring.slot * FAST_SLOT_BYTES + lane * 8;
           }
-          write_frag_elem<T16>(P.xo, tok, hq * HD + dd, ov / denom);
+          uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
+          if (row0) {
+            const uint4 a = lds_v4(o_lane + s * (32 * W * 4));
+            ahi[0] = a.x; ahi[2] = a.y; alo[0] = a.z; alo[2] = a.w;
+          }
+          if (row1) {
+            const uint4 a = lds_v4(o_lane + s * (32 * W * 4) + 16);
+            ahi[1] = a.x; ahi[3] = a.y; alo[1] = a.z; alo[3] = a.w;
+          }
+          const uint2 bw = lds_v2(wb);
+          wb += FAST_TILE_BYTES;
+          mma_bf16(acc[p], ahi, bw.x, bw.y);
+          mma_bf16(acl[p], alo, bw.x, bw.y);
+          if (--in_chunk == 0) ring_release(ring, lane);
         }
       }
     }
+    ResidAdds<T16> ra[2];
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+      if (p < np) {
+        float c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[i] = acc[p][i] + acl[p][i];
+        resid_issue<T16>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, c, ra[p]);
+      }
+    }
+#pragma unroll
+    for (int p = 0; p < 2; ++p)
+      if (p < np) resid_finish<T16>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, ra[p]);
   }
 }
 
@@ -832,23 +855,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     const int bi = tid / P.R, r = tid % P.R;
     M.tok_stream[tid] = P.b0 + bi;
     M.tok_pos[tid] = P.len[P.b0 + bi] + r;
-  }
-
-  if (tid == 0) {
-    const int R = P.R, nb = P.nb, Hq = P.Hq;
-    int max_total = 0;
-    for (int bi = 0; bi < nb; ++bi) max_total = max(max_total, min(P.len[P.b0 + bi] + R, P.cap));
-    int nsplit = (max_total + P.keys_min - 1) / P.keys_min;
-    nsplit = max(1, min(nsplit, min(FAST_NSPLIT_CAP, max(1, P.m.n_cta / (nb * Hq)))));
-    M.attn_nsplit = nsplit;
-    const int item = cta;
-    if (item < nb * Hq * nsplit) {
-      const int c = item % nsplit, hq = (item / nsplit) % Hq, bi = item / (nsplit * Hq);
-      const int tot = min(P.len[P.b0 + bi] + R, P.cap);
-      const int per = (((tot + nsplit - 1) / nsplit) + 15) & ~15;
-      M.attn_item[0] = c; M.attn_item[1] = hq; M.attn_item[2] = bi;
-      M.attn_item[3] = c * per; M.attn_item[4] = min(c * per + per, tot);
-    }
   }
 
   // this warp's ring: barriers, then the first copies
@@ -919,7 +925,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   trace_mark(P, n_trace);
   // every CTA has read the base by now: publish the next launch's (this launch arrives 1 + 5 L times)
   if (ok && cta == 0 && tid == 0)
-    st_release_u32(P.epoch_base, epoch_base + (uint32_t)(1 + 5 * P.L) * (uint32_t)P.m.n_cta);
+    st_release_u32(P.epoch_base, epoch_base + (uint32_t)(1 + 4 * P.L) * (uint32_t)P.m.n_cta);
 
   // K slice of the down projection this CTA works on
   const int dsteps = P.F >> 4, dsl = cta % P.m.down_split;
@@ -927,13 +933,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   const int dk1 = (int)(((long long)(dsl + 1) * dsteps) / P.m.down_split) << 4;
   const float qscale = rsqrtf((float)P.hd);
 
-  // 5 phases per layer (QKV, attention, O, gate/up, down), then the LM head
-  const int n_phase = 5 * P.L + (P.logits ? 1 : 0);
+  // 4 phases per layer (QKV, attention + O, gate/up, down), then the LM head
+  const int n_phase = 4 * P.L + (P.logits ? 1 : 0);
+  const int n_ssq = (d + SSQ_COLS - 1) / SSQ_COLS * FAST_MAX_T;
   int l = 0, ph = 0;
 #pragma unroll 1
   for (int it = 0; it < n_phase && ok; ++it) {
-    if (it == 5 * P.L) ph = 5;
-    if (ph == 0 && cta == (l % P.m.n_cta) + 0 && l + 1 < P.L) {
+    if (it == 4 * P.L) ph = 4;
+    if (ph == 0 && cta == l % P.m.n_cta && l + 1 < P.L) {
       // the small per-layer constants are read once per forward, so they would miss all the way
       // to HBM in the middle of an epilogue: one CTA pulls the next layer's into L2 ahead of time
       const int nq = (P.Hq + 2 * P.Hkv) * P.hd;
@@ -942,38 +949,42 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       for (int i = tid; i < ((nq * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(bq + (size_t)i * 128);
       for (int i = tid; i < ((3 * d * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(gq + (size_t)i * 128);
     }
+    // A set of sums of squares is cleared while it is idle: the one the O projection adds to
+    // during the QKV phase, the one the down projection adds to during the attention + O phase.
+    if (ph < 2 && cta == P.m.n_cta - 1) {
+      long long* z = ph == 0 ? P.ssq_b : P.ssq_a;
+      for (int i = tid; i < n_ssq; i += FAST_THREADS) z[i] = 0;
+    }
+    PhaseDesc D;
+    D.layer = l;
+    D.qscale = qscale;
+    D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
+    D.xin = nullptr;
+    D.ssq_in = nullptr;
+    D.xout = nullptr;
+    D.ssq_out = nullptr;
+    D.gain_next = nullptr;
+    D.cinc = 0;
+    D.in_fix = 0;
+    D.kc = 0;
+    D.n_rows = d;
     if (ph == 1) {
-      if (cta == P.m.n_cta - 1) {
-        // both sets of sums of squares are idle during this phase (the O projection adds to one
-        // after the next barrier, the down projection to the other two barriers on): clear them
-        const int nw = (d + SSQ_COLS - 1) / SSQ_COLS * FAST_MAX_T;
-        for (int i = tid; i < nw; i += FAST_THREADS) P.ssq_a[i] = P.ssq_b[i] = 0;
-      }
-      if (P.hd == 64) attn_phase<64, T16>(P, M, uni, l);
-      else if (P.hd == 128) attn_phase<128, T16>(P, M, uni, l);
-      else attn_phase<32, T16>(P, M, uni, l);
+      D.op = FOP_O; D.epi = EPI_F_RESID;
+      D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
+      D.cinc = cta % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
+      if (P.hd == 64) attn_o_phase<64, T16>(P, M, uni, ring, D, l);
+      else if (P.hd == 128) attn_o_phase<128, T16>(P, M, uni, ring, D, l);
+      else attn_o_phase<32, T16>(P, M, uni, ring, D, l);
     } else {
-      PhaseDesc D;
-      D.layer = l;
-      D.qscale = qscale;
-      D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
-      D.ssq_in = nullptr;
-      D.xout = nullptr;
-      D.ssq_out = nullptr;
-      D.gain_next = nullptr;
-      D.cinc = 0;
       if (ph == 0) {
         D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
         D.kc = d; D.n_rows = qd + 2 * P.Hkv * P.hd;
       } else if (ph == 2) {
-        D.op = FOP_O; D.epi = EPI_F_RESID; D.in_fix = 0; D.xin = P.xo; D.kc = qd; D.n_rows = d;
-        D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
-      } else if (ph == 3) {
         D.op = FOP_GU; D.epi = EPI_F_SWIGLU; D.in_fix = 1; D.xin = P.xb; D.ssq_in = P.ssq_b;
         D.kc = d; D.n_rows = 2 * P.F;
-      } else if (ph == 4) {
-        D.op = FOP_DOWN; D.epi = EPI_F_RESID; D.in_fix = 0;
-        D.xin = P.xd + (size_t)(dk0 >> 4) * (T16 ? 256 : 128); D.kc = dk1 - dk0; D.n_rows = d;
+      } else if (ph == 3) {
+        D.op = FOP_DOWN; D.epi = EPI_F_RESID;
+        D.xin = P.xd + (size_t)(dk0 >> 4) * (T16 ? 256 : 128); D.kc = dk1 - dk0;
         D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = dsl == 0 ? 1 - P.m.down_split : 1;
         D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
       } else {
@@ -983,10 +994,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       gemm_phase<T16>(P, M, uni, ring, D, stage_parity);
     }
     trace_mark(P, n_trace);
-    if (ph < 5) {
+    if (ph < 4) {
       ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
       trace_mark(P, n_trace);
-      if (++ph == 5) {
+      if (++ph == 4) {
         ph = 0;
         ++l;
       }
@@ -1013,14 +1024,13 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
 
 }  // namespace
 
-size_t fast_union_bytes(int stage_k, int hd, int T, int R) {
+size_t fast_union_bytes(int stage_k, int hd, int T, int o_steps) {
   const bool t16 = T > 8;
   size_t af = (size_t)(stage_k / 16) * (t16 ? 1024 : 512);
   size_t red = (size_t)FAST_WARPS * FAST_MAXU * 32 * (t16 ? 16 : 8);
-  const int nrow = t16 ? 16 : 8;  // q operand, per-warp K / V tiles, per-warp partials (m, l, O)
+  const int nrow = t16 ? 16 : 8;  // q operand, per-warp K / V tiles, per-warp partials (m, l, O), output operand
   size_t attn = (size_t)(hd / 16) * 32 * (t16 ? 32 : 16) + (size_t)FAST_WARPS * 2 * 16 * (hd * 2 + 16) +
-                (size_t)FAST_WARPS * nrow * (hd + 2) * 4;
-  (void)R;
+                (size_t)FAST_WARPS * nrow * (hd + 2) * 4 + (size_t)o_steps * 32 * (t16 ? 32 : 16);
   size_t u = af + red > attn ? af + red : attn;
   return (u + 127) / 128 * 128;
 }
@@ -1029,7 +1039,7 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   FastParams p = p_in;
   if (p.T < 1 || p.T > FAST_MAX_T || p.m.n_cta > FAST_MAX_CTAS || p.m.max_units > FAST_MAX_UNITS)
     return cudaErrorInvalidValue;
-  const size_t uni = fast_union_bytes(p.m.max_stage_k, p.hd, p.T, p.R);
+  const size_t uni = fast_union_bytes(p.m.max_stage_k, p.hd, p.T, p.Hq / p.m.o_split * (p.hd / 16));
   const size_t misc = (sizeof(FastMisc) + 127) / 128 * 128;
   const size_t max_smem = 227 * 1024;
   if (uni + misc + (size_t)FAST_WARPS * 2 * FAST_SLOT_BYTES > max_smem) return cudaErrorInvalidValue;
@@ -1039,7 +1049,6 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   int nslot = (int)((max_smem - uni - misc) / ((size_t)FAST_WARPS * FAST_SLOT_BYTES));
   if (nslot > FAST_RING_SLOTS) nslot = FAST_RING_SLOTS;
   p.nslot = nslot;
-  p.keys_min = FAST_KEYS_MIN;
   p.ring_warp_bytes = nslot * FAST_SLOT_BYTES;
   p.union_off = FAST_WARPS * p.ring_warp_bytes;
   p.misc_off = p.union_off + (int)uni;

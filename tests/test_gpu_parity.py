@@ -245,7 +245,7 @@ def test_phase_trace_of_the_persistent_kernel():
     gs.forward(x, 4, lg)
     torch.cuda.synchronize()
     t = buf.cpu().numpy()
-    n_events = 3 + 2 * 5 * shape.n_layers + 1               # set-up, embedding + barrier, phases, head
+    n_events = 3 + 2 * 4 * shape.n_layers + 1               # set-up, embedding + barrier, phases, head
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     for cta in (0, sms - 1):
         row = t[cta]
