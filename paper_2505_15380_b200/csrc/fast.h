@@ -25,7 +25,7 @@ constexpr int FAST_WARPS = SSD_FAST_WARPS;  // warps per CTA; they split K of ev
 constexpr int FAST_THREADS = FAST_WARPS * 32;
 constexpr int FAST_TILE_BYTES = 256;  // one operand tile: 8 weight rows x 16 k, bf16
 #ifndef SSD_FAST_SLOT_TILES
-#define SSD_FAST_SLOT_TILES 16
+#define SSD_FAST_SLOT_TILES 20
 #endif
 constexpr int FAST_SLOT_TILES = SSD_FAST_SLOT_TILES;  // a ring slot holds one chunk of at most this many tiles
 constexpr int FAST_SLOT_BYTES = FAST_TILE_BYTES * FAST_SLOT_TILES;
