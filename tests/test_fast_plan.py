@@ -32,7 +32,7 @@ def test_plan_streams_every_projection_byte_once_and_evenly(L):
     # the algorithmic bytes of the step (norm gains, biases and head padding aside)
     assert abs(total - shape.streamed_weight_bytes()) < 256 * 1024
     assert mx <= 1.08 * total / 148 and mn >= 0.92 * total / 148      # balanced streams
-    assert down_split == 4 and max_units <= 16 and max_chunks <= 128
+    assert down_split == 8 and max_units <= 16 and max_chunks <= 128
     # tiles: every projection's tiles once; the O projection's once per query head and the down
     # projection's once per K slice (both are split over K)
     tiles = (qd + 2 * kvd) // 8 + shape.n_q_heads * d // 8 + 2 * F // 8 + down_split * d // 8 + (V + 7) // 8
