@@ -122,6 +122,14 @@ void ssd_streams_destroy(ssd_streams* s);
  * kernels only.  Both produce the same results up to fp32 summation order. */
 int ssd_streams_set_path(ssd_streams* s, int32_t path);
 
+/* Precision of the activations that enter the tensor cores in the persistent kernel (weights and
+ * K/V are bf16 as stored, accumulation is fp32, the residual stream is kept in fixed point, in
+ * both modes).  on = 1 (default): each activation enters as its bf16 leading part plus the bf16
+ * remainder, which agrees with a float64 evaluation of the 24-layer model to about 5e-4 in the
+ * logits.  on = 0: each activation is rounded to bf16, the arithmetic of ordinary bf16 inference;
+ * the logits then differ from a float64 evaluation by up to a few 1e-2. */
+int ssd_streams_set_activation_split(ssd_streams* s, int32_t on);
+
 /* Phase trace of the persistent kernel (a profiling aid, not part of the method).  With a device
  * buffer of ctas x events_per_cta int64 (ctas >= 256), thread 0 of every CTA stores its SM clock
  * (clock64) at each phase boundary of every later small-batch forward: after set-up, after the

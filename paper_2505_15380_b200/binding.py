@@ -20,6 +20,7 @@ _lib = None
 EXPORTS = [
     "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
     "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_streams_set_path",
+    "ssd_streams_set_activation_split",
     "ssd_streams_set_trace", "ssd_forward", "ssd_fast_plan_host",
     "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
@@ -68,6 +69,7 @@ def lib() -> ctypes.CDLL:
     L.ssd_streams_destroy.restype = None
     L.ssd_streams_destroy.argtypes = [vp]
     L.ssd_streams_set_path.argtypes = [vp, i32]
+    L.ssd_streams_set_activation_split.argtypes = [vp, i32]
     L.ssd_streams_set_trace.argtypes = [vp, vp, i32, i32]
     L.ssd_forward.argtypes = [vp, vp, vp, i32, vp, vp]
     L.ssd_fast_plan_host.argtypes = [cfgp, i32, ctypes.POINTER(ctypes.c_int64)]
@@ -183,6 +185,11 @@ class Streams:
     def set_path(self, path: int) -> None:
         """0: persistent small-batch kernel where the forward fits it (default); 1: generic kernels."""
         check(lib().ssd_streams_set_path(self.handle, path))
+
+    def set_activation_split(self, on: bool) -> None:
+        """Persistent kernel: True (default) feeds activations to the tensor cores as bf16 leading
+        part + remainder (near-fp32 inputs), False rounds them to bf16."""
+        check(lib().ssd_streams_set_activation_split(self.handle, 1 if on else 0))
 
     def set_trace(self, buf: Optional[torch.Tensor]) -> None:
         """buf: int64 CUDA tensor [ctas >= 256, events_per_cta] that receives the persistent

@@ -242,6 +242,7 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.logits = logits_out;
   p.flags = s->flags;
   p.epoch_base = s->epoch_base;
+  p.split_act = s->split_act;
   p.trace = s->trace;
   p.trace_cap = s->trace_cap;
   SSD_CUDA(launch_fast_forward(p, st));
@@ -489,6 +490,7 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->flags = (uint32_t*)(W + p.flags);
   s->epoch_base = (uint32_t*)(W + p.epoch_base);
   s->path = 0;
+  s->split_act = 1;
   s->trace = nullptr;
   s->trace_cap = 0;
   *out = s;
@@ -543,6 +545,13 @@ int ssd_forward(ssd_model* model, ssd_streams* s, const int32_t* dev_draft_token
   if (use_fast(model, s, rm)) return forward_fast(model, s, rm, nullptr, dev_draft_tokens, dev_logits, st);
   launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
   return forward(model, s, rm, dev_logits, st);
+}
+
+int ssd_streams_set_activation_split(ssd_streams* s, int32_t on) {
+  if (!s) return SSD_ERR_NULL;
+  if (on != 0 && on != 1) return SSD_ERR_BAD_PARAM;
+  s->split_act = on;
+  return SSD_OK;
 }
 
 int ssd_streams_set_path(ssd_streams* s, int32_t path) {

@@ -116,6 +116,7 @@ struct ssd_streams {
   uint32_t *xa, *xb, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
   long long *ssq_a, *ssq_b;
   uint32_t *flags, *epoch_base;
+  int split_act;     // persistent kernel: activations as bf16 hi + lo pairs (1) or plain bf16 (0)
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)
   int trace_cap;

@@ -158,11 +158,14 @@ struct FastParams {
   // phase boundary (before and after every grid barrier); null: off
   long long* trace;
   int trace_cap;
+  // 0: activations enter the tensor cores rounded to bf16 (one instruction per tile and k-step);
+  // 1: as bf16 leading part + bf16 remainder (two instructions, close to fp32 inputs)
+  int split_act;
   // shared-memory carve-up (bytes)
   int nslot, ring_warp_bytes, union_off, misc_off;
 };
 
-size_t fast_union_bytes(int stage_k, int head_dim, int T, int o_steps);
+size_t fast_union_bytes(int stage_k, int head_dim, int T, int o_steps, bool split);
 cudaError_t launch_fast_forward(const FastParams& p, cudaStream_t st);
 
 }  // namespace ssd

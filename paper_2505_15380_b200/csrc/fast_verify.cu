@@ -92,6 +92,10 @@ __device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t&
   hi = *reinterpret_cast<uint32_t*>(&h);
   lo = *reinterpret_cast<uint32_t*>(&l);
 }
+__device__ __forceinline__ uint32_t pack_bf16(float x, float y) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
 // Residual-stream word (2^-32 fixed point) -> fp32, through its two 32-bit halves.
 __device__ __forceinline__ float fix_to_float(long long v) {
   const int hi = (int)(v >> 32);
@@ -244,29 +248,53 @@ struct PhaseDesc {
 // (hi = bf16 leading part, lo = bf16 of the remainder) and, when more than 8 rows are in flight,
 // 16 more bytes for row g + 8.  Every value is converted once, by the thread that produces it,
 // instead of once per consuming CTA.
-template <bool T16>
+template <bool T16, bool LO>
+struct Lay {
+  static constexpr int WH = LO ? 4 : 2;          // words per (k-step, lane, row half)
+  static constexpr int W = WH * (T16 ? 2 : 1);   // words per (k-step, lane)
+  static constexpr int STEP = 32 * W * 4;        // bytes per k-step
+  // With at most 8 rows in flight the 16-row A operand has room for both parts of a split
+  // activation: rows 0..7 carry the bf16 leading parts, rows 8..15 the remainders of the same
+  // rows, so one instruction multiplies both and the two halves of the result are added at the end.
+  static constexpr bool MERGE = LO && !T16;
+};
+template <bool T16, bool LO>
 __device__ __forceinline__ uint32_t afrag_word(int row, int kk) {  // kk = column pair index
-  constexpr int W = T16 ? 8 : 4;
   const int s = kk >> 3, t = kk & 3, which = (kk >> 2) & 1;
-  return (uint32_t)(((s * 32 + (row & 7) * 4 + t) * W) + (row >> 3) * 4 + which);
+  return (uint32_t)(((s * 32 + (row & 7) * 4 + t) * Lay<T16, LO>::W) + (row >> 3) * Lay<T16, LO>::WH + which);
+}
+// One row half of this lane's share of a k-step of an operand in shared memory -> registers of
+// the A fragment (h = 0: rows g, registers 0 and 2; h = 1: rows g + 8, registers 1 and 3).
+template <bool LO>
+__device__ __forceinline__ void load_afrag(uint32_t addr, int h, uint32_t (&ahi)[4], uint32_t (&alo)[4]) {
+  if (LO) {
+    const uint4 a = lds_v4(addr);
+    ahi[h] = a.x; ahi[2 + h] = a.y; alo[h] = a.z; alo[2 + h] = a.w;
+  } else {
+    const uint2 a = lds_v2(addr);
+    ahi[h] = a.x; ahi[2 + h] = a.y;
+  }
 }
 // Columns (k, k + 1), k even, of row `row`.
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void write_frag_pair(uint32_t* buf, int row, int k, float x0, float x1) {
-  uint32_t hi, lo;
-  split2(x0, x1, hi, lo);
-  const uint32_t wd = afrag_word<T16>(row, k >> 1);
-  buf[wd] = hi;
-  buf[wd + 2] = lo;
+  const uint32_t wd = afrag_word<T16, LO>(row, k >> 1);
+  if (LO) {
+    uint32_t hi, lo;
+    split2(x0, x1, hi, lo);
+    buf[wd] = hi;
+    buf[wd + 2] = lo;
+  } else {
+    buf[wd] = pack_bf16(x0, x1);
+  }
 }
 // One column of row `row` (two 2-byte stores).
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void write_frag_elem(uint32_t* buf, int row, int k, float x) {
   const bf16 h = __float2bfloat16_rn(x);
-  const bf16 l = __float2bfloat16_rn(x - __bfloat162float(h));
-  bf16* w = reinterpret_cast<bf16*>(buf + afrag_word<T16>(row, k >> 1)) + (k & 1);
+  bf16* w = reinterpret_cast<bf16*>(buf + afrag_word<T16, LO>(row, k >> 1)) + (k & 1);
   w[0] = h;
-  w[4] = l;  // two words on
+  if (LO) w[4] = __float2bfloat16_rn(x - __bfloat162float(h));  // two words on
 }
 
 // inv_rms[t] = rsqrt(mean(x[t]^2) + eps) from the sums of squares the producers left, one 64-bit
@@ -303,11 +331,11 @@ __device__ __forceinline__ void ssq_finish(const SsqLoads& q, const long long* _
 }
 
 // One output element pair of a projection: token `tok`, packed weight rows n and n + 1.
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDesc& D, const FastMisc& M,
                                               int tok, int n, float c0, float c1) {
   if (D.epi == EPI_F_SWIGLU) {
-    write_frag_elem<T16>(P.xd, tok, n >> 1, __fdividef(c0, 1.f + __expf(-c0)) * c1);
+    write_frag_elem<T16, LO>(P.xd, tok, n >> 1, __fdividef(c0, 1.f + __expf(-c0)) * c1);
   } else if (D.epi == EPI_F_LOGITS) {
     if (n < D.n_rows) P.logits[(size_t)tok * P.V + n] = c0;
     if (n + 1 < D.n_rows) P.logits[(size_t)tok * P.V + n + 1] = c1;
@@ -322,8 +350,8 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
       const float o1 = x1 * cs.x - x2 * cs.y, o2 = x2 * cs.x + x1 * cs.y;
       if (n < qd) {
         const int col = (n & ~(hd - 1)) + j;  // q, pre-scaled, as the operand of the score contraction
-        write_frag_elem<T16>(P.xq, tok, col, o1 * D.qscale);
-        write_frag_elem<T16>(P.xq, tok, col + half, o2 * D.qscale);
+        write_frag_elem<T16, LO>(P.xq, tok, col, o1 * D.qscale);
+        write_frag_elem<T16, LO>(P.xq, tok, col + half, o2 * D.qscale);
       } else if (pos < P.cap) {
         const int gk = (n - qd) >> hs;
         bf16* kdst = D.kv_layer + (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * hd + (size_t)pos * hd;
@@ -349,14 +377,14 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
 // sum is a multiple of 16).  That thread turns the element into the operand of the next
 // projection (x * gain as bf16 hi / lo in operand layout) and adds x^2 to the row's sums of
 // squares for the RMS norm, in fixed point as well.
-template <bool T16>
+template <bool T16, bool LO>
 struct ResidAdds {
   long long inc[T16 ? 2 : 1][2], old[T16 ? 2 : 1][2];
   float2 gn;
 };
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void resid_issue(const FastParams& P, const PhaseDesc& D, int tile, int lane,
-                                            const float* c, ResidAdds<T16>& A) {
+                                            const float* c, ResidAdds<T16, LO>& A) {
   constexpr int NH = T16 ? 2 : 1;
   const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
   A.gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
@@ -372,9 +400,9 @@ __device__ __forceinline__ void resid_issue(const FastParams& P, const PhaseDesc
     }
   }
 }
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void resid_finish(const FastParams& P, const PhaseDesc& D, int tile, int lane,
-                                             const ResidAdds<T16>& A) {
+                                             const ResidAdds<T16, LO>& A) {
   constexpr int NH = T16 ? 2 : 1;
   const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
 #pragma unroll
@@ -388,7 +416,7 @@ __device__ __forceinline__ void resid_finish(const FastParams& P, const PhaseDes
         const long long now = A.old[h][j] + A.inc[h][j];
         if ((now & 15) == 0) {  // this add completed the element
           const float x = fix_to_float(now >> 4);
-          write_frag_elem<T16>(D.xout, row, n + j, x * (j ? A.gn.y : A.gn.x));
+          write_frag_elem<T16, LO>(D.xout, row, n + j, x * (j ? A.gn.y : A.gn.x));
           sq += __float2ll_rn(x * x * FIX_SCALE);
           any = true;
         }
@@ -399,23 +427,24 @@ __device__ __forceinline__ void resid_finish(const FastParams& P, const PhaseDes
     }
   }
 }
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
                                            const float* c) {
-  ResidAdds<T16> A;
-  resid_issue<T16>(P, D, tile, lane, c, A);
-  resid_finish<T16>(P, D, tile, lane, A);
+  ResidAdds<T16, LO> A;
+  resid_issue<T16, LO>(P, D, tile, lane, c, A);
+  resid_finish<T16, LO>(P, D, tile, lane, A);
 }
 
 // The tensor-core work of one round of CNT tiles over this warp's k-steps [s0, s1): straight-line
 // per chunk (one ring slot = SPC whole k-steps), partial sums to shared memory at the end.
-template <int CNT, bool T16>
+template <int CNT, bool T16, bool LO>
 __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, int s0, int s1, bool row0,
                                           bool row1, float* red_dst) {
   constexpr int SPC = FAST_SLOT_TILES / CNT;
-  constexpr uint32_t STEP = T16 ? 1024u : 512u;
+  constexpr uint32_t STEP = Lay<T16, LO>::STEP;
   constexpr int NACC = T16 ? 4 : 2;
-  constexpr bool TWO = CNT <= 4;  // few tiles: keep the hi and lo terms in separate accumulators
+  constexpr bool MERGE = Lay<T16, LO>::MERGE;
+  constexpr bool TWO = LO && !MERGE && CNT <= 4;  // few tiles: the hi and lo terms in separate accumulators
   float acc[CNT][4], acl[TWO ? CNT : 1][4];
 #pragma unroll
   for (int u = 0; u < CNT; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
@@ -428,24 +457,22 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 #pragma unroll
     for (int i = 0; i < SPC; ++i) {
       if (SPC == 1 || s + i < s1) {
-        uint32_t ahi[4], alo[4];
-        uint4 a = make_uint4(0u, 0u, 0u, 0u);
-        if (row0) a = lds_v4(af_lane + (uint32_t)(s + i) * STEP);
-        ahi[0] = a.x; ahi[2] = a.y; alo[0] = a.z; alo[2] = a.w;
-        if (T16) {
-          uint4 a2 = make_uint4(0u, 0u, 0u, 0u);
-          if (row1) a2 = lds_v4(af_lane + (uint32_t)(s + i) * STEP + 16u);
-          ahi[1] = a2.x; ahi[3] = a2.y; alo[1] = a2.z; alo[3] = a2.w;
-        } else {
-          ahi[1] = ahi[3] = alo[1] = alo[3] = 0u;
-        }
+        uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
+        if (row0) load_afrag<LO>(af_lane + (uint32_t)(s + i) * STEP, 0, ahi, alo);
+        if (T16 && row1) load_afrag<LO>(af_lane + (uint32_t)(s + i) * STEP + Lay<T16, LO>::WH * 4, 1, ahi, alo);
         uint2 b[CNT];
 #pragma unroll
         for (int u = 0; u < CNT; ++u) b[u] = lds_v2(wb + (uint32_t)(i * CNT + u) * FAST_TILE_BYTES);
+        if (MERGE) {
+          ahi[1] = alo[0];
+          ahi[3] = alo[2];
+        }
 #pragma unroll
         for (int u = 0; u < CNT; ++u) mma_bf16(acc[u], ahi, b[u].x, b[u].y);
+        if (LO && !MERGE) {
 #pragma unroll
-        for (int u = 0; u < CNT; ++u) mma_bf16(TWO ? acl[u] : acc[u], alo, b[u].x, b[u].y);
+          for (int u = 0; u < CNT; ++u) mma_bf16(TWO ? acl[u] : acc[u], alo, b[u].x, b[u].y);
+        }
       }
     }
     ring_release(r, lane);
@@ -460,6 +487,10 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 #pragma unroll
   for (int u = 0; u < CNT; ++u) {
     float* dst = red_dst + (size_t)u * 32 * NACC;
+    if (MERGE) {
+      acc[u][0] += acc[u][2];
+      acc[u][1] += acc[u][3];
+    }
     *reinterpret_cast<float2*>(dst) = make_float2(acc[u][0], acc[u][1]);
     if (T16) *reinterpret_cast<float2*>(dst + 2) = make_float2(acc[u][2], acc[u][3]);
   }
@@ -467,7 +498,7 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
 
 // One projection phase: copy the input operand to shared memory, run this CTA's tiles (the warps
 // split K), add the warps' partial sums in shared memory and apply the epilogue.
-template <bool T16>
+template <bool T16, bool LO>
 __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
                                            const PhaseDesc& D, uint32_t& stage_parity) {
   constexpr int NACC = T16 ? 4 : 2;
@@ -476,7 +507,7 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   const int T = P.T, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2;
   const int KS = D.kc >> 4;
   uint32_t* af = reinterpret_cast<uint32_t*>(uni);                             // A operand, KS steps
-  float* red = reinterpret_cast<float*>(uni + (size_t)KS * (T16 ? 1024 : 512));  // [warp][MAXU][32][NACC]
+  float* red = reinterpret_cast<float*>(uni + (size_t)KS * Lay<T16, LO>::STEP);  // [warp][MAXU][32][NACC]
   const int s0 = fast_warp_k0(warp, KS), s1 = fast_warp_k1(warp, KS);
   SsqLoads ssq;
   if (D.in_fix) ssq_issue(ssq, D.ssq_in, (P.d + SSQ_COLS - 1) / SSQ_COLS, T);
@@ -484,33 +515,33 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   // this warp's k-steps of the operand: one bulk copy from L2 (the producers' stores were made
   // visible by the grid barrier; the proxy fence orders that observation before the async read)
   const uint32_t sbar = smem_u32(&M.sbar[warp]);
-  const uint32_t stage_bytes = (uint32_t)(s1 - s0) * (T16 ? 1024u : 512u);
+  const uint32_t stage_bytes = (uint32_t)(s1 - s0) * Lay<T16, LO>::STEP;
   if (stage_bytes && lane == 0) {
     asm volatile("fence.proxy.async;" ::: "memory");
     mbar_expect_tx(sbar, stage_bytes);
-    bulk_g2s(smem_u32(af) + (uint32_t)s0 * (T16 ? 1024u : 512u),
-             reinterpret_cast<const uint8_t*>(D.xin) + (size_t)s0 * (T16 ? 1024 : 512), stage_bytes, sbar);
+    bulk_g2s(smem_u32(af) + (uint32_t)s0 * Lay<T16, LO>::STEP,
+             reinterpret_cast<const uint8_t*>(D.xin) + (size_t)s0 * Lay<T16, LO>::STEP, stage_bytes, sbar);
   }
   if (stage_bytes) {
     if (!mbar_try_wait(sbar, stage_parity) && !bounded_mbar_wait(sbar, stage_parity)) ring.dead = true;
     stage_parity ^= 1u;
   }
-  const uint32_t af_lane = smem_u32(af) + lane * (T16 ? 32u : 16u);
+  const uint32_t af_lane = smem_u32(af) + lane * (Lay<T16, LO>::W * 4);
   float* red_dst = red + ((size_t)warp * FAST_MAXU * 32 + lane) * NACC;
 
   for (int u0 = 0; u0 < cnt_total; u0 += FAST_MAXU) {
     const int cnt = min(FAST_MAXU, cnt_total - u0);
     switch (cnt) {
-      case 1: mma_round<1, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 2: mma_round<2, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 3: mma_round<3, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 4: mma_round<4, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 5: mma_round<5, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 6: mma_round<6, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 7: mma_round<7, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 8: mma_round<8, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      case 9: mma_round<9, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
-      default: mma_round<10, T16>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 1: mma_round<1, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 2: mma_round<2, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 3: mma_round<3, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 4: mma_round<4, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 5: mma_round<5, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 6: mma_round<6, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 7: mma_round<7, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 8: mma_round<8, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      case 9: mma_round<9, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
+      default: mma_round<10, T16, LO>(ring, lane, af_lane, s0, s1, row0, row1, red_dst); break;
     }
     if (D.in_fix && u0 == 0) ssq_finish(ssq, D.ssq_in, (P.d + SSQ_COLS - 1) / SSQ_COLS, T, D.kc, P.eps, M);
     __syncthreads();
@@ -527,16 +558,16 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
       }
       const int tile = M.utile[D.op][u0 + u];
       if (D.epi == EPI_F_RESID) {
-        resid_tile<T16>(P, D, tile, l, c);
+        resid_tile<T16, LO>(P, D, tile, l, c);
       } else {
         const int n = tile * 8 + 2 * tt;
         if (gg < T) {
           const float inv = D.in_fix ? M.inv_rms[gg] : 1.f;
-          epilogue_pair<T16>(P, D, M, gg, n, c[0] * inv, c[1] * inv);
+          epilogue_pair<T16, LO>(P, D, M, gg, n, c[0] * inv, c[1] * inv);
         }
         if (T16 && gg + 8 < T) {
           const float inv = D.in_fix ? M.inv_rms[gg + 8] : 1.f;
-          epilogue_pair<T16>(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv);
+          epilogue_pair<T16, LO>(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv);
         }
       }
     }
@@ -573,12 +604,14 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 //
 // O projection: the warps split the CTA's tiles (tile u: warp u % 8), two tiles at a time so that
 // the residual adds of both are in flight together.
-template <int HD, bool T16>
+template <int HD, bool T16, bool LO>
 __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
                                              const PhaseDesc& D, int layer) {
   constexpr int ROWB = HD * 2 + 16;       // padded K / V row in bytes (conflict-free fragment loads)
   constexpr int NH = T16 ? 2 : 1;         // row halves: rows g and g + 8
-  constexpr int W = T16 ? 8 : 4;          // words per (k-step, lane) of an operand
+  constexpr int W = Lay<T16, LO>::W;      // words per (k-step, lane) of an operand
+  constexpr int WH = Lay<T16, LO>::WH;
+  constexpr bool MERGE = Lay<T16, LO>::MERGE;
   constexpr int KSTEPS = HD / 16;
   constexpr int DT = HD / 8;              // 8-dim tiles of the output
   constexpr int CH = HD / 8;              // 16-byte chunks per row
@@ -594,8 +627,11 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
   uint8_t* kv_w = uni + KSTEPS * 32 * W * 4 + warp * (2 * 16 * ROWB);     // this warp's K then V tile
   float* cm = reinterpret_cast<float*>(uni + KSTEPS * 32 * W * 4 + FAST_WARPS * 2 * 16 * ROWB);  // [warp][NROW]
   float* cl = cm + FAST_WARPS * NROW;
-  float* co = cl + FAST_WARPS * NROW;                                      // [warp][NROW][HD]
-  uint32_t* osm = reinterpret_cast<uint32_t*>(co + FAST_WARPS * NROW * HD);  // attention output, KS steps
+  uint32_t* osm = reinterpret_cast<uint32_t*>(cl + FAST_WARPS * NROW);     // attention output, KS steps
+  // a warp's partial output [NROW][HD] takes the place of its K / V tiles once its keys are done
+  static_assert(NROW * HD * 4 <= 2 * 16 * ROWB, "partial output must fit the warp's staging area");
+  constexpr int CO_W = 2 * 16 * ROWB / 4;                                  // floats between warps' partials
+  float* co = reinterpret_cast<float*>(uni + KSTEPS * 32 * W * 4);
   const uint32_t q_lane = smem_u32(qsm) + lane * (W * 4);
   const uint32_t k_lane = smem_u32(kv_w) + g * ROWB + t * 4;
   const uint32_t v_lane = smem_u32(kv_w) + 16 * ROWB + (lane & 15) * ROWB;
@@ -671,17 +707,25 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
       for (int j = 0; j < 2; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
 #pragma unroll
       for (int s = 0; s < KSTEPS; ++s) {
-        const uint4 qa = lds_v4(q_lane + s * (32 * W * 4));
-        uint32_t ahi[4] = {qa.x, 0u, qa.y, 0u}, alo[4] = {qa.z, 0u, qa.w, 0u};
-        if (T16) {
-          const uint4 qb = lds_v4(q_lane + s * (32 * W * 4) + 16);
-          ahi[1] = qb.x; ahi[3] = qb.y; alo[1] = qb.z; alo[3] = qb.w;
+        uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
+        load_afrag<LO>(q_lane + s * (32 * W * 4), 0, ahi, alo);
+        if (T16) load_afrag<LO>(q_lane + s * (32 * W * 4) + WH * 4, 1, ahi, alo);
+        if (MERGE) {
+          ahi[1] = alo[0];
+          ahi[3] = alo[2];
         }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           const uint32_t b0 = lds_u32(k_lane + j * 8 * ROWB + s * 32), b1 = lds_u32(k_lane + j * 8 * ROWB + s * 32 + 16);
           mma_bf16(sc[j], ahi, b0, b1);
-          mma_bf16(sc[j], alo, b0, b1);
+          if (LO && !MERGE) mma_bf16(sc[j], alo, b0, b1);
+        }
+      }
+      if (MERGE) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          sc[j][0] += sc[j][2];
+          sc[j][1] += sc[j][3];
         }
       }
       // mask, running max / sum, weights as the A operand of the second contraction
@@ -718,20 +762,45 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
         l_run[h] = l_run[h] * corr + ls;
         m_run[h] = m_new;
 #pragma unroll
-        for (int dt = 0; dt < DT; ++dt) { o[dt][2 * h] *= corr; o[dt][2 * h + 1] *= corr; }
-        split2(pw[0][0], pw[0][1], phi[h], plo[h]);          // keys 2t, 2t + 1
-        split2(pw[1][0], pw[1][1], phi[2 + h], plo[2 + h]);  // keys 8 + 2t, 8 + 2t + 1
+        for (int dt = 0; dt < DT; ++dt) {
+          o[dt][2 * h] *= corr;
+          o[dt][2 * h + 1] *= corr;
+          if (MERGE) {
+            o[dt][2] *= corr;
+            o[dt][3] *= corr;
+          }
+        }
+        if (LO) {
+          split2(pw[0][0], pw[0][1], phi[h], plo[h]);          // keys 2t, 2t + 1
+          split2(pw[1][0], pw[1][1], phi[2 + h], plo[2 + h]);  // keys 8 + 2t, 8 + 2t + 1
+        } else {
+          phi[h] = pack_bf16(pw[0][0], pw[0][1]);
+          phi[2 + h] = pack_bf16(pw[1][0], pw[1][1]);
+          plo[h] = plo[2 + h] = 0u;
+        }
       }
       if (!T16) phi[1] = phi[3] = plo[1] = plo[3] = 0u;
+      if (MERGE) {
+        phi[1] = plo[0];
+        phi[3] = plo[2];
+      }
 #pragma unroll
       for (int dt = 0; dt < DT; ++dt) {
         uint32_t b0, b1;
         ldmatrix_x2_trans(v_lane + dt * 16, b0, b1);
         mma_bf16(o[dt], phi, b0, b1);
-        mma_bf16(o[dt], plo, b0, b1);
+        if (LO && !MERGE) mma_bf16(o[dt], plo, b0, b1);
+      }
+    }
+    if (MERGE) {
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        o[dt][0] += o[dt][2];
+        o[dt][1] += o[dt][3];
       }
     }
     // this warp's partial -> shared memory; then all warps combine
+    __syncwarp();  // every lane is done with the warp's last K / V tile
     if (t == 0) {
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
@@ -743,7 +812,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
     for (int dt = 0; dt < DT; ++dt) {
 #pragma unroll
       for (int h = 0; h < NH; ++h)
-        *reinterpret_cast<float2*>(co + ((size_t)warp * NROW + g + 8 * h) * HD + dt * 8 + 2 * t) =
+        *reinterpret_cast<float2*>(co + (size_t)warp * CO_W + (g + 8 * h) * HD + dt * 8 + 2 * t) =
             make_float2(o[dt][2 * h], o[dt][2 * h + 1]);
     }
     __syncthreads();
@@ -759,13 +828,13 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
 #pragma unroll
       for (int w = 0; w < FAST_WARPS; ++w) {  // fixed order: bit-reproducible
         const float e = mw[w] == -CUDART_INF_F ? 0.f : __expf(mw[w] - m);
-        const float2 ov = *reinterpret_cast<const float2*>(co + ((size_t)w * NROW + tok) * HD + dd);
+        const float2 ov = *reinterpret_cast<const float2*>(co + (size_t)w * CO_W + tok * HD + dd);
         l = fmaf(cl[w * NROW + tok], e, l);
         o0 = fmaf(ov.x, e, o0);
         o1 = fmaf(ov.y, e, o1);
       }
       const float il = 1.f / l;
-      write_frag_pair<T16>(osm, tok, hl * HD + dd, o0 * il, o1 * il);
+      write_frag_pair<T16, LO>(osm, tok, hl * HD + dd, o0 * il, o1 * il);
     }
   }
   __syncthreads();
@@ -792,41 +861,43 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
             wb = ring.ring + ring.slot * FAST_SLOT_BYTES + lane * 8;
           }
           uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
-          if (row0) {
-            const uint4 a = lds_v4(o_lane + s * (32 * W * 4));
-            ahi[0] = a.x; ahi[2] = a.y; alo[0] = a.z; alo[2] = a.w;
-          }
-          if (row1) {
-            const uint4 a = lds_v4(o_lane + s * (32 * W * 4) + 16);
-            ahi[1] = a.x; ahi[3] = a.y; alo[1] = a.z; alo[3] = a.w;
+          if (row0) load_afrag<LO>(o_lane + s * (32 * W * 4), 0, ahi, alo);
+          if (row1) load_afrag<LO>(o_lane + s * (32 * W * 4) + WH * 4, 1, ahi, alo);
+          if (MERGE) {
+            ahi[1] = alo[0];
+            ahi[3] = alo[2];
           }
           const uint2 bw = lds_v2(wb);
           wb += FAST_TILE_BYTES;
           mma_bf16(acc[p], ahi, bw.x, bw.y);
-          mma_bf16(acl[p], alo, bw.x, bw.y);
+          if (LO && !MERGE) mma_bf16(acl[p], alo, bw.x, bw.y);
           if (--in_chunk == 0) ring_release(ring, lane);
         }
       }
     }
-    ResidAdds<T16> ra[2];
+    ResidAdds<T16, LO> ra[2];
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
       if (p < np) {
         float c[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[i] = acc[p][i] + acl[p][i];
-        resid_issue<T16>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, c, ra[p]);
+        if (MERGE) {
+          c[0] += c[2];
+          c[1] += c[3];
+        }
+        resid_issue<T16, LO>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, c, ra[p]);
       }
     }
 #pragma unroll
     for (int p = 0; p < 2; ++p)
-      if (p < np) resid_finish<T16>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, ra[p]);
+      if (p < np) resid_finish<T16, LO>(P, D, M.utile[FOP_O][u + p * FAST_WARPS], lane, ra[p]);
   }
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
 
-template <bool T16>
+template <bool T16, bool LO>
 __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __grid_constant__ FastParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, cta = blockIdx.x;
@@ -905,7 +976,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
         const float2 gn = __ldg(g0 + kk);
         *reinterpret_cast<longlong2*>(P.hfix + (size_t)tok * d + 2 * kk) =
             make_longlong2(__float2ll_rn(x.x * FIX_SCALE) * 16, __float2ll_rn(x.y * FIX_SCALE) * 16);
-        write_frag_pair<T16>(P.xa, tok, 2 * kk, x.x * gn.x, x.y * gn.y);
+        write_frag_pair<T16, LO>(P.xa, tok, 2 * kk, x.x * gn.x, x.y * gn.y);
         ss = __float2ll_rn(x.x * x.x * FIX_SCALE) + __float2ll_rn(x.y * x.y * FIX_SCALE);
       }
 #pragma unroll
@@ -972,9 +1043,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       D.op = FOP_O; D.epi = EPI_F_RESID;
       D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
       D.cinc = cta % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
-      if (P.hd == 64) attn_o_phase<64, T16>(P, M, uni, ring, D, l);
-      else if (P.hd == 128) attn_o_phase<128, T16>(P, M, uni, ring, D, l);
-      else attn_o_phase<32, T16>(P, M, uni, ring, D, l);
+      if (P.hd == 64) attn_o_phase<64, T16, LO>(P, M, uni, ring, D, l);
+      else if (P.hd == 128) attn_o_phase<128, T16, LO>(P, M, uni, ring, D, l);
+      else attn_o_phase<32, T16, LO>(P, M, uni, ring, D, l);
     } else {
       if (ph == 0) {
         D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
@@ -984,14 +1055,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
         D.kc = d; D.n_rows = 2 * P.F;
       } else if (ph == 3) {
         D.op = FOP_DOWN; D.epi = EPI_F_RESID;
-        D.xin = P.xd + (size_t)(dk0 >> 4) * (T16 ? 256 : 128); D.kc = dk1 - dk0;
+        D.xin = P.xd + (size_t)(dk0 >> 4) * (32 * Lay<T16, LO>::W); D.kc = dk1 - dk0;
         D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = dsl == 0 ? 1 - P.m.down_split : 1;
         D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
       } else {
         D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
         D.layer = 0; D.kc = d; D.n_rows = P.V;
       }
-      gemm_phase<T16>(P, M, uni, ring, D, stage_parity);
+      gemm_phase<T16, LO>(P, M, uni, ring, D, stage_parity);
     }
     trace_mark(P, n_trace);
     if (ph < 4) {
@@ -1024,13 +1095,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
 
 }  // namespace
 
-size_t fast_union_bytes(int stage_k, int hd, int T, int o_steps) {
+size_t fast_union_bytes(int stage_k, int hd, int T, int o_steps, bool split) {
   const bool t16 = T > 8;
-  size_t af = (size_t)(stage_k / 16) * (t16 ? 1024 : 512);
+  const size_t step = (size_t)128 * (t16 ? 2 : 1) * (split ? 4 : 2);  // operand bytes per k-step
+  size_t af = (size_t)(stage_k / 16) * step;
   size_t red = (size_t)FAST_WARPS * FAST_MAXU * 32 * (t16 ? 16 : 8);
-  const int nrow = t16 ? 16 : 8;  // q operand, per-warp K / V tiles, per-warp partials (m, l, O), output operand
-  size_t attn = (size_t)(hd / 16) * 32 * (t16 ? 32 : 16) + (size_t)FAST_WARPS * 2 * 16 * (hd * 2 + 16) +
-                (size_t)FAST_WARPS * nrow * (hd + 2) * 4 + (size_t)o_steps * 32 * (t16 ? 32 : 16);
+  const int nrow = t16 ? 16 : 8;  // q operand, per-warp K / V tiles (later the partial O), m and l, output operand
+  size_t attn = (size_t)(hd / 16) * step + (size_t)FAST_WARPS * 2 * 16 * (hd * 2 + 16) +
+                (size_t)FAST_WARPS * nrow * 2 * 4 + (size_t)o_steps * step;
   size_t u = af + red > attn ? af + red : attn;
   return (u + 127) / 128 * 128;
 }
@@ -1039,7 +1111,7 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   FastParams p = p_in;
   if (p.T < 1 || p.T > FAST_MAX_T || p.m.n_cta > FAST_MAX_CTAS || p.m.max_units > FAST_MAX_UNITS)
     return cudaErrorInvalidValue;
-  const size_t uni = fast_union_bytes(p.m.max_stage_k, p.hd, p.T, p.Hq / p.m.o_split * (p.hd / 16));
+  const size_t uni = fast_union_bytes(p.m.max_stage_k, p.hd, p.T, p.Hq / p.m.o_split * (p.hd / 16), p.split_act != 0);
   const size_t misc = (sizeof(FastMisc) + 127) / 128 * 128;
   const size_t max_smem = 227 * 1024;
   if (uni + misc + (size_t)FAST_WARPS * 2 * FAST_SLOT_BYTES > max_smem) return cudaErrorInvalidValue;
@@ -1054,7 +1126,9 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   p.misc_off = p.union_off + (int)uni;
   const size_t smem = (size_t)p.misc_off + misc;
   const bool t16 = p.T > 8;
-  const void* kern = t16 ? (const void*)fast_forward_kernel<true> : (const void*)fast_forward_kernel<false>;
+  const void* kern = p.split_act
+                         ? (t16 ? (const void*)fast_forward_kernel<true, true> : (const void*)fast_forward_kernel<false, true>)
+                         : (t16 ? (const void*)fast_forward_kernel<true, false> : (const void*)fast_forward_kernel<false, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   void* args[] = {(void*)&p};

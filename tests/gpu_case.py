@@ -61,7 +61,7 @@ def _topk_gap_small(logits_row: np.ndarray, temperature: float, top_k: int) -> b
 def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "prefill",
              oracle_streams: Optional[List[int]] = None, logit_tol: Optional[float] = None,
              uniform_seed: int = 0, commit_and_repeat: bool = False,
-             capacity: Optional[int] = None, path: int = 0) -> CaseResult:
+             capacity: Optional[int] = None, path: int = 0, split: bool = True) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -74,6 +74,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
     cap = capacity or (max(wl.prefix_lens) + 2 * R + 8)
     gs = binding.Streams(gmodel, B, cap, gamma)
     gs.set_path(path)          # 0: persistent kernel where the forward fits it, 1: generic kernels
+    gs.set_activation_split(split)   # persistent kernel: bf16 activations, or bf16 hi + lo pairs
     which = list(range(B)) if oracle_streams is None else list(oracle_streams)
     prefixes = [synth.make_prefix(wl, b) for b in range(B)]
     ostreams = {}

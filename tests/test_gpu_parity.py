@@ -74,8 +74,16 @@ def test_mha_no_grouping_and_single_kv_head():
 
 
 def test_cfg1_qwen2_style_prefill_300():
+    """The 24-layer step sits far inside the 3e-2 bound: activations enter the tensor cores as
+    bf16 hi + lo pairs, so what is left is fp32 accumulation order and the K/V storage rounding."""
     r = _case(synth.workload(1), beta=0.0, sigma=0.5, commit_and_repeat=True)
-    assert r.max_logit_err < 3e-2
+    assert r.max_logit_err < 1e-3
+
+
+def test_cfg1_with_plain_bf16_activations():
+    """The optional mode that rounds every activation to bf16 (ordinary bf16 inference)."""
+    r = _case(synth.workload(1), beta=0.0, sigma=0.5, split=False, logit_tol=6e-2)
+    assert r.max_logit_err > 1e-3      # the mode really is a different arithmetic
 
 
 @pytest.mark.parametrize("gamma,prefix", [(2, 256), (4, 512), (6, 1024), (8, 2048)])
@@ -179,13 +187,16 @@ def _fast_shape(hd, hq=4, hkv=2, d=128, f=256, v=300, layers=2):
 @pytest.mark.parametrize("hd,batch,gamma,lens", [
     (64, 1, 4, [20]), (64, 2, 2, [70, 129]), (32, 1, 8, [300]), (128, 3, 4, [1, 64, 700]),
     (64, 1, 15, [33]), (64, 4, 3, [5, 127, 128, 129])])
-def test_persistent_kernel_against_oracle(hd, batch, gamma, lens):
+@pytest.mark.parametrize("split", [False, True])
+def test_persistent_kernel_against_oracle(hd, batch, gamma, lens, split):
     """Rows <= 8 and <= 16, several streams in one forward, prefixes around the 16-key tiles and
-    the 128-key passes of the attention phase, all three head sizes."""
+    the 128-key passes of the attention phase, all three head sizes; activations as bf16 hi + lo
+    pairs (the default), which must sit close to the float64 oracle, and as plain bf16."""
     shape = _fast_shape(hd, hq=14 if hd == 64 else 4, hkv=2)
     wl = _wl(shape, batch, gamma, lens)
-    _case(wl, beta=0.0, sigma=0.5, path=0)
-    _case(wl, beta=0.4, sigma=2.0, commit_and_repeat=True, path=0)
+    tol = 2e-4 if split else 6e-2     # plain bf16 activations: the rounding of ordinary bf16 inference
+    _case(wl, beta=0.0, sigma=0.5, path=0, split=split, logit_tol=tol)
+    _case(wl, beta=0.4, sigma=2.0, commit_and_repeat=True, path=0, split=split, logit_tol=tol)
 
 
 def test_generic_kernels_still_cover_small_bf16_forwards():
@@ -210,6 +221,7 @@ def test_both_paths_agree_and_forward_only_matches():
     for path in (0, 1):
         gs = binding.Streams(model, B, 200, g)
         gs.set_path(path)
+        gs.set_activation_split(True)                         # near-fp32 inputs, like the generic kernels
         synth.fill_synthetic_kv(gs.kv, lens, seed=5)
         gs.kv_truncate(lens, [3, 4])
         k = torch.zeros(B, dtype=torch.int32, device=dev)
