@@ -6,22 +6,26 @@
 // mbarriers; a slot is refilled the moment its chunk has been consumed, whatever phase the consumer
 // is in, so the weight stream runs ahead of the dependency chain across phase boundaries.  The
 // ring is kept shallow on purpose: a few KB in flight per warp already saturate HBM (measured).
-// The phases of a layer (QKV projection, attention, O projection, gate/up, down) are separated by
+// The phases of a layer (QKV projection, attention + O projection, gate/up, down) are separated by
 // grid barriers on one monotonic arrival counter, with bounded waits.
 //
-// The forward is a chain of 5 dependent phases per layer, each far shorter than a microsecond of
+// The forward is a chain of 4 dependent phases per layer, each far shorter than a microsecond of
 // memory time, so what bounds it is latency: the instructions a warp executes per phase (eight
 // warps per SM hide little) and the round trips through L2 between phases.  Hence: every activation
 // is converted to the tensor-core operand layout (bf16 hi + lo) once, by the thread that produces
 // it, and consumers fetch their slice with one bulk copy; the weight stream is pre-cut into chunks
 // of whole k-steps so the inner loop is straight-line for each tile count; everything rare is out
-// of line; attention keeps its weights in registers between its two contractions.
+// of line; attention keeps its weights in registers between its two contractions; projections
+// that are split over K across CTAs (O by query head, down by column range) add into a
+// fixed-point residual stream whose words carry an arrival count, so the thread that completes
+// an element finishes it without a further exchange.
 //
 // Projections: D[token, weight row] = sum_k X[token, k] * W[row, k] on mma.m16n8k16 (bf16 inputs,
 // fp32 accumulate): the 16-row A operand holds the tokens, the B operand one packed tile of 8 weight
 // rows.  Activations are fp32 and enter the instruction as a two-term bf16 split (hi + lo), so the
-// products are exact to ~2^-17 relative; weights are exactly their stored bf16 values.  The warps
-// of a CTA split K; their partial sums are added in a fixed order in shared memory.
+// products are exact to ~2^-17 relative; weights are exactly their stored bf16 values.  With at
+// most 8 rows both terms ride in one instruction (rows 0..7 hi, rows 8..15 lo).  The warps of a
+// CTA split K; their partial sums are added in a fixed order in shared memory.
 #include <math_constants.h>
 
 #include "fast.h"
