@@ -155,11 +155,9 @@ def run_reference(args):
 def run_cuda(args):
     import torch
     import torch.distributed as dist
-    from paper_2505_15380_b200 import binding, synth
+    from paper_2505_15380_b200 import binding, replicas, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
     torch.cuda.set_device(local)
@@ -225,8 +223,7 @@ def run_cuda(args):
         for _ in range(max(args.warmup, 3)):
             graph.replay()
         stream.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(world)
         torch.cuda.synchronize()
         clocks = ClockSampler(local)
         clocks.start()
@@ -237,6 +234,7 @@ def run_cuda(args):
         e1.record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
+        replicas.barrier(world)
         dev_ms = e0.elapsed_time(e1)
         k_timed = d_k.cpu().numpy().copy()
         # the dominant kernel alone: the decoder forward (one persistent kernel when the forward has
@@ -289,10 +287,7 @@ def run_cuda(args):
     assert gs.last_status() == 0, "device status flags raised during the benchmark"
     assert np.array_equal(h_k.numpy(), k_timed), "host-buffer path disagrees with the device path"
 
-    t = torch.tensor([dev_ms, e2e_ms, fwd_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dev_ms, e2e_ms, fwd_ms = float(t[0]), float(t[1]), float(t[2])
+    dev_ms, e2e_ms, fwd_ms = replicas.slowest([dev_ms, e2e_ms, fwd_ms], world, dev)   # max over ranks
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
