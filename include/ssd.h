@@ -230,8 +230,8 @@ int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_draft_tokens,
 
 /* Plan of the persistent small-batch kernel for a bf16 model on n_cta CTAs.  out8 receives:
  * packed bytes in total, fewest / most bytes any CTA streams, most output tiles a CTA owns for one
- * projection, most chunks in a warp's table, K slices of the down projection, warps per CTA,
- * output tiles over all CTAs and projections.  SSD_ERR_BAD_CONFIG if the model has no such path. */
+ * projection, most chunks in a warp's table, K slices of the down projection, K slices (groups
+ * of query heads) of the O projection, output tiles over all CTAs and projections.  SSD_ERR_BAD_CONFIG if the model has no such path. */
 int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8);
 /* Packs the projection weights of host_weights (blob of ssd_model_create) into the per-warp streams
  * and walks the streams back into host_out (same layout and size; only the projection matrices and

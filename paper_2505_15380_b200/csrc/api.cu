@@ -518,7 +518,7 @@ int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8
   out8[3] = mu;
   out8[4] = p.max_chunks;
   out8[5] = p.ops[FOP_DOWN].ksplit;
-  out8[6] = FAST_WARPS;
+  out8[6] = p.ops[FOP_O].ksplit;
   out8[7] = (int64_t)p.unit_tile.size();
   return SSD_OK;
 }

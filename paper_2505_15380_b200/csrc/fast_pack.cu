@@ -115,8 +115,10 @@ bool fast_supported(const ssd_model_config& c) {
 }
 
 int fast_o_split(const ssd_model_config& c, int n_cta) {
+  // whole heads per slice; at most 16 slices, the most the 4-bit arrival count of a residual
+  // element can tell apart (and every slice needs a CTA)
   int s = 1;
-  for (int v = 1; v <= c.n_q_heads && v <= n_cta; ++v)
+  for (int v = 1; v <= c.n_q_heads && v <= n_cta && v <= 16; ++v)
     if (c.n_q_heads % v == 0) s = v;
   return s;
 }

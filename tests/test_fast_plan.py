@@ -22,7 +22,7 @@ def _plan(L, shape, n_cta):
 
 def test_plan_streams_every_projection_byte_once_and_evenly(L):
     shape = synth.workload(1).target                      # 24 layers, d 896, FFN 4864, vocab 6564
-    rc, (total, mn, mx, max_units, max_chunks, down_split, warps, n_tiles) = _plan(L, shape, 148)
+    rc, (total, mn, mx, max_units, max_chunks, down_split, o_split, n_tiles) = _plan(L, shape, 148)
     assert rc == 0
     d, F, V, Lyr = shape.d_model, shape.d_ffn, shape.vocab_out, shape.n_layers
     qd, kvd = shape.n_q_heads * shape.head_dim, shape.n_kv_heads * shape.head_dim
@@ -32,7 +32,7 @@ def test_plan_streams_every_projection_byte_once_and_evenly(L):
     # the algorithmic bytes of the step (norm gains, biases and head padding aside)
     assert abs(total - shape.streamed_weight_bytes()) < 256 * 1024
     assert mx <= 1.08 * total / 148 and mn >= 0.92 * total / 148      # balanced streams
-    assert down_split == 8 and max_units <= 16 and max_chunks <= 128
+    assert down_split == 8 and o_split == 14 and max_units <= 16 and max_chunks <= 128
     # tiles: every projection's tiles once; the O projection's once per query head and the down
     # projection's once per K slice (both are split over K)
     tiles = (qd + 2 * kvd) // 8 + shape.n_q_heads * d // 8 + 2 * F // 8 + down_split * d // 8 + (V + 7) // 8
@@ -50,6 +50,17 @@ def test_plan_holds_for_other_sm_counts(L, n_cta):
         assert out[2] <= 1.35 * out[0] / n_cta
 
 
+def test_k_slices_stay_within_the_arrival_count(L):
+    """Projections split over K add into residual words that count arrivals in 4 bits: never more
+    than 16 slices, whole heads per slice of the O projection, and a CTA for every slice."""
+    for hq, hkv, n_cta, want in [(14, 2, 148, 14), (32, 2, 148, 16), (28, 4, 148, 14), (17, 17, 148, 1),
+                                 (12, 2, 148, 12), (8, 1, 7, 4), (8, 1, 1, 1), (64, 8, 148, 16)]:
+        shape = synth.ModelShape(2, 256, hq, hkv, 32, 8960, 500, 0, 1e4, weight_dtype=synth.BF16)
+        rc, out = _plan(L, shape, n_cta)
+        assert rc == 0 and out[6] == want and out[5] <= 16
+        assert hq % out[6] == 0
+
+
 def test_plan_rejects_models_without_the_path(L):
     assert _plan(L, synth.workload(0).target, 148)[0] == -2            # fp32 weights
     odd = synth.ModelShape(2, 128, 6, 2, 64, 200, 300, 8, 1e4, weight_dtype=synth.BF16)
@@ -61,6 +72,8 @@ def test_plan_rejects_models_without_the_path(L):
     (synth.ModelShape(2, 128, 14, 2, 64, 256, 301, 8, 1e4, weight_dtype=synth.BF16), 148),
     (synth.ModelShape(1, 256, 4, 2, 128, 2816, 700, 8, 1e4, weight_dtype=synth.BF16), 37),
     (synth.ModelShape(2, 128, 4, 2, 32, 512, 513, 0, 1e4, weight_dtype=synth.BF16), 5),
+    (synth.ModelShape(1, 64, 32, 4, 32, 64, 100, 0, 1e4, weight_dtype=synth.BF16), 148),   # two heads per O slice
+    (synth.ModelShape(1, 64, 5, 5, 64, 64, 100, 0, 1e4, weight_dtype=synth.BF16), 3),      # all heads in one slice
 ])
 def test_pack_then_walk_the_streams_reproduces_every_weight(L, shape, n_cta):
     """Packing permutes rows (rotary partners and gate/up made adjacent), tiles and splits K;

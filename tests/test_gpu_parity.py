@@ -199,6 +199,14 @@ def test_persistent_kernel_against_oracle(hd, batch, gamma, lens, split):
     _case(wl, beta=0.4, sigma=2.0, commit_and_repeat=True, path=0, split=split, logit_tol=tol)
 
 
+def test_persistent_kernel_with_several_heads_per_o_slice():
+    """32 query heads: the O projection is cut into 16 K slices of two heads, so a CTA computes the
+    attention of two heads and its warps walk chunks that straddle output tiles."""
+    shape = _fast_shape(32, hq=32, hkv=4, d=128, f=256, v=300, layers=2)
+    _case(_wl(shape, 2, 3, [40, 200]), beta=0.2, sigma=1.0, commit_and_repeat=True, path=0, logit_tol=2e-4)
+    _case(_wl(shape, 3, 4, [17, 90, 33]), beta=0.0, sigma=0.5, path=0, logit_tol=2e-4)      # 15 rows
+
+
 def test_generic_kernels_still_cover_small_bf16_forwards():
     shape = _fast_shape(64, hq=14, hkv=2)
     _case(_wl(shape, 2, 4, [70, 129]), beta=0.0, sigma=0.5, path=1)
