@@ -13,7 +13,7 @@
 
 namespace ssd {
 
-constexpr int SAMP_THREADS = 256;
+constexpr int SAMP_THREADS = 1024;  // a row of a few thousand logits: short per-thread loops
 
 struct RowStats {
   float zmax;        // max of z = logit / T over the row
@@ -121,15 +121,28 @@ __device__ int block_inverse_cdf(const float* w, int V, float u, SampSmem& sm, d
   const int t0 = min(threadIdx.x * seg, V), t1 = min(t0 + seg, V);
   double s = 0.0;
   for (int t = t0; t < t1; ++t) s += (double)w[t];
-  sm.scan[threadIdx.x] = s;
   if (threadIdx.x == 0) sm.y = -1;
-  __syncthreads();
-  if (threadIdx.x == 0) {  // 256 adds: a serial scan is cheap and order-exact
-    double run = 0.0;
-    for (int i = 0; i < SAMP_THREADS; ++i) {
-      run += sm.scan[i];
-      sm.scan[i] = run;
+  {  // inclusive scan of the threads' sums in a fixed order: inside each warp, then over the warps
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double n = __shfl_up_sync(0xffffffffu, s, o);
+      if (lane >= o) s += n;
     }
+    if (lane == 31) sm.red_d[wp] = s;
+    __syncthreads();
+    if (wp == 0) {
+      double v = lane < SAMP_THREADS / 32 ? sm.red_d[lane] : 0.0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const double n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+      }
+      if (lane < SAMP_THREADS / 32) sm.red_d[lane] = v;
+    }
+    __syncthreads();
+    if (wp > 0) s += sm.red_d[wp - 1];
+    sm.scan[threadIdx.x] = s;
   }
   __syncthreads();
   const double total = sm.scan[SAMP_THREADS - 1];
