@@ -64,6 +64,20 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// The same copy with an L2 eviction priority.  The weight stream is read once per forward and is
+// six times the size of L2: marked evict-first it stops pushing out what the phases re-read (the
+// operands between phases, the prefetched keys and values, the per-layer constants).
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                              uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -156,7 +170,7 @@ __device__ __forceinline__ void ring_request(Ring& r, uint32_t slot, int lane) {
     if (lane == 0) {
       const uint32_t bar = r.bars + slot * 8;
       mbar_expect_tx(bar, n * FAST_TILE_BYTES);
-      bulk_g2s(r.ring + slot * FAST_SLOT_BYTES, r.src, n * FAST_TILE_BYTES, bar);
+      bulk_g2s_hint(r.ring + slot * FAST_SLOT_BYTES, r.src, n * FAST_TILE_BYTES, bar, policy_evict_first());
     }
     r.src += n * FAST_TILE_BYTES;
     r.outstanding++;
