@@ -201,8 +201,9 @@ __device__ __forceinline__ void ring_release(Ring& r, int lane) {
   }
 }
 
+template <bool TRACE>
 __device__ __forceinline__ void trace_mark(const FastParams& P, int& n_trace) {
-  if (P.trace && threadIdx.x == 0 && n_trace < P.trace_cap)
+  if (TRACE && threadIdx.x == 0 && n_trace < P.trace_cap)
     P.trace[(size_t)blockIdx.x * P.trace_cap + n_trace++] = clock64();
 }
 
@@ -916,7 +917,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
 
 // ---- the kernel --------------------------------------------------------------------------------
 
-template <bool T16, bool LO>
+template <bool T16, bool LO, bool TRACE>
 __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __grid_constant__ FastParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, cta = blockIdx.x;
@@ -972,7 +973,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   const uint32_t epoch_base = ld_acquire_u32(P.epoch_base);
   uint32_t epoch = 0;
   __syncthreads();
-  trace_mark(P, n_trace);
+  trace_mark<TRACE>(P, n_trace);
 
   const int T = P.T, d = P.d, qd = P.Hq * P.hd, half = P.hd >> 1;
 
@@ -1010,9 +1011,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       P.rope_cs[((size_t)tok * half + j) * 2 + 1] = (float)sn;
     }
   }
-  trace_mark(P, n_trace);
+  trace_mark<TRACE>(P, n_trace);
   bool ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, false);
-  trace_mark(P, n_trace);
+  trace_mark<TRACE>(P, n_trace);
   // every CTA has read the base by now: publish the next launch's (this launch arrives 1 + 5 L times)
   if (ok && cta == 0 && tid == 0)
     st_release_u32(P.epoch_base, epoch_base + (uint32_t)(1 + 4 * P.L) * (uint32_t)P.m.n_cta);
@@ -1083,10 +1084,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       }
       gemm_phase<T16, LO>(P, M, uni, ring, D, stage_parity);
     }
-    trace_mark(P, n_trace);
+    trace_mark<TRACE>(P, n_trace);
     if (ph < 4) {
       ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
-      trace_mark(P, n_trace);
+      trace_mark<TRACE>(P, n_trace);
       if (++ph == 4) {
         ph = 0;
         ++l;
@@ -1145,9 +1146,13 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   p.misc_off = p.union_off + (int)uni;
   const size_t smem = (size_t)p.misc_off + misc;
   const bool t16 = p.T > 8;
-  const void* kern = p.split_act
-                         ? (t16 ? (const void*)fast_forward_kernel<true, true> : (const void*)fast_forward_kernel<false, true>)
-                         : (t16 ? (const void*)fast_forward_kernel<true, false> : (const void*)fast_forward_kernel<false, false>);
+  // the phase trace is a variant of its own: the common path carries no trace code
+  const void* table[8] = {
+      (const void*)fast_forward_kernel<false, false, false>, (const void*)fast_forward_kernel<false, false, true>,
+      (const void*)fast_forward_kernel<false, true, false>,  (const void*)fast_forward_kernel<false, true, true>,
+      (const void*)fast_forward_kernel<true, false, false>,  (const void*)fast_forward_kernel<true, false, true>,
+      (const void*)fast_forward_kernel<true, true, false>,   (const void*)fast_forward_kernel<true, true, true>};
+  const void* kern = table[(t16 ? 4 : 0) + (p.split_act ? 2 : 0) + (p.trace ? 1 : 0)];
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   void* args[] = {(void*)&p};
