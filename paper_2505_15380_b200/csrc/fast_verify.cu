@@ -915,6 +915,58 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
   }
 }
 
+// What the phases of one CTA share for the whole forward.
+struct PhaseCtx {
+  float qscale;
+  int dk0, dk1, dsl;  // K slice of the down projection this CTA works on
+  int qd;
+};
+
+// Phase PH of layer l: 0 QKV, 1 attention + O projection, 2 gate/up, 3 down, 4 LM head.
+template <int PH, bool T16, bool LO>
+__device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
+                                          const PhaseCtx& C, int l, uint32_t& stage_parity) {
+  const int d = P.d;
+  PhaseDesc D;
+  D.layer = l;
+  D.qscale = C.qscale;
+  D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
+  D.xin = nullptr;
+  D.ssq_in = nullptr;
+  D.xout = nullptr;
+  D.ssq_out = nullptr;
+  D.gain_next = nullptr;
+  D.cinc = 0;
+  D.in_fix = 0;
+  D.kc = 0;
+  D.n_rows = d;
+  if (PH == 1) {
+    D.op = FOP_O; D.epi = EPI_F_RESID;
+    D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
+    D.cinc = (int)blockIdx.x % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
+    if (P.hd == 64) attn_o_phase<64, T16, LO>(P, M, uni, ring, D, l);
+    else if (P.hd == 128) attn_o_phase<128, T16, LO>(P, M, uni, ring, D, l);
+    else attn_o_phase<32, T16, LO>(P, M, uni, ring, D, l);
+    return;
+  }
+  if (PH == 0) {
+    D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
+    D.kc = d; D.n_rows = C.qd + 2 * P.Hkv * P.hd;
+  } else if (PH == 2) {
+    D.op = FOP_GU; D.epi = EPI_F_SWIGLU; D.in_fix = 1; D.xin = P.xb; D.ssq_in = P.ssq_b;
+    D.kc = d; D.n_rows = 2 * P.F;
+  } else if (PH == 3) {
+    D.op = FOP_DOWN; D.epi = EPI_F_RESID;
+    D.xin = P.xd + (size_t)(C.dk0 >> 4) * (32 * Lay<T16, LO>::W); D.kc = C.dk1 - C.dk0;
+    D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = C.dsl == 0 ? 1 - P.m.down_split : 1;
+    D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
+  } else {
+    D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
+    D.layer = 0; D.kc = d; D.n_rows = P.V;
+  }
+  gemm_phase<T16, LO>(P, M, uni, ring, D, stage_parity);
+}
+
 // ---- the kernel --------------------------------------------------------------------------------
 
 template <bool T16, bool LO, bool TRACE>
@@ -1024,14 +1076,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   const int dk1 = (int)(((long long)(dsl + 1) * dsteps) / P.m.down_split) << 4;
   const float qscale = rsqrtf((float)P.hd);
 
-  // 4 phases per layer (QKV, attention + O, gate/up, down), then the LM head
-  const int n_phase = 4 * P.L + (P.logits ? 1 : 0);
+  // 4 phases per layer (QKV, attention + O, gate/up, down), then the LM head.  Each phase is its
+  // own call site, so that what a phase is (its projection, input, epilogue) is known at compile
+  // time there: every instruction between two barriers is on the critical path.
   const int n_ssq = (d + SSQ_COLS - 1) / SSQ_COLS * FAST_MAX_T;
-  int l = 0, ph = 0;
+  const PhaseCtx C{qscale, dk0, dk1, dsl, qd};
 #pragma unroll 1
-  for (int it = 0; it < n_phase && ok; ++it) {
-    if (it == 4 * P.L) ph = 4;
-    if (ph == 0 && cta == l % P.m.n_cta && l + 1 < P.L) {
+  for (int l = 0; l < P.L && ok; ++l) {
+    if (l + 1 < P.L && cta == l % P.m.n_cta) {
       // the small per-layer constants are read once per forward, so they would miss all the way
       // to HBM in the middle of an epilogue: one CTA pulls the next layer's into L2 ahead of time
       const int nq = (P.Hq + 2 * P.Hkv) * P.hd;
@@ -1042,59 +1094,34 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     }
     // A set of sums of squares is cleared while it is idle: the one the O projection adds to
     // during the QKV phase, the one the down projection adds to during the attention + O phase.
-    if (ph < 2 && cta == P.m.n_cta - 1) {
-      long long* z = ph == 0 ? P.ssq_b : P.ssq_a;
-      for (int i = tid; i < n_ssq; i += FAST_THREADS) z[i] = 0;
-    }
-    PhaseDesc D;
-    D.layer = l;
-    D.qscale = qscale;
-    D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
-    D.xin = nullptr;
-    D.ssq_in = nullptr;
-    D.xout = nullptr;
-    D.ssq_out = nullptr;
-    D.gain_next = nullptr;
-    D.cinc = 0;
-    D.in_fix = 0;
-    D.kc = 0;
-    D.n_rows = d;
-    if (ph == 1) {
-      D.op = FOP_O; D.epi = EPI_F_RESID;
-      D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
-      D.cinc = cta % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
-      if (P.hd == 64) attn_o_phase<64, T16, LO>(P, M, uni, ring, D, l);
-      else if (P.hd == 128) attn_o_phase<128, T16, LO>(P, M, uni, ring, D, l);
-      else attn_o_phase<32, T16, LO>(P, M, uni, ring, D, l);
-    } else {
-      if (ph == 0) {
-        D.op = FOP_QKV; D.epi = EPI_F_QKV; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
-        D.kc = d; D.n_rows = qd + 2 * P.Hkv * P.hd;
-      } else if (ph == 2) {
-        D.op = FOP_GU; D.epi = EPI_F_SWIGLU; D.in_fix = 1; D.xin = P.xb; D.ssq_in = P.ssq_b;
-        D.kc = d; D.n_rows = 2 * P.F;
-      } else if (ph == 3) {
-        D.op = FOP_DOWN; D.epi = EPI_F_RESID;
-        D.xin = P.xd + (size_t)(dk0 >> 4) * (32 * Lay<T16, LO>::W); D.kc = dk1 - dk0;
-        D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = dsl == 0 ? 1 - P.m.down_split : 1;
-        D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
-      } else {
-        D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
-        D.layer = 0; D.kc = d; D.n_rows = P.V;
-      }
-      gemm_phase<T16, LO>(P, M, uni, ring, D, stage_parity);
-    }
+    if (cta == P.m.n_cta - 1)
+      for (int i = tid; i < n_ssq; i += FAST_THREADS) P.ssq_b[i] = 0;
+    run_phase<0, T16, LO>(P, M, uni, ring, C, l, stage_parity);
     trace_mark<TRACE>(P, n_trace);
-    if (ph < 4) {
-      ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
-      trace_mark<TRACE>(P, n_trace);
-      if (++ph == 4) {
-        ph = 0;
-        ++l;
-      }
-    } else if (__syncthreads_or(ring.dead ? 1 : 0)) {
-      ok = false;
-    }
+    ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
+    trace_mark<TRACE>(P, n_trace);
+    if (!ok) break;
+    if (cta == P.m.n_cta - 1)
+      for (int i = tid; i < n_ssq; i += FAST_THREADS) P.ssq_a[i] = 0;
+    run_phase<1, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    trace_mark<TRACE>(P, n_trace);
+    ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
+    trace_mark<TRACE>(P, n_trace);
+    if (!ok) break;
+    run_phase<2, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    trace_mark<TRACE>(P, n_trace);
+    ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
+    trace_mark<TRACE>(P, n_trace);
+    if (!ok) break;
+    run_phase<3, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    trace_mark<TRACE>(P, n_trace);
+    ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
+    trace_mark<TRACE>(P, n_trace);
+  }
+  if (ok && P.logits) {
+    run_phase<4, T16, LO>(P, M, uni, ring, C, 0, stage_parity);
+    trace_mark<TRACE>(P, n_trace);
+    if (__syncthreads_or(ring.dead ? 1 : 0)) ok = false;
   }
   if (!ok && tid == 0) {
     // a wait ran out here or elsewhere: make the failure sticky
