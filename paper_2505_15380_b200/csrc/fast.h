@@ -1,5 +1,5 @@
 // Persistent small-batch verify kernel ("fast path"): shared definitions of the host-side plan /
-// weight packer (fast_pack.cu) and of the kernel and its launcher (fast_verify.cu).
+// weight packer (fast_pack.cu) and of the kernel (fast_kernel.cuh) and its launcher (fast_verify.cu).
 //
 // The verify forward of Eq. 4 over T = B * (gamma + 1) <= 16 rows is bound by streaming every
 // weight byte once and, because each of its ~120 phases depends on the one before, by how few
@@ -147,7 +147,7 @@ struct FastParams {
   long long* hfix;  // residual stream [T][d]: 2^-32 fixed point above a 4-bit arrival count
   float *rope_cs, *logits;  // logits null: skip the LM head
   // Inputs of the projections, written by their producers already in the tensor-core operand layout
-  // (bf16 leading part + remainder, see fast_verify.cu): the RMS-norm inputs x * gain of the QKV /
+  // (bf16 leading part + remainder, see fast_kernel.cuh): the RMS-norm inputs x * gain of the QKV /
   // LM-head projection (xa) and of gate/up (xb), SiLU(g) * u (xd); and
   // per 64 columns and row the sums of squares that go with xa / xb.
   uint32_t *xa, *xb, *xd, *xq;  // xq: the rotated, scaled queries
