@@ -29,6 +29,9 @@ constexpr int FAST_TILE_BYTES = 256;  // one operand tile: 8 weight rows x 16 k,
 #endif
 constexpr int FAST_SLOT_TILES = SSD_FAST_SLOT_TILES;  // a ring slot holds one chunk of at most this many tiles
 constexpr int FAST_SLOT_BYTES = FAST_TILE_BYTES * FAST_SLOT_TILES;
+// Chunks of the O projection's stream (runs of a warp's own tiles): a power of two, so that a pair
+// of output tiles with 2, 4 or 8 k-steps each never straddles two chunks.
+constexpr int FAST_O_CHUNK = 16;
 constexpr int FAST_MAX_SLOTS = 8;     // most ring slots per warp (barrier storage)
 #ifndef SSD_FAST_RING_SLOTS
 #define SSD_FAST_RING_SLOTS 3

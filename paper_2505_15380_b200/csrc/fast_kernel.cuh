@@ -876,12 +876,45 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
     for (int p = 0; p < 2; ++p) {
       acc[p][0] = acc[p][1] = acc[p][2] = acc[p][3] = 0.f;
       acl[p][0] = acl[p][1] = acl[p][2] = acl[p][3] = 0.f;
+    }
+    if (hps == 1) {
+      // One head per slice (any GPU with at least as many SMs as query heads): KSTEPS k-steps, and
+      // a pair of tiles never straddles a chunk, so both run as independent chains, unrolled.  With
+      // a single tile the second chain multiplies whatever follows in shared memory, unused.
+      if (in_chunk == 0) {
+        ring_acquire(ring);
+        in_chunk = min(FAST_O_CHUNK, left);
+        left -= in_chunk;
+        wb = ring.ring + ring.slot * FAST_SLOT_BYTES + lane * 8;
+      }
+#pragma unroll
+      for (int s = 0; s < KSTEPS; ++s) {
+        uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
+        if (row0) load_afrag<LO>(o_lane + s * (32 * W * 4), 0, ahi, alo);
+        if (row1) load_afrag<LO>(o_lane + s * (32 * W * 4) + WH * 4, 1, ahi, alo);
+        if (MERGE) {
+          ahi[1] = alo[0];
+          ahi[3] = alo[2];
+        }
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          const uint2 bw = lds_v2(wb + (p * KSTEPS + s) * FAST_TILE_BYTES);
+          mma_bf16(acc[p], ahi, bw.x, bw.y);
+          if (LO && !MERGE) mma_bf16(acl[p], alo, bw.x, bw.y);
+        }
+      }
+      wb += np * KSTEPS * FAST_TILE_BYTES;
+      in_chunk -= np * KSTEPS;
+      if (in_chunk == 0) ring_release(ring, lane);
+    } else {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
       if (p < np) {
 #pragma unroll 1
         for (int s = 0; s < KS; ++s) {
           if (in_chunk == 0) {
             ring_acquire(ring);
-            in_chunk = min(FAST_SLOT_TILES, left);
+            in_chunk = min(FAST_O_CHUNK, left);
             left -= in_chunk;
             wb = ring.ring + ring.slot * FAST_SLOT_BYTES + lane * 8;
           }
@@ -899,6 +932,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
           if (--in_chunk == 0) ring_release(ring, lane);
         }
       }
+    }
     }
     ResidAdds<T16, LO> ra[2];
 #pragma unroll

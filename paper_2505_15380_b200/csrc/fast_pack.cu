@@ -16,7 +16,7 @@
 // at most FAST_SLOT_TILES tiles: one chunk is one bulk copy into one ring slot.  The O projection
 // is the exception: its K is split by groups of query heads over the CTAs, the warps of a CTA split
 // its tiles (warp w: tiles w, w + FAST_WARPS, ..), each tile with all k-steps of the slice in
-// order, and the chunks are simply runs of FAST_SLOT_TILES tiles of that sequence.
+// order, and the chunks are simply runs of FAST_O_CHUNK tiles of that sequence.
 #include <string.h>
 
 #include <algorithm>
@@ -193,7 +193,7 @@ FastPlan fast_make_plan(const ssd_model_config& c, int n_cta) {
         std::vector<uint8_t>& ch = op == FOP_HEAD ? ch_head : ch_layer;
         if (p.ops[op].by_tile) {
           const int nt = fast_warp_tiles(w, cnt_total) * slice_steps;
-          for (int t0 = 0; t0 < nt; t0 += FAST_SLOT_TILES) ch.push_back((uint8_t)std::min(FAST_SLOT_TILES, nt - t0));
+          for (int t0 = 0; t0 < nt; t0 += FAST_O_CHUNK) ch.push_back((uint8_t)std::min(FAST_O_CHUNK, nt - t0));
           tiles_layer += (uint64_t)nt;
           continue;
         }
@@ -314,7 +314,7 @@ long long fast_unpack_streams(const ssd_model_config& c, const FastPlan& plan, c
             int left = fast_warp_tiles(w, cnt_total) * steps, in_chunk = 0, u = w, ks = 0;
             while (left > 0) {
               if (in_chunk == 0) {
-                in_chunk = std::min(FAST_SLOT_TILES, left);
+                in_chunk = std::min(FAST_O_CHUNK, left);
                 if (tab[ci++] != in_chunk) ++bad;
               }
               scatter_tile(c, v, blob_out, op, ll, tiles[u] * 8, sk0 + ks, src);
