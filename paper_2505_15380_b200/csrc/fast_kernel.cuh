@@ -681,7 +681,8 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
         vq[i] = __ldcg(vg + (size_t)key * CH + idx % CH);
       }
     }
-    __syncthreads();  // the previous user of the shared memory (projection phase or item) is done
+    if (item > 0) __syncthreads();  // the previous item is done with the shared memory (the first
+                                    // item starts right behind a grid barrier)
     {                 // q of this head (operand layout, bf16 hi / lo as the QKV epilogue left it)
       const uint4* src = reinterpret_cast<const uint4*>(P.xq + (size_t)hq * KSTEPS * 32 * W);
       for (int i = tid; i < KSTEPS * 32 * W / 4; i += FAST_THREADS) reinterpret_cast<uint4*>(qsm)[i] = __ldcg(src + i);
