@@ -31,9 +31,9 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   const size_t misc = (fast_misc_bytes() + 127) / 128 * 128;
   const size_t max_smem = 227 * 1024;
   if (uni + misc + (size_t)FAST_WARPS * 2 * FAST_SLOT_BYTES > max_smem) return cudaErrorInvalidValue;
-  // A shallow ring on purpose: 8 KB in flight per warp already saturate HBM, and refill traffic in
-  // flight beyond that only queues ahead of the phases' latency-critical loads (3 slots of 4 KB
-  // measured best: 852 us against 861 with 2 and 885 with 4 on the 24-layer d = 896 model).
+  // A shallow ring on purpose: a few KB in flight per warp already saturate HBM, and refill traffic
+  // in flight beyond that only queues ahead of the phases' latency-critical loads (3 slots of 5 KB
+  // measured best on the 24-layer d = 896 model: 637 us per step against 645 with 4 and 654 with 2).
   int nslot = (int)((max_smem - uni - misc) / ((size_t)FAST_WARPS * FAST_SLOT_BYTES));
   if (nslot > FAST_RING_SLOTS) nslot = FAST_RING_SLOTS;
   p.nslot = nslot;
