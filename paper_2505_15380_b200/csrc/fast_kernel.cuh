@@ -355,10 +355,26 @@ __device__ __forceinline__ void ssq_finish(const SsqLoads& q, const long long* _
   }
 }
 
+// The constants the QKV epilogue needs for one output pair of token `tok`: the biases of packed
+// rows n, n + 1 and the rotation (cos, sin) of the token's position.  The threads that run the
+// first pass of the epilogue load theirs at the start of the phase, off the critical path.
+struct QkvConsts {
+  float2 bias, cs;
+};
+__device__ __forceinline__ QkvConsts qkv_consts(const FastParams& P, const PhaseDesc& D, int tok, int n) {
+  const int hd = P.hd, hs = P.hd_shift, qd = P.Hq << hs, kvd = P.Hkv << hs;
+  QkvConsts q;
+  q.bias = *reinterpret_cast<const float2*>(P.m.bias_qkv + (size_t)D.layer * (qd + 2 * kvd) + n);
+  q.cs = make_float2(1.f, 0.f);
+  if (n < qd + kvd)
+    q.cs = __ldcg(reinterpret_cast<const float2*>(P.rope_cs + ((size_t)tok * (hd >> 1) + ((n & (hd - 1)) >> 1)) * 2));
+  return q;
+}
+
 // One output element pair of a projection: token `tok`, packed weight rows n and n + 1.
 template <bool T16, bool LO>
 __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDesc& D, const FastMisc& M,
-                                              int tok, int n, float c0, float c1) {
+                                              int tok, int n, float c0, float c1, const QkvConsts& qc) {
   if (D.epi == EPI_F_SWIGLU) {
     write_frag_elem<T16, LO>(P.xd, tok, n >> 1, __fdividef(c0, 1.f + __expf(-c0)) * c1);
   } else if (D.epi == EPI_F_LOGITS) {
@@ -366,12 +382,11 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
     if (n + 1 < D.n_rows) P.logits[(size_t)tok * P.V + n + 1] = c1;
   } else {  // EPI_F_QKV: bias, rotary embedding, q scaling, K/V append
     const int hd = P.hd, hs = P.hd_shift, half = hd >> 1, qd = P.Hq << hs, kvd = P.Hkv << hs;
-    const float2 bias = *reinterpret_cast<const float2*>(P.m.bias_qkv + (size_t)D.layer * (qd + 2 * kvd) + n);
-    const float x1 = c0 + bias.x, x2 = c1 + bias.y;
+    const float x1 = c0 + qc.bias.x, x2 = c1 + qc.bias.y;
     const int stream = M.tok_stream[tok], pos = M.tok_pos[tok];
     if (n < qd + kvd) {
       const int j = (n & (hd - 1)) >> 1;
-      const float2 cs = __ldcg(reinterpret_cast<const float2*>(P.rope_cs + ((size_t)tok * half + j) * 2));
+      const float2 cs = qc.cs;
       const float o1 = x1 * cs.x - x2 * cs.y, o2 = x2 * cs.x + x1 * cs.y;
       if (n < qd) {
         const int col = (n & ~(hd - 1)) + j;  // q, pre-scaled, as the operand of the score contraction
@@ -537,6 +552,13 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
   SsqLoads ssq;
   if (D.in_fix) ssq_issue(ssq, D.ssq_in, (P.d + SSQ_COLS - 1) / SSQ_COLS, T);
   const bool row0 = g < T, row1 = T16 && g + 8 < T;
+  QkvConsts qc0, qc1;  // of this thread's outputs in the first pass of the first round's epilogue
+  qc0.bias = qc0.cs = qc1.bias = qc1.cs = make_float2(0.f, 0.f);
+  if (D.epi == EPI_F_QKV && tid < min(FAST_MAXU, cnt_total) * 32) {
+    const int n = M.utile[D.op][warp] * 8 + 2 * (lane & 3);
+    if (row0) qc0 = qkv_consts(P, D, g, n);
+    if (row1) qc1 = qkv_consts(P, D, g + 8, n);
+  }
   // this warp's k-steps of the operand: one bulk copy from L2 (the producers' stores were made
   // visible by the grid barrier; the proxy fence orders that observation before the async read)
   const uint32_t sbar = smem_u32(&M.sbar[warp]);
@@ -586,13 +608,18 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
         resid_tile<T16, LO>(P, D, tile, l, c);
       } else {
         const int n = tile * 8 + 2 * tt;
+        const bool first = u0 == 0 && idx == tid;  // the pass whose constants were loaded ahead
         if (gg < T) {
           const float inv = D.in_fix ? M.inv_rms[gg] : 1.f;
-          epilogue_pair<T16, LO>(P, D, M, gg, n, c[0] * inv, c[1] * inv);
+          QkvConsts qc = qc0;
+          if (D.epi == EPI_F_QKV && !first) qc = qkv_consts(P, D, gg, n);
+          epilogue_pair<T16, LO>(P, D, M, gg, n, c[0] * inv, c[1] * inv, qc);
         }
         if (T16 && gg + 8 < T) {
           const float inv = D.in_fix ? M.inv_rms[gg + 8] : 1.f;
-          epilogue_pair<T16, LO>(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv);
+          QkvConsts qc = qc1;
+          if (D.epi == EPI_F_QKV && !first) qc = qkv_consts(P, D, gg + 8, n);
+          epilogue_pair<T16, LO>(P, D, M, gg + 8, n, c[NACC - 2] * inv, c[NACC - 1] * inv, qc);
         }
       }
     }
