@@ -424,10 +424,12 @@ struct ResidAdds {
 };
 template <bool T16, bool LO>
 __device__ __forceinline__ void resid_issue(const FastParams& P, const PhaseDesc& D, int tile, int lane,
-                                            const float* c, ResidAdds<T16, LO>& A) {
+                                            const float* c, ResidAdds<T16, LO>& A, const float2* gn_ready = nullptr) {
   constexpr int NH = T16 ? 2 : 1;
   const int gg = lane >> 2, tt = lane & 3, n = tile * 8 + 2 * tt, T = P.T;
-  A.gn = __ldg(reinterpret_cast<const float2*>(D.gain_next + n));  // early: a cold load
+  // the gains of the next norm for these two columns: a cold load, taken at the start of the
+  // phase where the caller could
+  A.gn = gn_ready ? *gn_ready : __ldg(reinterpret_cast<const float2*>(D.gain_next + n));
 #pragma unroll
   for (int h = 0; h < NH; ++h) {
     if (gg + 8 * h < T) {
@@ -469,9 +471,9 @@ __device__ __forceinline__ void resid_finish(const FastParams& P, const PhaseDes
 }
 template <bool T16, bool LO>
 __device__ __forceinline__ void resid_tile(const FastParams& P, const PhaseDesc& D, int tile, int lane,
-                                           const float* c) {
+                                           const float* c, const float2* gn_ready = nullptr) {
   ResidAdds<T16, LO> A;
-  resid_issue<T16, LO>(P, D, tile, lane, c, A);
+  resid_issue<T16, LO>(P, D, tile, lane, c, A, gn_ready);
   resid_finish<T16, LO>(P, D, tile, lane, A);
 }
 
@@ -559,6 +561,9 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
     if (row0) qc0 = qkv_consts(P, D, g, n);
     if (row1) qc1 = qkv_consts(P, D, g + 8, n);
   }
+  float2 gn0 = make_float2(0.f, 0.f);  // residual epilogue, first pass: this thread's two gains
+  if (D.epi == EPI_F_RESID && tid < min(FAST_MAXU, cnt_total) * 32)
+    gn0 = __ldg(reinterpret_cast<const float2*>(D.gain_next + M.utile[D.op][warp] * 8 + 2 * (lane & 3)));
   // this warp's k-steps of the operand: one bulk copy from L2 (the producers' stores were made
   // visible by the grid barrier; the proxy fence orders that observation before the async read)
   const uint32_t sbar = smem_u32(&M.sbar[warp]);
@@ -604,11 +609,11 @@ __device__ __forceinline__ void gemm_phase(const FastParams& P, FastMisc& M, uin
         for (int i = 0; i < NACC; ++i) c[i] += src[i];
       }
       const int tile = M.utile[D.op][u0 + u];
+      const bool first = u0 == 0 && idx == tid;  // the pass whose constants were loaded ahead
       if (D.epi == EPI_F_RESID) {
-        resid_tile<T16, LO>(P, D, tile, l, c);
+        resid_tile<T16, LO>(P, D, tile, l, c, first ? &gn0 : nullptr);
       } else {
         const int n = tile * 8 + 2 * tt;
-        const bool first = u0 == 0 && idx == tid;  // the pass whose constants were loaded ahead
         if (gg < T) {
           const float inv = D.in_fix ? M.inv_rms[gg] : 1.f;
           QkvConsts qc = qc0;
