@@ -216,7 +216,7 @@ __device__ __forceinline__ void trace_mark(const FastParams& P, int& n_trace) {
 // reached `target`.  One thread per CTA arrives (release reduction) and polls (acquire loads).
 // A CTA whose wait ran out raises the failure word next to the base; every poller looks at that
 // word now and then, so all CTAs give up together.  Returns false in that case.
-__device__ __noinline__ bool grid_sync(const FastParams& P, uint32_t target, bool failed) {
+__device__ __forceinline__ bool grid_sync(const FastParams& P, uint32_t target, bool failed) {
   const int bad_in = __syncthreads_or(failed ? 1 : 0);
   bool ok = bad_in == 0;
   if (threadIdx.x == 0) {
