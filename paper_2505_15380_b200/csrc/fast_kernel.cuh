@@ -498,7 +498,8 @@ __device__ __forceinline__ void mma_round(Ring& r, int lane, uint32_t af_lane, i
     const uint32_t wb = r.ring + r.slot * FAST_SLOT_BYTES + lane * 8;
 #pragma unroll
     for (int i = 0; i < SPC; ++i) {
-      if (SPC == 1 || s + i < s1) {
+      if (SPC > 1 && s + i >= s1) break;  // the last chunk of the slice may hold fewer k-steps
+      {
         uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
         if (row0) load_afrag<LO>(af_lane + (uint32_t)(s + i) * STEP, 0, ahi, alo);
         if (T16 && row1) load_afrag<LO>(af_lane + (uint32_t)(s + i) * STEP + Lay<T16, LO>::WH * 4, 1, ahi, alo);
