@@ -348,9 +348,12 @@ __device__ __forceinline__ void ssq_finish(const SsqLoads& q, const long long* _
     if (row < T) {  // uniform per warp
       long long v = q.v[h];
       for (int wd = lane + 32; wd < nwords; wd += 32) v += __ldcg(ssq + wd * FAST_MAX_T + row);
+      // the words are exact (integer sums), so a fixed shuffle tree over their fp32 values gives
+      // the same result in every run; half the instructions of a 64-bit tree
+      float f = fix_to_float(v);
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);  // integer: any order
-      if (lane == 0) M.inv_rms[row] = rsqrtf(fix_to_float(v) / (float)K + eps);
+      for (int o = 16; o > 0; o >>= 1) f += __shfl_xor_sync(0xffffffffu, f, o);
+      if (lane == 0) M.inv_rms[row] = rsqrtf(f / (float)K + eps);
     }
   }
 }
