@@ -157,6 +157,8 @@ struct Ring {
   uint32_t nslot;
   uint32_t outstanding;     // copies issued and not yet waited for
   bool dead;                // a bounded wait ran out
+  uint64_t policy;          // L2 eviction priority of the stream's copies, made once (making it
+                            // anew for every copy cost 11 us per forward)
 };
 
 // Tiles of the next chunk to request (0: the stream is exhausted).
@@ -175,7 +177,7 @@ __device__ __forceinline__ void ring_request(Ring& r, uint32_t slot, int lane) {
     if (lane == 0) {
       const uint32_t bar = r.bars + slot * 8;
       mbar_expect_tx(bar, n * FAST_TILE_BYTES);
-      bulk_g2s_hint(r.ring + slot * FAST_SLOT_BYTES, r.src, n * FAST_TILE_BYTES, bar, policy_evict_first());
+      bulk_g2s_hint(r.ring + slot * FAST_SLOT_BYTES, r.src, n * FAST_TILE_BYTES, bar, r.policy);
     }
     r.src += n * FAST_TILE_BYTES;
     r.outstanding++;
@@ -1090,6 +1092,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   ring.nslot = (uint32_t)P.nslot;
   ring.outstanding = 0;
   ring.dead = false;
+  ring.policy = policy_evict_first();
   uint32_t stage_parity = 0;
   if (lane == 0) {
     mbar_init(smem_u32(&M.sbar[warp]), 1);
