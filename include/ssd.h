@@ -60,9 +60,11 @@ enum {
 /* bits of the device status word (ssd_last_status) */
 enum {
   SSD_STATUS_KV_OVERFLOW = 1, /* len + rows > capacity: rows beyond capacity were not written */
-  SSD_STATUS_BAD_TOKEN = 2,   /* a token id outside the embedding table was clamped */
+  SSD_STATUS_BAD_TOKEN = 2,   /* a token id outside the embedding table was clamped; a draft token
+                                 outside the vocabulary was rejected; ssd_kv_commit was handed an
+                                 accepted length outside 0..max_gamma and left that stream alone */
   SSD_STATUS_NONFINITE = 4,   /* a logit row held NaN/Inf */
-  SSD_STATUS_BAD_PROB = 8,    /* a draft probability p_i(x_i) was negative or not finite */
+  SSD_STATUS_BAD_PROB = 8,    /* a draft probability p_i(x_i) was negative or not finite: rejected */
   SSD_STATUS_TIMEOUT = 16     /* a bounded wait inside a kernel ran out; the streams object refuses
                                  further small-batch launches until it is created anew */
 };
@@ -220,7 +222,10 @@ int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t
  * looks up the array's address (cudaGetSymbolAddress, with that device current); make that first
  * call before starting any stream capture.  All calls share the one array, which keeps the last
  * call's contents: the per-stream counters are cleared on `stream` at the start of each call, and
- * two calls that overlap on the GPU (different streams, or different threads) race on it. */
+ * two calls that overlap on the GPU (different streams, or different threads) race on it.
+ * This call reports no device status bits (there is no streams object to hold them): a draft token
+ * outside [0, vocab) or a draft probability that is negative or not finite is treated as rejected
+ * at its position, so accepted_len stops in front of it and next_token is the resample there. */
 int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_draft_tokens,
                        const float* dev_draft_probs, const float* dev_uniforms,
                        const ssd_verify_params* params, int32_t batch, int32_t vocab,
@@ -239,10 +244,39 @@ int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8
 int ssd_fast_pack_roundtrip_host(const ssd_model_config* cfg, int32_t n_cta, const void* host_weights,
                                  size_t nbytes, void* host_out, int64_t* bad_chunks);
 
+/* ---- the tensor-core projection kernel alone (tests of the batched forward's building block) -- */
+
+/* One projection of the decoder (Sec. 3.1; Eq. 4) as the batched forward runs it on the tcgen05
+ * tensor cores: acc[t, r] = sum_k x[t, k] * w[r, k] for M token rows (17..512 are what the forward
+ * uses; 1..512 accepted) and n_rows weight rows, K a multiple of 8.
+ *   dev_w   bf16 [n_rows, K] row-major;  dev_x  float [M, K];  both device pointers, read-only.
+ *   dev_scratch  device buffer of at least ssd_tc_gemm_scratch_bytes(M, n_rows, K) bytes (256-byte
+ *                aligned), zero-filled by the caller: receives the packed operands.
+ *   epilogue 0: K split `ksplit` ways; dev_out float [ksplit, Mpad, ld] receives one slab of
+ *               partial sums per K slice (Mpad = M rounded up to 16, ld = n_rows rounded up to
+ *               128): element [s, t, r].  Their sum over s is acc.
+ *   epilogue 1: ksplit must be 1; dev_out float [M, n_rows] = acc (the LM-head form).
+ *   epilogue 2: ksplit must be 1; weight rows are (gate_j, up_j) pairs; dev_out receives
+ *               SiLU(gate_j) * up_j as a packed operand of n_rows / 2 columns:
+ *               byte(part, t, j) = (j / 16) * Mpad * 64 + part * Mpad * 32 + ((j / 8) % 2) * Mpad * 16
+ *                                  + t * 16 + (j % 8) * 2,  part 0 = bf16 leading part of the
+ *               value, part 1 = bf16 of the remainder ((n_rows / 2 rounded up to 16) * Mpad * 4 bytes).
+ * Enqueues on `stream`; SSD_ERR_BAD_PARAM for sizes outside the ranges above. */
+size_t ssd_tc_gemm_scratch_bytes(int32_t M, int32_t n_rows, int32_t K);
+int ssd_tc_gemm_check(const void* dev_w, const float* dev_x, int32_t M, int32_t n_rows, int32_t K,
+                      int32_t ksplit, int32_t epilogue, void* dev_scratch, size_t scratch_bytes,
+                      void* dev_out, int32_t* dev_status, void* stream);
+
 /* ---- diagnostics ------------------------------------------------------------------------- */
 
 /* Reads and clears the device status word (SSD_STATUS_* bits).  Synchronises `stream`. */
 int ssd_last_status(ssd_streams* s, int32_t* status, void* stream);
+/* Host-made failure for tests of the error path: marks the streams object exactly as a bounded
+ * wait that ran out inside the persistent kernel marks it.  Every later small-batch forward on
+ * these streams returns at once without touching its outputs and raises SSD_STATUS_TIMEOUT; the
+ * object must be created anew to be used again.  No kernel is made to wait or fail for this.
+ * Synchronises `stream`. */
+int ssd_streams_inject_failure(ssd_streams* s, void* stream);
 /* Number of kernels this library has enqueued in this process so far (all handles). */
 uint64_t ssd_kernel_launch_count(void);
 /* Text of the last CUDA error seen by this library on this thread ("" if none). */

@@ -24,7 +24,9 @@ EXPORTS = [
     "ssd_streams_set_trace", "ssd_forward", "ssd_fast_plan_host",
     "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
-    "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_kernel_launch_count",
+    "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_streams_inject_failure",
+    "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check",
+    "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
 
@@ -83,6 +85,10 @@ def lib() -> ctypes.CDLL:
     L.ssd_kv_commit.argtypes = [vp, vp, vp, vp]
     L.ssd_kv_restore.argtypes = [vp, vp, vp, vp]
     L.ssd_accept_noalloc.argtypes = [vp, vp, vp, vp, parp, i32, i32, vp, vp, vp]
+    L.ssd_streams_inject_failure.argtypes = [vp, vp]
+    L.ssd_tc_gemm_scratch_bytes.restype = sz
+    L.ssd_tc_gemm_scratch_bytes.argtypes = [i32, i32, i32]
+    L.ssd_tc_gemm_check.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, sz, vp, vp, vp]
     L.ssd_kernel_launch_count.restype = ctypes.c_uint64
     L.ssd_kernel_launch_count.argtypes = []
     L.ssd_last_status.argtypes = [vp, ctypes.POINTER(i32), vp]
@@ -221,6 +227,10 @@ class Streams:
                                           _stream_ptr(stream)))
         return a, p
 
+    def inject_failure(self, stream=None) -> None:
+        """Marks the streams object as failed, as a timed-out wait in the persistent kernel would."""
+        check(lib().ssd_streams_inject_failure(self.handle, _stream_ptr(stream)))
+
     def last_status(self, stream=None) -> int:
         v = ctypes.c_int32(0)
         check(lib().ssd_last_status(self.handle, ctypes.byref(v), _stream_ptr(stream)))
@@ -307,3 +317,32 @@ def accept_noalloc(logits: torch.Tensor, draft_tokens: torch.Tensor, draft_probs
                                        draft_probs.data_ptr(), uniforms.data_ptr(),
                                        ctypes.byref(params), B, V, accepted_len.data_ptr(),
                                        next_token.data_ptr(), _stream_ptr(stream)))
+
+
+def tc_gemm_check(w: torch.Tensor, x: torch.Tensor, ksplit: int, epilogue: int, stream=None):
+    """ssd_tc_gemm_check: one tensor-core projection on caller data.  w bf16 [n_rows, K], x float32
+    [M, K], both CUDA.  Returns (raw output tensor, status word): float32 [ksplit, Mpad, ld] partial
+    sums (epilogue 0), float32 [M, n_rows] (1), or the packed SiLU(gate) * up operand as uint8 (2)."""
+    _require_cuda()
+    L = lib()
+    assert w.dtype == torch.bfloat16 and x.dtype == torch.float32 and w.is_cuda and x.is_cuda
+    assert w.is_contiguous() and x.is_contiguous() and w.shape[1] == x.shape[1]
+    n_rows, K = w.shape
+    M = x.shape[0]
+    Mpad, ld = (M + 15) // 16 * 16, (n_rows + 127) // 128 * 128
+    need = L.ssd_tc_gemm_scratch_bytes(M, n_rows, K)
+    if need == 0:
+        raise SsdError("sizes outside the range of the tensor-core projection")
+    with torch.cuda.device(w.device):
+        scratch = torch.zeros(need, dtype=torch.uint8, device=w.device)
+        status = torch.zeros(1, dtype=torch.int32, device=w.device)
+        if epilogue == 0:
+            out = torch.zeros((ksplit, Mpad, ld), dtype=torch.float32, device=w.device)
+        elif epilogue == 1:
+            out = torch.zeros((M, n_rows), dtype=torch.float32, device=w.device)
+        else:
+            out = torch.zeros(((n_rows // 2 + 15) // 16) * Mpad * 64, dtype=torch.uint8, device=w.device)
+        check(L.ssd_tc_gemm_check(w.data_ptr(), x.data_ptr(), M, n_rows, K, ksplit, epilogue,
+                                  scratch.data_ptr(), need, out.data_ptr(), status.data_ptr(),
+                                  _stream_ptr(stream)))
+    return out, status

@@ -20,7 +20,6 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-FLAGS += os.environ.get("SSD_NVCC_EXTRA", "").split()   # extra nvcc flags, e.g. -DSSD_FAST_WARPS=16
 
 
 def _sources():

@@ -9,6 +9,7 @@
 
 #include "fast.h"
 #include "kernels.h"
+#include "tc.h"
 
 using namespace ssd;
 
@@ -53,6 +54,10 @@ struct ArenaPlan {
   bool fast;
   size_t f_stream, f_stream_off, f_chunks, f_chunk_cnt, f_unit_cnt, f_unit_off, f_unit_tile, f_bias,
       f_gains;
+  // weights packed for the tensor-core projections of batched forwards (bf16 models only)
+  bool tc;
+  std::vector<LayerOff> tc_layers;  // w_qkv, w_o, w_gu, w_d used
+  size_t tc_head;
 };
 
 // CTAs of the persistent kernel: one per SM of the current device (148 when none is present, the
@@ -105,6 +110,17 @@ ArenaPlan plan_arena(const ssd_model_config& c, const FastPlan* fp = nullptr) {
     p.f_bias = take((size_t)c.n_layers * nq * 4);
     p.f_gains = take(((size_t)c.n_layers * 2 + 1) * d * 4);
   }
+  p.tc = c.weight_dtype == 1;
+  if (p.tc) {
+    p.tc_layers.resize(c.n_layers);
+    for (auto& L : p.tc_layers) {
+      L.w_qkv = take(tc_weight_bytes((int)(qd + 2 * kvd), (int)d));
+      L.w_o = take(tc_weight_bytes((int)d, (int)qd));
+      L.w_gu = take(tc_weight_bytes((int)(2 * F), (int)d));
+      L.w_d = take(tc_weight_bytes((int)d, (int)F));
+    }
+    p.tc_head = take(tc_weight_bytes(c.vocab_out, (int)d));
+  }
   p.total = off;
   return p;
 }
@@ -121,6 +137,7 @@ struct WsPlan {
   size_t h, qkv, qrot, rope_cs, part, logits, row_stats, xn, attn_out, act;
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
   size_t hfix, flags, epoch_base, xa, xb, xd, xq, ssq_a, ssq_b;
+  size_t tc_xa, tc_xattn, tc_xact, tc_part;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -165,6 +182,21 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.ssq_b = take((d / 64 + 1) * FAST_MAX_T * 8);
   p.flags = take(64);
   p.epoch_base = take(2 * 4);
+  p.tc_xa = p.tc_xattn = p.tc_xact = p.tc_part = 0;
+  if (c.weight_dtype == 1 && M > FAST_MAX_T && M <= TC_MAX_ROWS) {
+    const int Mpad = tc_round16((int)M), n_sm = fast_cta_count();
+    p.tc_xa = take(tc_act_bytes(Mpad, (int)d));
+    p.tc_xattn = take(tc_act_bytes(Mpad, (int)qd));
+    p.tc_xact = take(tc_act_bytes(Mpad, (int)F));
+    size_t part = 0;
+    const int rows[3] = {(int)(qd + 2 * kvd), (int)d, (int)d}, ks[3] = {(int)d, (int)qd, (int)F};
+    for (int i = 0; i < 3; ++i) {
+      const size_t tiles = (rows[i] + TC_TILE_ROWS - 1) / TC_TILE_ROWS;
+      const size_t b = (size_t)tc_ksplit(rows[i], ks[i], n_sm) * Mpad * tiles * TC_TILE_ROWS * 4;
+      part = b > part ? b : part;
+    }
+    p.tc_part = take(part);
+  }
   p.total = off;
   return p;
 }
@@ -249,8 +281,68 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   return SSD_OK;
 }
 
+// Forwards of more than FAST_MAX_T rows over a bf16 model: projections on the tcgen05 tensor cores
+// (each weight byte read once), attention on the warp-level tensor-core instruction.
+bool use_tc(const ssd_model* m, const ssd_streams* s, RowMap rm) {
+  const int M = rm.nb * rm.R;
+  return m->tc.enabled && s->path == 0 && s->tc_part && M > FAST_MAX_T && M <= TC_MAX_ROWS && M <= s->max_rows;
+}
+
+int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cudaStream_t st) {
+  const ssd_model_config& c = m->cfg;
+  const int M = rm.nb * rm.R, Mpad = tc_round16(M), d = c.d_model;
+  const int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn, nq = qd + 2 * kvd;
+  const int n_sm = m->tc.n_sm;
+  auto ld_of = [](int rows) { return (rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS * TC_TILE_ROWS; };
+  const int ks_qkv = tc_ksplit(nq, d, n_sm), ks_o = tc_ksplit(d, qd, n_sm), ks_d = tc_ksplit(d, F, n_sm);
+  // key splits of the attention: enough CTAs for two to three waves, whole 64-key tiles each
+  const int G = c.n_q_heads / c.n_kv_heads, rowgroups = (G * rm.R + 63) / 64;
+  long long kps = ((long long)s->cap * rm.nb * c.n_kv_heads * rowgroups * 2 + 5LL * n_sm - 1) / (5LL * n_sm);
+  kps = (kps + 63) / 64 * 64;
+  if (kps < 64) kps = 64;
+  const int nsplit = (int)((s->cap + kps - 1) / kps);
+  launch_embed(1, m->embed, c.vocab_out + c.vocab_text, d, s->row_ids, M, s->h, s->status, st);
+  launch_rope_table(s->len, rm, m->inv_freq, c.head_dim / 2, s->rope_cs, st);
+  const float* part = nullptr;
+  int nsp = 0, ldp = 0;
+  TcGemm g{};
+  g.M = M;
+  g.status = s->status;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerW& w = m->layers[l];
+    const ssd_tc_layer& t = m->tc.layers[l];
+    bf16* kv_layer = (bf16*)(s->kv + (size_t)l * s->kv_layer_elems * s->el);
+    launch_tc_norm_pack(s->h, part, nsp, ldp, M, d, (const bf16*)w.norm1, c.rms_eps, s->tc_xa, st);
+    g.w = t.w_qkv; g.a = s->tc_xa; g.n_rows = nq; g.K = d; g.ksplit = ks_qkv; g.epi = TC_EPI_PARTIAL; g.part = s->tc_part;
+    SSD_CUDA(launch_tc_gemm(g, st));
+    launch_tc_qkv_post(s->tc_part, ks_qkv, ld_of(nq), Mpad, (const bf16*)w.b_qkv, s->rope_cs, s->qrot, kv_layer,
+                       s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim, s->status, st);
+    SSD_CUDA(launch_tc_attention(s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, st));
+    g.w = t.w_o; g.a = s->tc_xattn; g.n_rows = d; g.K = qd; g.ksplit = ks_o;
+    SSD_CUDA(launch_tc_gemm(g, st));
+    launch_tc_norm_pack(s->h, s->tc_part, ks_o, ld_of(d), M, d, (const bf16*)w.norm2, c.rms_eps, s->tc_xa, st);
+    g.w = t.w_gu; g.a = s->tc_xa; g.n_rows = 2 * F; g.K = d; g.ksplit = 1; g.epi = TC_EPI_SWIGLU; g.act_out = s->tc_xact;
+    SSD_CUDA(launch_tc_gemm(g, st));
+    g.w = t.w_d; g.a = s->tc_xact; g.n_rows = d; g.K = F; g.ksplit = ks_d; g.epi = TC_EPI_PARTIAL;
+    SSD_CUDA(launch_tc_gemm(g, st));
+    part = s->tc_part;
+    nsp = ks_d;
+    ldp = ld_of(d);
+  }
+  if (logits_out) {
+    launch_tc_norm_pack(s->h, part, nsp, ldp, M, d, (const bf16*)m->norm_f, c.rms_eps, s->tc_xa, st);
+    g.w = m->tc.head; g.a = s->tc_xa; g.n_rows = c.vocab_out; g.K = d; g.ksplit = 1; g.epi = TC_EPI_STORE;
+    g.out = logits_out; g.ldo = c.vocab_out;
+    SSD_CUDA(launch_tc_gemm(g, st));
+  }
+  SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
 int forward(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cudaStream_t st) {
   if (use_fast(m, s, rm)) return forward_fast(m, s, rm, s->row_ids, nullptr, logits_out, st);
+  if (use_tc(m, s, rm)) return forward_tc(m, s, rm, logits_out, st);
   const ssd_model_config& c = m->cfg;
   const int dt = c.weight_dtype, M = rm.nb * rm.R, d = c.d_model;
   const int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn;
@@ -410,6 +502,27 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
     if (down_w > f.max_stage_k) f.max_stage_k = down_w;
     f.enabled = f.max_units <= FAST_MAX_UNITS && fplan.max_chunks <= FAST_MAX_CHUNKS;
   }
+  if (p.tc && e == cudaSuccess) {
+    // third arrangement of the projection weights: 128-row tiles in the tensor cores' canonical
+    // shared-memory layout, made on the device from the row-major copy
+    ssd_tc_model& t = m->tc;
+    t.n_sm = fast_cta_count();
+    t.layers.resize(c.n_layers);
+    auto pack = [&](const void* src, int rows, int K, size_t dst_off) {
+      if (e == cudaSuccess) e = tc_pack_weights((const bf16*)src, rows, K, (uint8_t*)(A + dst_off), 0);
+      return (const uint8_t*)(A + dst_off);
+    };
+    for (int l = 0; l < c.n_layers; ++l) {
+      const LayerW& w = m->layers[l];
+      const LayerOff& o = p.tc_layers[l];
+      t.layers[l].w_qkv = pack(w.w_qkv, (int)(qd + 2 * kvd), (int)d, o.w_qkv);
+      t.layers[l].w_o = pack(w.w_o, (int)d, (int)qd, o.w_o);
+      t.layers[l].w_gu = pack(w.w_gu, (int)(2 * F), (int)d, o.w_gu);
+      t.layers[l].w_d = pack(w.w_d, (int)d, (int)F, o.w_d);
+    }
+    t.head = pack(m->head, c.vocab_out, (int)d, p.tc_head);
+    t.enabled = e == cudaSuccess;
+  }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete m;
@@ -489,6 +602,10 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->ssq_b = (long long*)(W + p.ssq_b);
   s->flags = (uint32_t*)(W + p.flags);
   s->epoch_base = (uint32_t*)(W + p.epoch_base);
+  s->tc_xa = p.tc_part ? (uint8_t*)(W + p.tc_xa) : nullptr;
+  s->tc_xattn = p.tc_part ? (uint8_t*)(W + p.tc_xattn) : nullptr;
+  s->tc_xact = p.tc_part ? (uint8_t*)(W + p.tc_xact) : nullptr;
+  s->tc_part = p.tc_part ? (float*)(W + p.tc_part) : nullptr;
   s->path = 0;
   s->split_act = 1;
   s->trace = nullptr;
@@ -677,7 +794,7 @@ int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_token
 int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
                   void* stream) {
   if (!s || !dev_accepted_len || !dev_next_token) return SSD_ERR_NULL;
-  launch_kv_commit(s->len, s->pending, dev_accepted_len, dev_next_token, s->B, s->cap, s->status,
+  launch_kv_commit(s->len, s->pending, dev_accepted_len, dev_next_token, s->B, s->cap, s->max_gamma, s->status,
                    (cudaStream_t)stream);
   SSD_CUDA(cudaGetLastError());
   return SSD_OK;
@@ -690,10 +807,13 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
   if (!target || !s || !host_draft_tokens || !host_draft_probs || !host_uniforms ||
       !host_accepted_len || !host_next_token)
     return SSD_ERR_NULL;
+  // every check ssd_verify makes comes first: nothing may be enqueued on an error, and the
+  // staging buffers were sized from the streams' own shape
+  if (!same_shape(target->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
   int rc = params_ok(s, params, true);
   if (rc != SSD_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t B = s->B, g = params->gamma, V = target->cfg.vocab_out;
+  const size_t B = s->B, g = params->gamma, V = s->cfg.vocab_out;
   SSD_CUDA(cudaMemcpyAsync(s->st_tokens, host_draft_tokens, B * g * 4, cudaMemcpyHostToDevice, st));
   SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, st));
   SSD_CUDA(cudaMemcpyAsync(s->st_uni, host_uniforms, B * (g + 1) * 2 * 4, cudaMemcpyHostToDevice, st));
@@ -713,6 +833,52 @@ int ssd_last_status(ssd_streams* s, int32_t* status, void* stream) {
   cudaStream_t st = (cudaStream_t)stream;
   SSD_CUDA(cudaMemcpyAsync(status, s->status, 4, cudaMemcpyDeviceToHost, st));
   SSD_CUDA(cudaMemsetAsync(s->status, 0, 4, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+size_t ssd_tc_gemm_scratch_bytes(int32_t M, int32_t n_rows, int32_t K) {
+  if (M < 1 || M > TC_MAX_ROWS || n_rows < 1 || K < 8 || (K & 7)) return 0;
+  return align_up(tc_weight_bytes(n_rows, K)) + align_up(tc_act_bytes(tc_round16(M), K));
+}
+
+int ssd_tc_gemm_check(const void* dev_w, const float* dev_x, int32_t M, int32_t n_rows, int32_t K,
+                      int32_t ksplit, int32_t epilogue, void* dev_scratch, size_t scratch_bytes,
+                      void* dev_out, int32_t* dev_status, void* stream) {
+  if (!dev_w || !dev_x || !dev_scratch || !dev_out || !dev_status) return SSD_ERR_NULL;
+  const size_t need = ssd_tc_gemm_scratch_bytes(M, n_rows, K);
+  if (need == 0 || ksplit < 1 || ksplit > (K + 15) / 16 || epilogue < 0 || epilogue > 2 ||
+      (epilogue != TC_EPI_PARTIAL && ksplit != 1) || (epilogue == TC_EPI_SWIGLU && (n_rows & 1)))
+    return SSD_ERR_BAD_PARAM;
+  if ((uintptr_t)dev_scratch & 255) return SSD_ERR_MISALIGNED;
+  if (scratch_bytes < need) return SSD_ERR_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* wp = (uint8_t*)dev_scratch;
+  uint8_t* ap = wp + align_up(tc_weight_bytes(n_rows, K));
+  SSD_CUDA(tc_pack_weights((const bf16*)dev_w, n_rows, K, wp, st));
+  launch_tc_pack_rows(dev_x, M, K, ap, st);
+  TcGemm g{};
+  g.w = wp;
+  g.a = ap;
+  g.n_rows = n_rows;
+  g.K = K;
+  g.M = M;
+  g.ksplit = ksplit;
+  g.epi = epilogue;
+  g.part = (float*)dev_out;
+  g.out = (float*)dev_out;
+  g.ldo = n_rows;
+  g.act_out = (uint8_t*)dev_out;
+  g.status = dev_status;
+  SSD_CUDA(launch_tc_gemm(g, st));
+  return SSD_OK;
+}
+
+int ssd_streams_inject_failure(ssd_streams* s, void* stream) {
+  if (!s) return SSD_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint32_t one = 1u;  // the sticky failure word next to the barrier's launch base
+  SSD_CUDA(cudaMemcpyAsync(s->epoch_base + 1, &one, 4, cudaMemcpyHostToDevice, st));
   SSD_CUDA(cudaStreamSynchronize(st));
   return SSD_OK;
 }

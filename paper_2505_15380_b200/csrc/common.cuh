@@ -85,6 +85,17 @@ struct ssd_fast_model {
   int n_cta = 0, max_units = 0, down_split = 1, o_split = 1, max_stage_k = 0;
 };
 
+// Device-side view of the weights packed for the tensor-core projections of batched forwards (tc.h).
+struct ssd_tc_layer {
+  const uint8_t *w_qkv, *w_o, *w_gu, *w_d;
+};
+struct ssd_tc_model {
+  bool enabled = false;
+  std::vector<ssd_tc_layer> layers;
+  const uint8_t* head = nullptr;
+  int n_sm = 148;  // SMs of the device the model was created on: sizes the K splits
+};
+
 struct ssd_model {
   ssd_model_config cfg;
   int el;  // bytes per weight element
@@ -94,6 +105,7 @@ struct ssd_model {
   const void *norm_f, *head;
   const double* inv_freq;  // [head_dim / 2]
   ssd_fast_model fast;
+  ssd_tc_model tc;
 };
 
 struct ssd_streams {
@@ -116,6 +128,10 @@ struct ssd_streams {
   uint32_t *xa, *xb, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
   long long *ssq_a, *ssq_b;
   uint32_t *flags, *epoch_base;
+  // batched tensor-core forward: packed operands (inputs of QKV / gate-up / head, of O, of down)
+  // and the partial sums of the K-split projections
+  uint8_t *tc_xa, *tc_xattn, *tc_xact;
+  float* tc_part;
   int split_act;     // persistent kernel: activations as bf16 hi + lo pairs (1) or plain bf16 (0)
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)

@@ -127,7 +127,7 @@ __global__ void qkv_post_kernel(const float* __restrict__ qkv, const float* __re
     qrot[(size_t)m * Hq * hd + hh * hd + j] = (x1 * co - x2 * si) * scale;
     qrot[(size_t)m * Hq * hd + hh * hd + j + half] = (x2 * co + x1 * si) * scale;
   }
-  if (pos >= cap) {
+  if (pos < 0 || pos >= cap) {  // never write outside the stream's slice of the cache
     if (threadIdx.x == 0) atomicOr(status, SSD_STATUS_KV_OVERFLOW);
     return;
   }

@@ -18,25 +18,16 @@
 
 namespace ssd {
 
-#ifndef SSD_FAST_WARPS
-#define SSD_FAST_WARPS 8
-#endif
-constexpr int FAST_WARPS = SSD_FAST_WARPS;  // warps per CTA; they split K of every projection
+constexpr int FAST_WARPS = 8;  // warps per CTA; they split K of every projection
 constexpr int FAST_THREADS = FAST_WARPS * 32;
 constexpr int FAST_TILE_BYTES = 256;  // one operand tile: 8 weight rows x 16 k, bf16
-#ifndef SSD_FAST_SLOT_TILES
-#define SSD_FAST_SLOT_TILES 20
-#endif
-constexpr int FAST_SLOT_TILES = SSD_FAST_SLOT_TILES;  // a ring slot holds one chunk of at most this many tiles
+constexpr int FAST_SLOT_TILES = 20;  // a ring slot holds one chunk of at most this many tiles
 constexpr int FAST_SLOT_BYTES = FAST_TILE_BYTES * FAST_SLOT_TILES;
 // Chunks of the O projection's stream (runs of a warp's own tiles): a power of two, so that a pair
 // of output tiles with 2, 4 or 8 k-steps each never straddles two chunks.
 constexpr int FAST_O_CHUNK = 16;
 constexpr int FAST_MAX_SLOTS = 8;     // most ring slots per warp (barrier storage)
-#ifndef SSD_FAST_RING_SLOTS
-#define SSD_FAST_RING_SLOTS 3
-#endif
-constexpr int FAST_RING_SLOTS = SSD_FAST_RING_SLOTS;  // ring slots per warp actually used
+constexpr int FAST_RING_SLOTS = 3;    // ring slots per warp actually used
 constexpr int FAST_MAXU = 10;         // output tiles a CTA accumulates at once (one "round")
 constexpr int FAST_MAX_UNITS = 64;    // output tiles per CTA and op (table size in shared memory)
 constexpr int FAST_MAX_CHUNKS = 128;  // chunks per warp: one layer's plus the LM head's

@@ -397,7 +397,7 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
         const int col = (n & ~(hd - 1)) + j;  // q, pre-scaled, as the operand of the score contraction
         write_frag_elem<T16, LO>(P.xq, tok, col, o1 * D.qscale);
         write_frag_elem<T16, LO>(P.xq, tok, col + half, o2 * D.qscale);
-      } else if (pos < P.cap) {
+      } else if (pos >= 0 && pos < P.cap) {
         const int gk = (n - qd) >> hs;
         bf16* kdst = D.kv_layer + (((size_t)stream * 2 + 0) * P.Hkv + gk) * (size_t)P.cap * hd + (size_t)pos * hd;
         kdst[j] = __float2bfloat16_rn(o1);
@@ -405,7 +405,7 @@ __device__ __forceinline__ void epilogue_pair(const FastParams& P, const PhaseDe
       } else {
         atomicOr(P.status, SSD_STATUS_KV_OVERFLOW);
       }
-    } else if (pos < P.cap) {
+    } else if (pos >= 0 && pos < P.cap) {
       const int nn = n - qd - kvd, gk = nn >> hs, jj = nn & (hd - 1);
       bf16* vdst = D.kv_layer + (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * hd + (size_t)pos * hd;
       *reinterpret_cast<__nv_bfloat162*>(vdst + jj) = __floats2bfloat162_rn(x1, x2);
@@ -1145,7 +1145,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   trace_mark<TRACE>(P, n_trace);
   bool ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, false);
   trace_mark<TRACE>(P, n_trace);
-  // every CTA has read the base by now: publish the next launch's (this launch arrives 1 + 5 L times)
+  // every CTA has read the base by now: publish the next launch's (this launch arrives 1 + 4 L times)
   if (ok && cta == 0 && tid == 0)
     st_release_u32(P.epoch_base, epoch_base + (uint32_t)(1 + 4 * P.L) * (uint32_t)P.m.n_cta);
 

@@ -57,6 +57,7 @@ cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, cons
                                  float* out_prob_row, int32_t* pending, int32_t* status,
                                  cudaStream_t st);
 void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_len,
-                      const int32_t* next_token, int B, int cap, int32_t* status, cudaStream_t st);
+                      const int32_t* next_token, int B, int cap, int max_gamma, int32_t* status,
+                      cudaStream_t st);
 
 }  // namespace ssd

@@ -208,18 +208,20 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
     if (r < gamma) {  // Eq. 5: accept x_i iff r_i < min(1, q_i(x_i) / p_i(x_i)) + beta
       int x = draft_tokens[b * gamma + r];
       float qx = 0.f, px = 0.f;
+      bool valid = true;  // a draft token or probability that cannot be one is rejected, never accepted
       if (x < 0 || x >= V) {
         atomicOr(status, SSD_STATUS_BAD_TOKEN);
+        valid = false;
       } else {
         if (is_kept(z[x], x, st)) qx = expf(z[x] - st.zmax) / st.sum;
         px = draft_probs[((size_t)b * gamma + r) * V + x];
         if (!(px >= 0.f) || !isfinite(px)) {
           atomicOr(status, SSD_STATUS_BAD_PROB);
-          px = 0.f;
+          valid = false;
         }
       }
       float ratio = px <= qx ? 1.f : qx / px;
-      flag = uniforms[((size_t)b * R + r) * 2] < ratio + beta;
+      flag = valid && uniforms[((size_t)b * R + r) * 2] < ratio + beta;
     }
     float* rs = row_stats + ((size_t)b * R + r) * 4;
     rs[0] = st.zmax;
@@ -357,10 +359,16 @@ cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, cons
 
 // "Append to T_in" (Algorithm 1): the prefix grows by the k accepted tokens plus the new one.
 __global__ void kv_commit_kernel(int32_t* len, int32_t* pending, const int32_t* accepted_len,
-                                 const int32_t* next_token, int B, int cap, int32_t* status) {
+                                 const int32_t* next_token, int B, int cap, int max_gamma,
+                                 int32_t* status) {
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
-  int nl = len[b] + 1 + accepted_len[b];
+  const int k = accepted_len[b];
+  if (k < 0 || k > max_gamma) {  // not an accepted length: the stream stays as it is
+    atomicOr(status, SSD_STATUS_BAD_TOKEN);
+    return;
+  }
+  int nl = max(len[b], 0) + 1 + k;
   if (nl > cap) {
     atomicOr(status, SSD_STATUS_KV_OVERFLOW);
     nl = cap;
@@ -370,9 +378,10 @@ __global__ void kv_commit_kernel(int32_t* len, int32_t* pending, const int32_t* 
 }
 
 void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_len,
-                      const int32_t* next_token, int B, int cap, int32_t* status, cudaStream_t st) {
+                      const int32_t* next_token, int B, int cap, int max_gamma, int32_t* status,
+                      cudaStream_t st) {
   kv_commit_kernel<<<(B + 127) / 128, 128, 0, st>>>(len, pending, accepted_len, next_token, B, cap,
-                                                    status);
+                                                    max_gamma, status);
   count_launch();
 }
 

@@ -1,0 +1,102 @@
+// Batched verify forward (Eq. 4 for more than 16 rows: many streams, or a prefill chunk) on the
+// 5th-generation tensor cores: declarations shared by the tcgen05 projection kernel (tc_gemm.cu),
+// the row-wise kernels around it (tc_rows.cu), the batched attention (tc_attention.cu) and the
+// host code that strings them together (api.cu).
+//
+// Projections run "swapped": D[weight row, token] = sum_k W[row, k] * X[token, k].  A CTA owns a
+// tile of 128 weight rows - the M of one tcgen05.mma, so a tile's accumulator fills the 128 lanes
+// of tensor memory - and all tokens (the instruction's N, up to 256 per instruction, more as
+// several column ranges of the same accumulator).  Weights are therefore read from HBM exactly
+// once per forward, whatever the number of rows.  Both operands are staged in shared memory by
+// plain bulk copies: weights are packed once, at model creation, and activations are written by
+// their producers, in the layout the instruction's shared-memory descriptors expect, so that no
+// tensor map and no swizzle is involved:
+//
+//   canonical K-major layout without swizzle: a "core matrix" is 8 rows x 16 bytes (8 bf16 along
+//   K), stored as 128 contiguous bytes; the descriptor gives the byte distance between core
+//   matrices that are neighbours along K ("leading" offset) and along the rows ("stride" offset).
+//
+//   weights, per (tile of 128 rows, k-step of 16 columns) one 4 KB block:
+//       byte(r, k) = (k / 8) * 2048 + r * 16 + (k % 8) * 2           leading 2048, stride 128
+//   activations (Mpad token rows, a multiple of 16), per k-step one block of Mpad * 64 bytes:
+//       byte(part, t, k) = part * Mpad * 32 + (k / 8) * Mpad * 16 + t * 16 + (k % 8) * 2
+//   with part 0 = bf16 leading part of the fp32 activation, part 1 = bf16 of the remainder: the
+//   tensor cores multiply both with the exact bf16 weights into one fp32 accumulator, so products
+//   are exact to ~2^-17 relative, as in the small-batch kernel.
+//
+// K is split across CTAs where a projection has too few row tiles to occupy the GPU; the partial
+// sums go to a workspace and the row-wise kernel that consumes the projection adds them in a
+// fixed order (bit-reproducible, no atomics).
+#pragma once
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace ssd {
+
+constexpr int TC_TILE_ROWS = 128;                 // weight rows per tile = M of the MMA
+constexpr int TC_WBLOCK = TC_TILE_ROWS * 16 * 2;  // bytes of one (tile, k-step) weight block
+constexpr int TC_MAX_ROWS = 512;                  // token rows per forward (tensor-memory columns)
+constexpr int TC_THREADS = 192;                   // copy warp, MMA warp, four epilogue warps
+
+enum TcEpilogue {
+  TC_EPI_PARTIAL = 0,  // part[split][token][row] = acc                (summed by the consumer)
+  TC_EPI_STORE = 1,    // out[token * ldo + row] = acc                  (LM head -> logits)
+  TC_EPI_SWIGLU = 2    // rows interleaved (gate_j, up_j): packed[token, j] = SiLU(gate) * up
+};
+
+inline int tc_round16(int m) { return (m + 15) / 16 * 16; }
+inline size_t tc_weight_bytes(int n_rows, int K) {
+  return (size_t)((n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS) * ((K + 15) / 16) * TC_WBLOCK;
+}
+// Bytes of a packed activation operand of K columns for Mpad rows.
+inline size_t tc_act_bytes(int Mpad, int K) { return (size_t)((K + 15) / 16) * Mpad * 64; }
+// K slices for a projection of n_rows x K on n_sm SMs: enough CTAs to occupy the GPU, at least
+// four k-steps each.
+inline int tc_ksplit(int n_rows, int K, int n_sm) {
+  const int tiles = (n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS, ks = (K + 15) / 16;
+  int s = n_sm / tiles;
+  if (s > ks / 4) s = ks / 4;
+  return s < 1 ? 1 : s;
+}
+
+struct TcGemm {
+  const uint8_t* w;   // packed weights of the projection
+  const uint8_t* a;   // packed activations
+  int n_rows, K;      // weight rows, input columns
+  int M;              // token rows
+  int ksplit;
+  int epi;
+  float* part;        // TC_EPI_PARTIAL: [ksplit][Mpad][tiles * 128]
+  float* out;         // TC_EPI_STORE
+  int ldo;
+  uint8_t* act_out;   // TC_EPI_SWIGLU: packed operand of n_rows / 2 columns
+  int32_t* status;
+};
+
+// tc_gemm.cu
+cudaError_t tc_pack_weights(const bf16* w_rowmajor, int n_rows, int K, uint8_t* packed, cudaStream_t st);
+cudaError_t tc_unpack_weights(const uint8_t* packed, int n_rows, int K, bf16* w_rowmajor, cudaStream_t st);
+cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st);
+
+// tc_rows.cu
+// h[m, :] += sum of `nsplit` partial projections (part may be null); then the RMS norm of the row
+// times `gain`, written as a packed operand (hi + lo) of d columns.  h_in may differ from h (the
+// first layer reads the embedding rows).
+void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, int M, int d,
+                         const bf16* gain, float eps, uint8_t* apack, cudaStream_t st);
+// Packs fp32 rows x[M, K] as an operand (used by tests of the projection kernel).
+void launch_tc_pack_rows(const float* x, int M, int K, uint8_t* apack, cudaStream_t st);
+// q/k/v = sum of partials + bias; rotary embedding; q (scaled) to qrot [M, Hq * hd] fp32, K and V
+// appended to the cache at len + r.
+void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, const bf16* bias,
+                        const float* cs, float* qrot, bf16* kv_layer, const int32_t* len, RowMap rm,
+                        int cap, int Hq, int Hkv, int hd, int32_t* status, cudaStream_t st);
+
+// tc_attention.cu: verify attention for all streams of the forward (causal inside the block, GQA),
+// split over the keys; the merged result is written as the packed operand of the O projection.
+cudaError_t launch_tc_attention(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm,
+                                int cap, int Hq, int Hkv, int hd, float* part, int nsplit,
+                                int keys_per_split, uint8_t* apack_out, int Mpad, cudaStream_t st);
+
+}  // namespace ssd

@@ -1,0 +1,138 @@
+// Row-wise kernels of the batched verify forward (Eq. 4's decoder pass for more than 16 rows):
+// what sits between the tensor-core projections.  Each consumes a projection's partial sums
+// (one slab per K slice, added here in a fixed order, so results are bit-reproducible) and
+// produces the next projection's input already packed as a tensor-core operand (tc.h).
+#include "kernels.h"
+#include "tc.h"
+
+namespace ssd {
+
+namespace {
+
+// Byte offset of element (part, t, k) of a packed activation operand (tc.h).
+__device__ __forceinline__ size_t act_off(int Mpad, int part, int t, int k) {
+  return (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)part * ((size_t)Mpad * 32) +
+         (size_t)((k >> 3) & 1) * ((size_t)Mpad * 16) + (size_t)t * 16 + (size_t)(k & 7) * 2;
+}
+// Columns (k, k + 1), k even, of token t: bf16 leading parts and remainders.
+__device__ __forceinline__ void store_pair(uint8_t* apack, int Mpad, int t, int k, float x0, float x1) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+  *reinterpret_cast<__nv_bfloat162*>(apack + act_off(Mpad, 0, t, k)) = h;
+  *reinterpret_cast<__nv_bfloat162*>(apack + act_off(Mpad, 1, t, k)) = l;
+}
+
+// One CTA per row.  h[m, :] += sum_s part[s][m][:]; out = h / rms(h) * gain, packed.
+__global__ void __launch_bounds__(256)
+tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
+                    int d, const bf16* __restrict__ gain, float eps, uint8_t* __restrict__ apack) {
+  extern __shared__ float row[];
+  __shared__ float red[8];
+  const int m = blockIdx.x, tid = threadIdx.x;
+  float ss = 0.f;
+  for (int j = tid * 2; j < d; j += 512) {
+    float2 v = *reinterpret_cast<const float2*>(h + (size_t)m * d + j);
+    for (int s = 0; s < nsplit; ++s) {  // fixed order
+      const float2 p = *reinterpret_cast<const float2*>(part + ((size_t)s * Mpad + m) * ld_part + j);
+      v.x += p.x;
+      v.y += p.y;
+    }
+    if (nsplit > 0) *reinterpret_cast<float2*>(h + (size_t)m * d + j) = v;
+    row[j] = v.x;
+    row[j + 1] = v.y;
+    ss += v.x * v.x + v.y * v.y;
+  }
+  ss = warp_sum(ss);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float inv = rsqrtf(tot / (float)d + eps);
+  for (int j = tid * 2; j < d; j += 512) {
+    const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + j));
+    store_pair(apack, Mpad, m, j, row[j] * inv * g.x, row[j + 1] * inv * g.y);
+  }
+}
+
+__global__ void tc_pack_rows_kernel(const float* __restrict__ x, int K, int Mpad, uint8_t* __restrict__ apack) {
+  const int m = blockIdx.x;
+  for (int j = threadIdx.x * 2; j < K; j += blockDim.x * 2)
+    store_pair(apack, Mpad, m, j, x[(size_t)m * K + j], x[(size_t)m * K + j + 1]);
+}
+
+// One CTA per row: q/k/v = sum of the K slices + bias; rotate q and k by the row's position
+// (rotate-half pairs (j, j + hd/2)); q scaled by 1/sqrt(hd) to qrot; K (rotated) and V to the
+// cache at slot len + r.
+__global__ void __launch_bounds__(256)
+tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
+                   const bf16* __restrict__ bias, const float* __restrict__ cs, float* __restrict__ qrot,
+                   bf16* __restrict__ kv_layer, const int32_t* __restrict__ len, RowMap rm, int cap, int Hq,
+                   int Hkv, int hd, float scale, int32_t* status) {
+  extern __shared__ float row[];  // [(Hq + 2 Hkv) * hd]
+  const int m = blockIdx.x, tid = threadIdx.x;
+  const int bi = m / rm.R, r = m % rm.R, b = rm.b0 + bi;
+  const int pos = len[b] + r, half = hd >> 1, nq = (Hq + 2 * Hkv) * hd;
+  for (int j = tid * 2; j < nq; j += 512) {
+    float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bias + j));
+    for (int s = 0; s < nsplit; ++s) {  // fixed order
+      const float2 p = *reinterpret_cast<const float2*>(part + ((size_t)s * Mpad + m) * ld_part + j);
+      v.x += p.x;
+      v.y += p.y;
+    }
+    row[j] = v.x;
+    row[j + 1] = v.y;
+  }
+  __syncthreads();
+  const float* c = cs + (size_t)m * half * 2;
+  for (int i = tid; i < Hq * half; i += 256) {
+    const int hh = i / half, j = i % half;
+    const float x1 = row[hh * hd + j], x2 = row[hh * hd + j + half], co = c[2 * j], si = c[2 * j + 1];
+    qrot[(size_t)m * Hq * hd + hh * hd + j] = (x1 * co - x2 * si) * scale;
+    qrot[(size_t)m * Hq * hd + hh * hd + j + half] = (x2 * co + x1 * si) * scale;
+  }
+  if (pos < 0 || pos >= cap) {  // never write outside the stream's slice of the cache
+    if (tid == 0) atomicOr(status, SSD_STATUS_KV_OVERFLOW);
+    return;
+  }
+  const float* krow = row + Hq * hd;
+  const float* vrow = krow + Hkv * hd;
+  for (int i = tid; i < Hkv * half; i += 256) {
+    const int g = i / half, j = i % half;
+    const float x1 = krow[g * hd + j], x2 = krow[g * hd + j + half], co = c[2 * j], si = c[2 * j + 1];
+    bf16* kdst = kv_layer + (((size_t)b * 2 + 0) * Hkv + g) * (size_t)cap * hd + (size_t)pos * hd;
+    kdst[j] = __float2bfloat16_rn(x1 * co - x2 * si);
+    kdst[j + half] = __float2bfloat16_rn(x2 * co + x1 * si);
+  }
+  for (int i = tid; i < Hkv * hd; i += 256) {
+    const int g = i / hd, j = i % hd;
+    bf16* vdst = kv_layer + (((size_t)b * 2 + 1) * Hkv + g) * (size_t)cap * hd + (size_t)pos * hd;
+    vdst[j] = __float2bfloat16_rn(vrow[g * hd + j]);
+  }
+}
+
+}  // namespace
+
+void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, int M, int d,
+                         const bf16* gain, float eps, uint8_t* apack, cudaStream_t st) {
+  tc_norm_pack_kernel<<<M, 256, (size_t)d * 4, st>>>(h, part, part ? nsplit : 0, ld_part, tc_round16(M), d, gain,
+                                                     eps, apack);
+  count_launch();
+}
+
+void launch_tc_pack_rows(const float* x, int M, int K, uint8_t* apack, cudaStream_t st) {
+  tc_pack_rows_kernel<<<M, 128, 0, st>>>(x, K, tc_round16(M), apack);
+  count_launch();
+}
+
+void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, const bf16* bias,
+                        const float* cs, float* qrot, bf16* kv_layer, const int32_t* len, RowMap rm,
+                        int cap, int Hq, int Hkv, int hd, int32_t* status, cudaStream_t st) {
+  const int M = rm.nb * rm.R;
+  const size_t smem = (size_t)(Hq + 2 * Hkv) * hd * 4;
+  tc_qkv_post_kernel<<<M, 256, smem, st>>>(part, nsplit, ld_part, Mpad, bias, cs, qrot, kv_layer, len, rm, cap, Hq,
+                                           Hkv, hd, 1.0f / sqrtf((float)hd), status);
+  count_launch();
+}
+
+}  // namespace ssd

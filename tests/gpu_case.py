@@ -5,11 +5,16 @@ Used by the GPU parity tests and by the smoke check.  The comparison rules:
 * logits: max-abs difference within `logit_tol` (3e-2 for bf16 storage, 2e-4 for fp32);
 * token decisions, strict: the oracle's acceptance arithmetic applied to the GPU's own logits
   must reproduce the GPU's (k, y) exactly, except for draws closer than 1e-3 to a decision
-  boundary (|r_i - a_i| < 1e-3, a categorical draw within 1e-3 of a CDF edge, or a top-k cut
-  whose neighbours differ by < 1e-3), after which the stream-step is no longer compared;
+  boundary (|r_i - a_i| < 1e-3, a categorical draw within 1e-5 (in mass) of a CDF edge, or a
+  top-k cut whose neighbours differ by < 1e-5), after which the stream-step is no longer compared;
 * token decisions, end to end: the pure oracle's (k, y) must equal the GPU's unless r_i falls
-  between the two sides' thresholds (widened by 1e-3), i.e. unless the logit rounding moved a
-  boundary across the uniform.
+  between the two sides' thresholds (widened by 1e-3), or the draw's uniform falls within 1e-5
+  (in mass) of where either side puts a CDF edge of the oracle's token, or the two sides keep
+  different top-k sets, i.e. unless the logit rounding moved a boundary across the uniform or an
+  id across the cut.  A bare disagreement is a failure.
+
+Excluded stream-steps are counted and bounded: a case passes only if at least one decision was
+compared and the excluded share stays small.
 """
 from __future__ import annotations
 
@@ -23,7 +28,16 @@ from oracle import ssd_oracle as orc
 from paper_2505_15380_b200 import binding, synth
 from tests.helpers import crafted_draft_rows, oracle_model
 
-WINDOW = 1e-3
+WINDOW = 1e-3        # acceptance test: |a_i - r_i| closer than this is not compared
+# Categorical draws and top-k cuts.  The strict comparison applies the oracle's float64 arithmetic
+# to the GPU's own logits, so the two sides differ only by fp32 rounding of exp, of the row sum and
+# of logit / T (about 1e-6 of the total mass, 1e-7 relative in z): a draw is skipped when it lies
+# within 1e-5 (in mass) of a CDF edge, a top-k cut when its two neighbours differ by < 1e-5.
+# End to end both CDFs are built explicitly and the uniform must fall inside the token's interval
+# on both sides by 1e-5; a top-k row is skipped only if the two sides really keep different sets.
+DRAW_WINDOW = 1e-5
+DRAW_EPS = 1e-5
+TOPK_GAP = 1e-5
 
 
 @dataclasses.dataclass
@@ -55,13 +69,36 @@ def _topk_gap_small(logits_row: np.ndarray, temperature: float, top_k: int) -> b
     if not (0 < top_k < V):
         return False
     z = np.sort(logits_row / temperature)[::-1]
-    return bool(z[top_k - 1] - z[top_k] < WINDOW)
+    return bool(z[top_k - 1] - z[top_k] < TOPK_GAP)
+
+
+def _draw_interval(q_row: np.ndarray, p_row: Optional[np.ndarray], y: int):
+    """[lo, hi) of token y in the normalised CDF the new token is drawn from: the residual
+    max(0, q - p) after a rejection (q itself when that has no mass), q for the bonus token."""
+    w = q_row.astype(np.float64)
+    if p_row is not None:
+        r = np.maximum(0.0, w - p_row.astype(np.float64))
+        w = r if r.sum() > 0.0 else w
+    cdf = np.cumsum(w) / w.sum()
+    return (float(cdf[y - 1]) if y > 0 else 0.0), float(cdf[y])
+
+
+def check_exclusions(res: "CaseResult", max_strict_frac: float = 0.10,
+                     max_e2e_frac: float = 0.34) -> None:
+    """A parity case must have compared something, and may skip only a small share."""
+    n = res.n_streams
+    assert n >= 1 and n - res.n_strict_excluded >= 1, "no decision was compared"
+    assert res.n_strict_excluded <= max(1, int(max_strict_frac * n)), \
+        f"{res.n_strict_excluded} of {n} stream-steps excluded from the strict comparison"
+    assert res.n_e2e_excluded <= max(1, int(max_e2e_frac * n)), \
+        f"{res.n_e2e_excluded} of {n} stream-steps excluded from the end-to-end comparison"
 
 
 def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "prefill",
              oracle_streams: Optional[List[int]] = None, logit_tol: Optional[float] = None,
              uniform_seed: int = 0, commit_and_repeat: bool = False,
-             capacity: Optional[int] = None, path: int = 0, split: bool = True) -> CaseResult:
+             capacity: Optional[int] = None, path: int = 0, split: bool = True,
+             max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -159,14 +196,18 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
                     break
             if not strict_excl:
                 assert g_k[b] == o2["k"], f"stream {b}: accepted length {g_k[b]} vs {o2['k']}"
-                if o2["draw_margin"] < WINDOW or _topk_gap_small(gl[o2["k"]], wl.temperature,
-                                                                 wl.top_k):
+                if o2["draw_margin"] < DRAW_WINDOW or _topk_gap_small(gl[o2["k"]], wl.temperature,
+                                                                      wl.top_k):
                     strict_excl = True
                 else:
                     assert g_y[b] == o2["y"], f"stream {b}: token {g_y[b]} vs {o2['y']}"
             res.n_strict_excluded += int(strict_excl)
             # end to end: pure oracle
-            e2e_excl = strict_excl
+            e2e_excl = False
+            n_rows_eval = min(max(o["k"], o2["k"]) + 1, R)
+            for i in range(n_rows_eval):
+                if not np.array_equal(o["q_rows"][i] > 0, q_g[i] > 0):
+                    e2e_excl = True     # the logit rounding moved an id across the top-k cut
             for i in range(min(max(o["k"], o2["k"]) + 1, gamma)):
                 lo = min(o["thresholds"][i] if i < len(o["thresholds"]) else 9.0,
                          o2["thresholds"][i] if i < len(o2["thresholds"]) else 9.0) - WINDOW
@@ -176,10 +217,15 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
                     e2e_excl = True
             if not e2e_excl:
                 assert g_k[b] == o["k"], f"stream {b}: e2e accepted length {g_k[b]} vs {o['k']}"
-                if o["y"] == o2["y"] and o["draw_margin"] >= WINDOW:
-                    assert g_y[b] == o["y"]
+                kk = o["k"]
+                prow = p_rows[b][kk] if kk < gamma else None
+                lo1, hi1 = _draw_interval(o["q_rows"][kk], prow, o["y"])
+                lo2, hi2 = _draw_interval(q_g[kk], prow, o["y"])
+                ud = float(uni[b, kk, 1])
+                if max(lo1, lo2) + DRAW_EPS <= ud < min(hi1, hi2) - DRAW_EPS:
+                    assert g_y[b] == o["y"], f"stream {b}: e2e token {g_y[b]} vs {o['y']}"
                 else:
-                    e2e_excl = True
+                    e2e_excl = True       # the uniform sits at an edge one side may have moved
             res.n_e2e_excluded += int(e2e_excl)
             if commit_and_repeat:
                 orc.commit(st, int(g_k[b]), int(g_y[b]))      # follow the GPU's trajectory
@@ -189,4 +235,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
             lens_g, pend_g = gs.get_state()
             for b in which:
                 assert lens_g[b] == ostreams[b].length and pend_g[b] == ostreams[b].pending
+    print(f"[{wl.name}] streams-steps {res.n_streams}, strict excluded {res.n_strict_excluded}, "
+          f"e2e excluded {res.n_e2e_excluded}, max|dlogit| {res.max_logit_err:.2e}, k {res.ks}")
+    check_exclusions(res, max_strict_frac, max_e2e_frac)
     return res

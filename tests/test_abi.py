@@ -36,9 +36,11 @@ def test_size_queries_follow_the_shape_arithmetic(L):
     arena = L.ssd_model_arena_bytes(ctypes.byref(cfg))
     streamed = synth.workload(1).target.streamed_weight_bytes()
     embed = (6564 + 32768) * 896 * 2
-    # a bf16 model is held twice: row-major for the generic kernels and packed in tensor-core
-    # operand order for the persistent small-batch kernel (plus its small tables)
-    assert 2 * streamed + embed - (1 << 20) <= arena <= 2 * streamed + embed + (2 << 20)
+    # a bf16 model is held three times: row-major for the generic kernels, packed in the operand
+    # order of the warp-level instruction for the persistent small-batch kernel (plus its small
+    # tables), and in 128-row tiles for the tcgen05 projections of batched forwards (whose last
+    # tile of the LM head is padded)
+    assert 3 * streamed + embed - (1 << 20) <= arena <= 3 * streamed + embed + (3 << 20)
     cfg0 = binding.make_config(synth.workload(0).target)           # fp32: one copy only
     arena0 = L.ssd_model_arena_bytes(ctypes.byref(cfg0))
     streamed0 = synth.workload(0).target.streamed_weight_bytes()

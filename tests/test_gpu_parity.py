@@ -88,7 +88,8 @@ def test_cfg1_with_plain_bf16_activations():
 
 @pytest.mark.parametrize("gamma,prefix", [(2, 256), (4, 512), (6, 1024), (8, 2048)])
 def test_cfg2_sweep_synthetic_kv(gamma, prefix):
-    _case(synth.workload(2, gamma=gamma, prefix=prefix), beta=0.4, sigma=1.0, kv_mode="synthetic")
+    _case(synth.workload(2, gamma=gamma, prefix=prefix), beta=0.4, sigma=1.0, kv_mode="synthetic",
+          commit_and_repeat=True)
 
 
 def test_cfg3_batch16_ragged_topk():
@@ -244,6 +245,19 @@ def test_both_paths_agree_and_forward_only_matches():
         res.append((lg.cpu(), k.cpu(), y.cpu(), gs.kv[:, :, :, :, :150].float().cpu()))
     assert (res[0][0] - res[1][0]).abs().max() < 2e-3
     assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+    # both against the oracle's forward from the same synthetic prefix (the K-split down projection
+    # at a small shape is checked here and nowhere else)
+    from oracle import ssd_oracle as orc
+    from tests.gpu_case import oracle_stream_from_gpu_kv
+    from tests.helpers import oracle_model
+    om = oracle_model(shape, w)
+    gs = binding.Streams(model, B, 200, g)
+    synth.fill_synthetic_kv(gs.kv, lens, seed=5)
+    for b, pend in enumerate([3, 4]):
+        st = oracle_stream_from_gpu_kv(om, gs, b, lens[b], pend)
+        ol = orc.forward(om, st, np.concatenate([[pend], x[b].cpu().numpy()]))
+        for path in (0, 1):
+            assert np.abs(res[path][0][b].numpy() - ol).max() < 2e-3, (b, path)
     # the appended K/V rows agree up to the storage rounding of values that differ in the last bits
     n0 = lens[0]
     assert (res[0][3][:, 0, :, :, n0:n0 + g + 1] - res[1][3][:, 0, :, :, n0:n0 + g + 1]).abs().max() < 2e-2
@@ -277,3 +291,60 @@ def test_phase_trace_of_the_persistent_kernel():
     gs.forward(x, 4, lg)
     torch.cuda.synchronize()
     assert not buf.any()
+
+
+def test_verify_host_rejects_a_model_of_another_shape_before_any_copy():
+    from paper_2505_15380_b200 import binding
+    shape = _small(synth.BF16, 64)
+    other = _small(synth.BF16, 64, v=900)               # larger vocabulary: larger p rows
+    model = binding.Model(shape, synth.weights_blob(shape, synth.make_weights(shape, 3)))
+    big = binding.Model(other, synth.weights_blob(other, synth.make_weights(other, 3)))
+    gs = binding.Streams(model, 2, 64, 4)
+    gs.kv_truncate([5, 9], [1, 2])
+    par = binding.VerifyParams(4, 1.0, 0, 0.0)
+    x = torch.zeros((2, 4), dtype=torch.int32).pin_memory()
+    p = torch.full((2, 4, 900), 1 / 900, dtype=torch.float32).pin_memory()
+    u = torch.zeros((2, 5, 2), dtype=torch.float32).pin_memory()
+    hk = torch.zeros(2, dtype=torch.int32).pin_memory()
+    hy = torch.zeros(2, dtype=torch.int32).pin_memory()
+    L = binding.lib()
+    before_ws = gs.ws.clone()
+    n0 = L.ssd_kernel_launch_count()
+    rc = L.ssd_verify_host(big.handle, gs.handle, x.data_ptr(), p.data_ptr(), u.data_ptr(),
+                           ctypes.byref(par), hk.data_ptr(), hy.data_ptr(), None)
+    torch.cuda.synchronize()
+    assert rc == -2
+    assert L.ssd_kernel_launch_count() == n0
+    assert torch.equal(gs.ws, before_ws)                # nothing was copied into the workspace
+
+
+def test_failed_streams_object_refuses_further_forwards():
+    """The error path of the persistent kernel's bounded waits, made on the host: once the sticky
+    failure word is set, the next forward returns at once, writes nothing, and raises the timeout
+    bit; a fresh streams object on the same model works."""
+    from paper_2505_15380_b200 import binding
+    shape = _fast_shape(64)
+    model = binding.Model(shape, synth.weights_blob(shape, synth.make_weights(shape, 3)))
+    dev = model.device
+    V = shape.vocab_out
+    x = torch.zeros((1, 4), dtype=torch.int32, device=dev)
+    gs = binding.Streams(model, 1, 64, 4)
+    gs.kv_truncate([0], [3])
+    good = torch.zeros((1, 5, V), dtype=torch.float32, device=dev)
+    gs.forward(x, 4, good)
+    torch.cuda.synchronize()
+    assert gs.last_status() == 0 and good.abs().sum() > 0
+    gs.inject_failure()
+    lg = torch.full((1, 5, V), 7.0, dtype=torch.float32, device=dev)
+    gs.forward(x, 4, lg)
+    torch.cuda.synchronize()
+    assert gs.last_status() & 16
+    assert bool((lg == 7.0).all())                      # the kernel left before writing anything
+    gs.forward(x, 4, lg)                                # and stays refused
+    torch.cuda.synchronize()
+    assert gs.last_status() & 16 and bool((lg == 7.0).all())
+    gs2 = binding.Streams(model, 1, 64, 4)
+    gs2.kv_truncate([0], [3])
+    gs2.forward(x, 4, lg)
+    torch.cuda.synchronize()
+    assert gs2.last_status() == 0 and torch.equal(lg, good)

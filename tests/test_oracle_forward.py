@@ -161,6 +161,29 @@ def test_kv_storage_rounding():
     assert np.array_equal(synth.bf16_round(k.astype(np.float32)).astype(np.float64), k)
 
 
+def test_bf16_rounding_is_round_to_nearest_even():
+    """The cache's storage rounding against torch's own float32 -> bfloat16 conversion (a library
+    routine) and against ties worked out by hand: bf16 keeps 8 significand bits, so around 1 the
+    spacing is 2^-7 and a value exactly half way goes to the even neighbour."""
+    rng = np.random.Generator(np.random.Philox(key=5))
+    x = np.concatenate([rng.standard_normal(4000) * 3.0, rng.standard_normal(2000) * 1e-3,
+                        rng.standard_normal(1000) * 1e4, [0.0, -0.0, 1.0, -1.0]]).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(orc._round_to_bf16(x.astype(np.float64)), ref)
+    e = 2.0 ** -8                                      # half a bf16 step at 1
+    cases = {1 + e: 1.0,                               # tie -> even (down)
+             1 + 3 * e: 1 + 4 * e,                     # tie -> even (up)
+             1 + e + 2.0 ** -20: 1 + 2 * e,            # just above the tie
+             1 + e - 2.0 ** -20: 1.0,                  # just below
+             -(1 + e): -1.0, -(1 + 3 * e): -(1 + 4 * e),
+             0.3: 0.30078125, -2.7: -2.703125}
+    for v, want in cases.items():
+        assert orc._round_to_bf16(np.array([v]))[0] == want, v
+    # truncation or round-half-up would each fail one of the ties above
+    assert orc._round_to_bf16(np.array([1 + 3 * e]))[0] != 1 + 2 * e
+    assert orc._round_to_bf16(np.array([1 + e]))[0] != 1 + 2 * e
+
+
 def test_commit_then_verify_equals_fresh_prefill():
     shape = small_shape()
     m, st, ids = _prefilled(shape)
