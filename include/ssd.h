@@ -206,6 +206,52 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
 int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
                   void* stream);
 
+/* One whole SSD iteration (the body of Algorithm 1's while loop) for all B streams, enqueued on
+ * `stream` without any host round trip: gamma draft steps (Eq. 2-3), the parallel verification and
+ * acceptance (Eq. 4-6), "append to T_in" on the target's and on the draft's cache, and the
+ * emitted tokens appended to a per-stream output.  Capture it in a CUDA graph and replay it to
+ * run the loop from the device.
+ *
+ * Draft-cache rule: after an iteration the draft holds K/V for the old pending token and
+ * x_1..x_{gamma-1}.  Every iteration therefore starts with a draft step over TWO ids, [the token
+ * before the pending one, the pending one], at draft len = target len - 1: after a full acceptance
+ * this computes the missing K/V of x_gamma, otherwise it recomputes one cached row from the same
+ * inputs.  One rule for all streams, so no stream's acceptance count ever reaches the host.
+ * Before the first iteration the caller prefills both models with the same prefix (>= 2 tokens),
+ * rolls the DRAFT streams back by one (ssd_kv_truncate to len - 1) and stores the prefix's last
+ * two ids in dev_in_ids.  The draft streams need max_gamma >= 1 and capacity for gamma + 1 more
+ * tokens than the target's prefix.
+ *
+ * ssd_loop_io (all device pointers, caller-owned):
+ *   dev_uniform_pool float [n_iterations][B][gamma + 2 (gamma + 1)]: per stream the gamma draws
+ *                    for x_i ~ p_i, then (r_i, u_i) for the gamma + 1 verify rows, all in [0, 1);
+ *   dev_iteration    int32 [1]: row of the pool the next iteration uses (modulo n_iterations);
+ *                    advanced by one at the end of the iteration;
+ *   dev_in_ids       int32 [B, 2]: the next iteration's first two draft inputs (see above); updated;
+ *   dev_draft_tokens int32 [B, gamma], dev_draft_probs float [B, gamma, V]: x_i and p_i of the
+ *                    iteration (outputs, also useful to inspect);
+ *   dev_accepted_len, dev_next_token  int32 [B]: k and the new token of the iteration;
+ *   dev_out_tokens   int32 [B, out_capacity], dev_out_count int32 [B]: x_1..x_k, y are appended at
+ *                    out_count (tokens beyond the capacity are counted, not stored);
+ *   dev_accept_log   int32 [n_iterations, B] or NULL: k of every iteration (row = pool row). */
+typedef struct {
+  const float* dev_uniform_pool;
+  int32_t n_iterations;
+  int32_t* dev_iteration;
+  int32_t* dev_in_ids;
+  int32_t* dev_draft_tokens;
+  float* dev_draft_probs;
+  int32_t* dev_accepted_len;
+  int32_t* dev_next_token;
+  int32_t* dev_out_tokens;
+  int32_t out_capacity;
+  int32_t* dev_out_count;
+  int32_t* dev_accept_log;
+} ssd_loop_io;
+int ssd_iteration(ssd_model* target, ssd_streams* target_streams, ssd_model* draft,
+                  ssd_streams* draft_streams, const ssd_verify_params* params, const ssd_loop_io* io,
+                  void* stream);
+
 /* Acceptance step without any device allocation (the paper has no counterpart: this is a
  * packaging variant of the acceptance kernel behind ssd_verify, not a step of the method).
  * For callers that may not allocate device memory at all - e.g. a serving loop whose memory pool

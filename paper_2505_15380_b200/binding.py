@@ -25,7 +25,7 @@ EXPORTS = [
     "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_streams_inject_failure",
-    "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check",
+    "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check", "ssd_iteration",
     "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
@@ -42,6 +42,16 @@ class ModelConfig(ctypes.Structure):
 class VerifyParams(ctypes.Structure):
     _fields_ = [("gamma", ctypes.c_int32), ("temperature", ctypes.c_float),
                 ("top_k", ctypes.c_int32), ("beta", ctypes.c_float)]
+
+
+class LoopIo(ctypes.Structure):
+    """ssd_loop_io of include/ssd.h: device pointers of the device-resident SSD iteration."""
+    _fields_ = [("dev_uniform_pool", ctypes.c_void_p), ("n_iterations", ctypes.c_int32),
+                ("dev_iteration", ctypes.c_void_p), ("dev_in_ids", ctypes.c_void_p),
+                ("dev_draft_tokens", ctypes.c_void_p), ("dev_draft_probs", ctypes.c_void_p),
+                ("dev_accepted_len", ctypes.c_void_p), ("dev_next_token", ctypes.c_void_p),
+                ("dev_out_tokens", ctypes.c_void_p), ("out_capacity", ctypes.c_int32),
+                ("dev_out_count", ctypes.c_void_p), ("dev_accept_log", ctypes.c_void_p)]
 
 
 class SsdError(RuntimeError):
@@ -86,6 +96,7 @@ def lib() -> ctypes.CDLL:
     L.ssd_kv_restore.argtypes = [vp, vp, vp, vp]
     L.ssd_accept_noalloc.argtypes = [vp, vp, vp, vp, parp, i32, i32, vp, vp, vp]
     L.ssd_streams_inject_failure.argtypes = [vp, vp]
+    L.ssd_iteration.argtypes = [vp, vp, vp, vp, parp, ctypes.POINTER(LoopIo), vp]
     L.ssd_tc_gemm_scratch_bytes.restype = sz
     L.ssd_tc_gemm_scratch_bytes.argtypes = [i32, i32, i32]
     L.ssd_tc_gemm_check.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, sz, vp, vp, vp]
@@ -346,3 +357,42 @@ def tc_gemm_check(w: torch.Tensor, x: torch.Tensor, ksplit: int, epilogue: int, 
                                   scratch.data_ptr(), need, out.data_ptr(), status.data_ptr(),
                                   _stream_ptr(stream)))
     return out, status
+
+
+class Loop:
+    """Buffers of the device-resident SSD iteration (ssd_iteration) and the call itself.
+
+    Both stream sets must already hold the same prefixes (prefill both models); this object rolls
+    the draft streams back by one token and keeps the last two prefix ids, as the call expects."""
+
+    def __init__(self, target: Streams, draft: Streams, prefixes: Sequence[np.ndarray], gamma: int,
+                 uniform_pool: np.ndarray, out_capacity: int):
+        B, V = target.B, target.model.shape.vocab_out
+        assert draft.B == B and len(prefixes) == B and all(len(p) >= 2 for p in prefixes)
+        per = gamma + 2 * (gamma + 1)
+        assert uniform_pool.dtype == np.float32 and uniform_pool.shape[1:] == (B, per)
+        dev = target.model.device
+        self.target, self.draft, self.gamma = target, draft, gamma
+        self.pool = torch.from_numpy(np.ascontiguousarray(uniform_pool)).to(dev)
+        self.iteration = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.in_ids = torch.from_numpy(np.stack([np.asarray(p[-2:], np.int32) for p in prefixes])).to(dev)
+        self.draft_tokens = torch.zeros((B, gamma), dtype=torch.int32, device=dev)
+        self.draft_probs = torch.zeros((B, gamma, V), dtype=torch.float32, device=dev)
+        self.accepted_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.next_token = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.out_tokens = torch.zeros((B, out_capacity), dtype=torch.int32, device=dev)
+        self.out_count = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.accept_log = torch.full((uniform_pool.shape[0], B), -9, dtype=torch.int32, device=dev)
+        lens, pend = draft.get_state()
+        draft.kv_truncate(lens - 1, pend)
+        self.io = LoopIo(self.pool.data_ptr(), uniform_pool.shape[0], self.iteration.data_ptr(),
+                         self.in_ids.data_ptr(), self.draft_tokens.data_ptr(), self.draft_probs.data_ptr(),
+                         self.accepted_len.data_ptr(), self.next_token.data_ptr(),
+                         self.out_tokens.data_ptr(), out_capacity, self.out_count.data_ptr(),
+                         self.accept_log.data_ptr())
+
+    def iterate(self, params: VerifyParams, stream=None) -> None:
+        assert params.gamma == self.gamma
+        check(lib().ssd_iteration(self.target.model.handle, self.target.handle, self.draft.model.handle,
+                                  self.draft.handle, ctypes.byref(params), ctypes.byref(self.io),
+                                  _stream_ptr(stream)))

@@ -29,6 +29,8 @@ int cuda_fail(cudaError_t e, const char* what) {
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
+constexpr size_t PREFILL_ROWS = 64;  // least rows a bf16 streams object can run in one forward
+
 bool cfg_ok(const ssd_model_config* c) {
   if (!c) return false;
   if (c->n_layers < 1 || c->d_model < 8 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
@@ -148,6 +150,8 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
   size_t F = c.d_ffn, V = c.vocab_out;
   size_t M = (size_t)B * (max_gamma + 1);
+  // bf16 models: room for prefill chunks large enough for the tensor-core forward
+  if (c.weight_dtype == 1 && M < PREFILL_ROWS) M = PREFILL_ROWS;
   p.max_rows = (int)M;
   p.nsplit_max = (cap + ATTN_CHUNK - 1) / ATTN_CHUNK;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
@@ -295,11 +299,13 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
   const int n_sm = m->tc.n_sm;
   auto ld_of = [](int rows) { return (rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS * TC_TILE_ROWS; };
   const int ks_qkv = tc_ksplit(nq, d, n_sm), ks_o = tc_ksplit(d, qd, n_sm), ks_d = tc_ksplit(d, F, n_sm);
-  // key splits of the attention: enough CTAs for two to three waves, whole 64-key tiles each
+  // key splits of the attention: whole 64-key tiles, and at most two CTAs per SM in all, which
+  // is what fits at once (a second, partly filled wave would cost as much as the first)
   const int G = c.n_q_heads / c.n_kv_heads, rowgroups = (G * rm.R + 63) / 64;
-  long long kps = ((long long)s->cap * rm.nb * c.n_kv_heads * rowgroups * 2 + 5LL * n_sm - 1) / (5LL * n_sm);
+  long long kps = ((long long)s->cap * rm.nb * c.n_kv_heads * rowgroups + 2LL * n_sm - 1) / (2LL * n_sm);
   kps = (kps + 63) / 64 * 64;
   if (kps < 64) kps = 64;
+  while ((s->cap + kps - 1) / kps > 128) kps += 64;  // the merge kernel's table of splits
   const int nsplit = (int)((s->cap + kps - 1) / kps);
   launch_embed(1, m->embed, c.vocab_out + c.vocab_text, d, s->row_ids, M, s->h, s->status, st);
   launch_rope_table(s->len, rm, m->inv_freq, c.head_dim / 2, s->rope_cs, st);
@@ -373,6 +379,30 @@ int forward(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cu
                               c.vocab_out, M, c.vocab_out, d, st));
   }
   SSD_CUDA(cudaGetLastError());
+  return SSD_OK;
+}
+
+// One autoregressive step of the draft model for every stream (Eq. 2-3): feeds n_in ids per
+// stream (ids [B, n_in], or null with n_in = 1: each stream's pending token), commits them, and
+// draws x ~ p from the transformed last row.  Token and row are written with the given strides.
+int draft_step_impl(ssd_model* draft, ssd_streams* ds, const int32_t* ids, int n_in, const float* uniform,
+                    const ssd_verify_params* params, int32_t* out_token, int tok_stride, float* out_prob,
+                    size_t prob_stride, cudaStream_t st) {
+  const int V = draft->cfg.vocab_out;
+  const RowMap rm{0, ds->B, n_in};
+  int rc;
+  if (use_fast(draft, ds, rm)) {  // explicit ids, or row 0 = pending when there are none
+    rc = forward_fast(draft, ds, rm, ids, nullptr, ds->logits, st);
+  } else {
+    SSD_CUDA(cudaMemcpyAsync(ds->row_ids, ids ? ids : ds->pending, (size_t)ds->B * n_in * 4,
+                             cudaMemcpyDeviceToDevice, st));
+    rc = forward(draft, ds, rm, ds->logits, st);
+  }
+  if (rc != SSD_OK) return rc;
+  launch_advance_all(ds->len, ds->B, n_in, ds->cap, ds->status, st);
+  SSD_CUDA(launch_draft_sampler(ds->logits + (size_t)(n_in - 1) * V, n_in * V, V, uniform, ds->B,
+                                1.0f / params->temperature, params->top_k, out_token, tok_stride, out_prob,
+                                prob_stride, ds->pending, ds->status, st));
   return SSD_OK;
 }
 
@@ -725,7 +755,11 @@ int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int3
     if (n - 1 > s->cap) return SSD_ERR_KV_OVERFLOW;
   }
   cudaStream_t st = (cudaStream_t)stream;
-  const int chunk = s->max_gamma + 1;
+  // rows per forward: as many as the workspace holds when the tensor-core forward can take them
+  // (one stream at a time, the chunk's rows causal among themselves), else a verify step's worth
+  int chunk = s->max_gamma + 1;
+  if (m->tc.enabled && s->path == 0 && s->tc_part && s->max_rows > FAST_MAX_T)
+    chunk = s->max_rows < TC_MAX_ROWS ? s->max_rows : TC_MAX_ROWS;
   for (int b = 0; b < s->B; ++b) {
     const int32_t* ids = dev_ids + host_offsets[b];
     int n = host_offsets[b + 1] - host_offsets[b];
@@ -751,15 +785,42 @@ int ssd_draft_step(ssd_model* draft, ssd_streams* ds, const int32_t* dev_in_ids,
   int rc = params_ok(ds, params, false);
   if (rc != SSD_OK) return rc;
   if (n_in < 1 || n_in > 2 || n_in > ds->max_gamma + 1) return SSD_ERR_BAD_PARAM;
-  cudaStream_t st = (cudaStream_t)stream;
-  const int V = draft->cfg.vocab_out;
-  SSD_CUDA(cudaMemcpyAsync(ds->row_ids, dev_in_ids, (size_t)ds->B * n_in * 4, cudaMemcpyDeviceToDevice, st));
-  rc = forward(draft, ds, RowMap{0, ds->B, n_in}, ds->logits, st);
+  return draft_step_impl(draft, ds, dev_in_ids, n_in, dev_uniform, params, dev_out_token, 1, dev_out_prob_row,
+                         (size_t)draft->cfg.vocab_out, (cudaStream_t)stream);
+}
+
+int ssd_iteration(ssd_model* target, ssd_streams* ts, ssd_model* draft, ssd_streams* ds,
+                  const ssd_verify_params* params, const ssd_loop_io* io, void* stream) {
+  if (!target || !ts || !draft || !ds || !io) return SSD_ERR_NULL;
+  if (!io->dev_uniform_pool || !io->dev_iteration || !io->dev_in_ids || !io->dev_draft_tokens ||
+      !io->dev_draft_probs || !io->dev_accepted_len || !io->dev_next_token || !io->dev_out_tokens ||
+      !io->dev_out_count)
+    return SSD_ERR_NULL;
+  if (!same_shape(target->cfg, ts->cfg) || !same_shape(draft->cfg, ds->cfg)) return SSD_ERR_BAD_CONFIG;
+  if (ts->B != ds->B || target->cfg.vocab_out != draft->cfg.vocab_out) return SSD_ERR_BAD_CONFIG;
+  int rc = params_ok(ts, params, true);
   if (rc != SSD_OK) return rc;
-  launch_advance_all(ds->len, ds->B, n_in, ds->cap, ds->status, st);
-  SSD_CUDA(launch_draft_sampler(ds->logits + (size_t)(n_in - 1) * V, n_in * V, V, dev_uniform, ds->B,
-                                1.0f / params->temperature, params->top_k, dev_out_token,
-                                dev_out_prob_row, ds->pending, ds->status, st));
+  const int B = ts->B, gamma = params->gamma, V = target->cfg.vocab_out;
+  if (ds->max_gamma < 1 || (size_t)gamma * B > (size_t)ds->max_rows * 2) return SSD_ERR_BAD_GAMMA;
+  if (io->n_iterations < 1 || io->out_capacity < 1) return SSD_ERR_BAD_PARAM;
+  cudaStream_t st = (cudaStream_t)stream;
+  launch_loop_stage_uniforms(io->dev_uniform_pool, io->n_iterations, io->dev_iteration, B, gamma, ds->st_uni,
+                             ts->st_uni, st);
+  for (int i = 0; i < gamma; ++i) {  // Eq. 2-3: x_i ~ p_i = M_p(T_in, x_1..x_{i-1})
+    rc = draft_step_impl(draft, ds, i == 0 ? io->dev_in_ids : nullptr, i == 0 ? 2 : 1, ds->st_uni + (size_t)i * B,
+                         params, io->dev_draft_tokens + i, gamma, io->dev_draft_probs + (size_t)i * V,
+                         (size_t)gamma * V, st);
+    if (rc != SSD_OK) return rc;
+  }
+  rc = ssd_verify(target, ts, io->dev_draft_tokens, io->dev_draft_probs, ts->st_uni, params,
+                  io->dev_accepted_len, io->dev_next_token, nullptr, stream);  // Eq. 4-6
+  if (rc != SSD_OK) return rc;
+  rc = ssd_kv_commit(ts, io->dev_accepted_len, io->dev_next_token, stream);
+  if (rc != SSD_OK) return rc;
+  launch_loop_finish(ds->len, ds->pending, ds->cap, io->dev_in_ids, io->dev_draft_tokens, gamma,
+                     io->dev_accepted_len, io->dev_next_token, B, io->dev_out_tokens, io->out_capacity,
+                     io->dev_out_count, io->dev_accept_log, io->n_iterations, io->dev_iteration, ts->status, st);
+  SSD_CUDA(cudaGetLastError());
   return SSD_OK;
 }
 

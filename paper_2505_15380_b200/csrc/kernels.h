@@ -52,10 +52,21 @@ cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* dra
                                   float* row_stats, int32_t* accept_flags, int32_t* counters,
                                   int32_t* accepted_len, int32_t* next_token, int32_t* status,
                                   cudaStream_t st);
+// out_token[b * tok_stride] and out_prob_row[b * prob_stride + t]: the strides let a loop write
+// step i of every stream straight into the [B, gamma] / [B, gamma, V] arrays the verifier reads.
 cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, const float* uniform,
                                  int B, float inv_temperature, int top_k, int32_t* out_token,
-                                 float* out_prob_row, int32_t* pending, int32_t* status,
-                                 cudaStream_t st);
+                                 int tok_stride, float* out_prob_row, size_t prob_stride,
+                                 int32_t* pending, int32_t* status, cudaStream_t st);
+
+// loop.cu: bookkeeping kernels of the device-resident SSD iteration
+void launch_loop_stage_uniforms(const float* pool, int n_rows, const int32_t* iteration, int B, int gamma,
+                                float* draft_uni, float* verify_uni, cudaStream_t st);
+void launch_loop_finish(int32_t* draft_len, int32_t* draft_pending, int cap, int32_t* in_ids,
+                        const int32_t* draft_tokens, int gamma, const int32_t* accepted_len,
+                        const int32_t* next_token, int B, int32_t* out_tokens, int out_capacity,
+                        int32_t* out_count, int32_t* accept_log, int n_rows, int32_t* iteration,
+                        int32_t* status, cudaStream_t st);
 void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_len,
                       const int32_t* next_token, int B, int cap, int max_gamma, int32_t* status,
                       cudaStream_t st);

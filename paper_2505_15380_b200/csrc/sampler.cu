@@ -305,8 +305,8 @@ cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* dra
 __global__ void __launch_bounds__(SAMP_THREADS)
 draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
                      const float* __restrict__ uniform, float inv_t, int top_k,
-                     int32_t* __restrict__ out_token, float* __restrict__ out_prob,
-                     int32_t* pending, int32_t* status) {
+                     int32_t* __restrict__ out_token, int tok_stride, float* __restrict__ out_prob,
+                     size_t prob_stride, int32_t* pending, int32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SampSmem& sm = *reinterpret_cast<SampSmem*>(smem_raw);
   float* z = reinterpret_cast<float*>(smem_raw + sizeof(SampSmem));
@@ -327,22 +327,22 @@ draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
   for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
     float p = is_kept(z[t], t, st) ? expf(z[t] - st.zmax) / st.sum : 0.f;
     z[t] = p;
-    out_prob[(size_t)b * V + t] = p;
+    out_prob[(size_t)b * prob_stride + t] = p;
   }
   __syncthreads();
   double total;
   int y = block_inverse_cdf(z, V, uniform[b], sm, &total);
   if (y < 0) y = 0;
   if (threadIdx.x == 0) {
-    out_token[b] = y;
+    out_token[(size_t)b * tok_stride] = y;
     pending[b] = y;
   }
 }
 
 cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, const float* uniform,
                                  int B, float inv_temperature, int top_k, int32_t* out_token,
-                                 float* out_prob_row, int32_t* pending, int32_t* status,
-                                 cudaStream_t st) {
+                                 int tok_stride, float* out_prob_row, size_t prob_stride,
+                                 int32_t* pending, int32_t* status, cudaStream_t st) {
   size_t smem = sizeof(SampSmem) + (size_t)V * sizeof(float);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   if (smem > 48 * 1024) {
@@ -351,8 +351,8 @@ cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, cons
     if (e != cudaSuccess) return e;
   }
   draft_sampler_kernel<<<B, SAMP_THREADS, smem, st>>>(logits, ld_logits, V, uniform,
-                                                      inv_temperature, top_k, out_token,
-                                                      out_prob_row, pending, status);
+                                                      inv_temperature, top_k, out_token, tok_stride,
+                                                      out_prob_row, prob_stride, pending, status);
   count_launch();
   return cudaGetLastError();
 }

@@ -258,24 +258,30 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
   const int total = min(len[b] + rm.R, cap);
   const int ns = (total + keys_per_split - 1) / keys_per_split;
   const float* src = part + ((size_t)m * Hq + h) * nsplit * (HD + 2);
-  float m_tot = -CUDART_INF_F;
-  for (int s = 0; s < ns; ++s) m_tot = fmaxf(m_tot, src[s * (HD + 2) + HD]);
-  float denom = 0.f;
-  for (int s = 0; s < ns; ++s) {
-    const float ms = src[s * (HD + 2) + HD];
-    if (ms != -CUDART_INF_F) denom += __expf(ms - m_tot) * src[s * (HD + 2) + HD + 1];
+  __shared__ float s_m[128], s_w[128];  // running max and sum of each split, then its weight
+  for (int s = threadIdx.x; s < ns; s += blockDim.x) {
+    s_m[s] = __ldcg(src + s * (HD + 2) + HD);
+    s_w[s] = __ldcg(src + s * (HD + 2) + HD + 1);
   }
+  __syncthreads();
+  float m_tot = -CUDART_INF_F;
+  for (int s = 0; s < ns; ++s) m_tot = fmaxf(m_tot, s_m[s]);
+  float denom = 0.f;
+  for (int s = 0; s < ns; ++s) {  // fixed order
+    const float e = s_m[s] == -CUDART_INF_F ? 0.f : __expf(s_m[s] - m_tot);
+    denom = fmaf(e, s_w[s], denom);
+  }
+  __syncthreads();
+  for (int s = threadIdx.x; s < ns; s += blockDim.x) s_w[s] = s_m[s] == -CUDART_INF_F ? 0.f : __expf(s_m[s] - m_tot);
+  __syncthreads();
   const float inv = 1.f / denom;
   for (int d = threadIdx.x * 2; d < HD; d += blockDim.x * 2) {
     float o0 = 0.f, o1 = 0.f;
+#pragma unroll 4
     for (int s = 0; s < ns; ++s) {  // fixed order
-      const float ms = src[s * (HD + 2) + HD];
-      if (ms != -CUDART_INF_F) {
-        const float e = __expf(ms - m_tot);
-        const float2 v = *reinterpret_cast<const float2*>(src + s * (HD + 2) + d);
-        o0 = fmaf(e, v.x, o0);
-        o1 = fmaf(e, v.y, o1);
-      }
+      const float2 v = __ldcg(reinterpret_cast<const float2*>(src + s * (HD + 2) + d));
+      o0 = fmaf(s_w[s], v.x, o0);
+      o1 = fmaf(s_w[s], v.y, o1);
     }
     o0 *= inv;
     o1 *= inv;

@@ -25,7 +25,7 @@ namespace ssd {
 namespace {
 
 constexpr unsigned long long TC_WAIT_CYCLES = 2000000000ull;  // ~1 s
-constexpr int TC_MAX_STAGES = 6;
+constexpr int TC_MAX_STAGES = 12;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -336,10 +336,21 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   p.act_out = g.act_out;
   p.status = g.status;
   if (g.ksplit > p.KS || (g.epi != TC_EPI_PARTIAL && g.ksplit != 1)) return cudaErrorInvalidValue;
-  // pipeline: at least three stages of as many k-steps as fit; small forwards leave room for a
-  // second CTA per SM, so that a grid slightly larger than the SM count still runs in one wave
+  // pipeline: at least three stages of as many k-steps as fit.  A grid that exceeds the SM count
+  // by a little leaves room for a second CTA per SM so that it still runs in one wave; any other
+  // grid takes the whole shared memory: with few token rows the weight stream is latency-bound,
+  // and what a CTA keeps in flight is what it gets.
   const size_t per_ks = (size_t)TC_WBLOCK + (size_t)p.Mpad * 64;
-  const size_t budget = p.Mpad <= 192 ? 96 * 1024 : 220 * 1024;
+  int n_sm = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
+      n_sm = 148;
+  }
+  const int ctas = tiles * g.ksplit;
+  const bool two_per_sm = p.Mpad <= 256 && ctas > n_sm && ctas <= 2 * n_sm;
+  const size_t budget = two_per_sm ? 100 * 1024 : 216 * 1024;
   p.sk = 4;
   while (p.sk > 1 && 3 * p.sk * per_ks > budget) p.sk >>= 1;
   p.stages = (int)(budget / (p.sk * per_ks));

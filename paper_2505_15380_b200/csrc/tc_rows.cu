@@ -22,6 +22,28 @@ __device__ __forceinline__ void store_pair(uint8_t* apack, int Mpad, int t, int 
   *reinterpret_cast<__nv_bfloat162*>(apack + act_off(Mpad, 1, t, k)) = l;
 }
 
+// Sum over the K slices of a projection's partial sums for two adjacent columns, in slice order
+// (bit-reproducible); the loads of eight slices are in flight together.
+__device__ __forceinline__ float2 sum_slices(float2 v, const float* __restrict__ p, size_t slice_stride, int nsplit) {
+  int s = 0;
+  for (; s + 8 <= nsplit; s += 8) {
+    float2 t[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t[i] = __ldcg(reinterpret_cast<const float2*>(p + (size_t)(s + i) * slice_stride));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      v.x += t[i].x;
+      v.y += t[i].y;
+    }
+  }
+  for (; s < nsplit; ++s) {
+    const float2 t = __ldcg(reinterpret_cast<const float2*>(p + (size_t)s * slice_stride));
+    v.x += t.x;
+    v.y += t.y;
+  }
+  return v;
+}
+
 // One CTA per row.  h[m, :] += sum_s part[s][m][:]; out = h / rms(h) * gain, packed.
 __global__ void __launch_bounds__(256)
 tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
@@ -32,12 +54,10 @@ tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int n
   float ss = 0.f;
   for (int j = tid * 2; j < d; j += 512) {
     float2 v = *reinterpret_cast<const float2*>(h + (size_t)m * d + j);
-    for (int s = 0; s < nsplit; ++s) {  // fixed order
-      const float2 p = *reinterpret_cast<const float2*>(part + ((size_t)s * Mpad + m) * ld_part + j);
-      v.x += p.x;
-      v.y += p.y;
+    if (nsplit > 0) {
+      v = sum_slices(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
+      *reinterpret_cast<float2*>(h + (size_t)m * d + j) = v;
     }
-    if (nsplit > 0) *reinterpret_cast<float2*>(h + (size_t)m * d + j) = v;
     row[j] = v.x;
     row[j + 1] = v.y;
     ss += v.x * v.x + v.y * v.y;
@@ -75,11 +95,7 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
   const int pos = len[b] + r, half = hd >> 1, nq = (Hq + 2 * Hkv) * hd;
   for (int j = tid * 2; j < nq; j += 512) {
     float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bias + j));
-    for (int s = 0; s < nsplit; ++s) {  // fixed order
-      const float2 p = *reinterpret_cast<const float2*>(part + ((size_t)s * Mpad + m) * ld_part + j);
-      v.x += p.x;
-      v.y += p.y;
-    }
+    v = sum_slices(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
     row[j] = v.x;
     row[j + 1] = v.y;
   }
