@@ -304,7 +304,7 @@ int ssd_fast_pack_roundtrip_host(const ssd_model_config* cfg, int32_t n_cta, con
  *   epilogue 1: ksplit must be 1; dev_out float [M, n_rows] = acc (the LM-head form).
  *   epilogue 2: ksplit must be 1; weight rows are (gate_j, up_j) pairs; dev_out receives
  *               SiLU(gate_j) * up_j as a packed operand of n_rows / 2 columns:
- *               byte(part, t, j) = (j / 16) * Mpad * 64 + part * Mpad * 32 + ((j / 8) % 2) * Mpad * 16
+ *               byte(part, t, j) = (j / 16) * Mpad * 64 + ((j / 8) % 2) * Mpad * 32 + part * Mpad * 16
  *                                  + t * 16 + (j % 8) * 2,  part 0 = bf16 leading part of the
  *               value, part 1 = bf16 of the remainder ((n_rows / 2 rounded up to 16) * Mpad * 4 bytes).
  * Enqueues on `stream`; SSD_ERR_BAD_PARAM for sizes outside the ranges above. */

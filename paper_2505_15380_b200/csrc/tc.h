@@ -19,10 +19,14 @@
 //   weights, per (tile of 128 rows, k-step of 16 columns) one 4 KB block:
 //       byte(r, k) = (k / 8) * 2048 + r * 16 + (k % 8) * 2           leading 2048, stride 128
 //   activations (Mpad token rows, a multiple of 16), per k-step one block of Mpad * 64 bytes:
-//       byte(part, t, k) = part * Mpad * 32 + (k / 8) * Mpad * 16 + t * 16 + (k % 8) * 2
+//       byte(part, t, k) = (k / 8) * Mpad * 32 + part * Mpad * 16 + t * 16 + (k % 8) * 2
 //   with part 0 = bf16 leading part of the fp32 activation, part 1 = bf16 of the remainder: the
-//   tensor cores multiply both with the exact bf16 weights into one fp32 accumulator, so products
-//   are exact to ~2^-17 relative, as in the small-batch kernel.
+//   tensor cores multiply both with the exact bf16 weights, so products are exact to ~2^-17
+//   relative, as in the small-batch kernel.  The two parts of a token sit Mpad rows apart in one
+//   2 * Mpad-row operand: with up to 256 token rows one instruction multiplies both (N = 2 Mpad,
+//   the two halves of the accumulator are added in the epilogue), which matters because an
+//   instruction costs ~190 cycles whatever its N (measured); with more rows the two parts are
+//   separate instructions into the same accumulator columns.
 //
 // K is split across CTAs where a projection has too few row tiles to occupy the GPU; the partial
 // sums go to a workspace and the row-wise kernel that consumes the projection adds them in a

@@ -288,10 +288,10 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
     const int k = h * HD + d;
     const __nv_bfloat162 hi = __floats2bfloat162_rn(o0, o1);
     const __nv_bfloat162 lo = __floats2bfloat162_rn(o0 - __low2float(hi), o1 - __high2float(hi));
-    uint8_t* e = apack + (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mpad * 16) +
+    uint8_t* e = apack + (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mpad * 32) +
                  (size_t)m * 16 + (size_t)(k & 7) * 2;
     *reinterpret_cast<__nv_bfloat162*>(e) = hi;
-    *reinterpret_cast<__nv_bfloat162*>(e + (size_t)Mpad * 32) = lo;
+    *reinterpret_cast<__nv_bfloat162*>(e + (size_t)Mpad * 16) = lo;
   }
 }
 

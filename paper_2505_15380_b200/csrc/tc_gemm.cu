@@ -3,9 +3,9 @@
 // are in flight).  Layouts and the reasons for them: tc.h.
 //
 // One CTA = one tile of 128 weight rows x one K slice x all token rows.  Warp 0 streams the
-// operands: one thread issues, per pipeline stage, one bulk copy of the stage's weight blocks
-// (read once, marked evict-first) and one of the matching activation blocks (re-read by every
-// tile, so they stay in L2), both completing on the stage's "full" barrier.  Warp 1 owns tensor
+// operands: per pipeline stage, eight of its lanes issue bulk copies of the stage's weight blocks
+// (read once, marked evict-first) and of the matching activation blocks (re-read by every tile,
+// so they stay in L2), in pieces of 8 KB, all completing on the stage's "full" barrier.  Warp 1 owns tensor
 // memory and issues the MMAs: per k-step of 16 columns, for the leading and the remainder part of
 // the activations and for each range of at most 256 token columns, one tcgen05.mma (128 x N x 16,
 // bf16 x bf16 -> fp32) reading both operands straight from shared memory; a tcgen05.commit hands
@@ -26,6 +26,11 @@ namespace {
 
 constexpr unsigned long long TC_WAIT_CYCLES = 2000000000ull;  // ~1 s
 constexpr int TC_MAX_STAGES = 12;
+// Operand copies are issued by several lanes of the copy warp, in pieces of at most 8 KB: measured
+// on a B200, one thread issuing one large copy per operand and stage moves 35-48 GB/s into an SM,
+// eight lanes issuing 8 KB pieces 46-90 GB/s.
+constexpr int TC_ISSUERS = 8;
+constexpr uint32_t TC_PIECE = 8192;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -120,7 +125,8 @@ struct TcKernelParams {
   const uint8_t* a;
   int n_rows, KS, M, Mpad, ld_part;  // KS = k-steps of the whole projection; ld_part = tiles * 128
   int sk, stages;                    // k-steps per stage, pipeline depth
-  int nchunks, chunk_n;              // token column ranges of one MMA (<= 256 each)
+  int wide;                          // 1: one instruction multiplies both parts (N over 2 * Mpad rows)
+  int nchunks, chunk_n;              // row ranges of the activation operand per MMA (<= 256 each)
   int tmem_cols;
   int epi;
   float* part;
@@ -150,7 +156,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
 
   if (tid == 0) {
     for (int s = 0; s < P.stages; ++s) {
-      mbar_init(smem_u32(&S.full[s]), 1);
+      mbar_init(smem_u32(&S.full[s]), TC_ISSUERS);
       mbar_init(smem_u32(&S.empty[s]), 1);
     }
     mbar_init(smem_u32(&S.accum), 1);
@@ -169,7 +175,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
   volatile int* abort = &S.abort;
 
   if (warp == 0) {
-    if (lane == 0) {  // ---- operand copies
+    if (lane < TC_ISSUERS) {  // ---- operand copies: piece i of a stage is issued by lane i % TC_ISSUERS
       const uint64_t pol = policy_evict_first();
       const uint8_t* wsrc = P.w + ((size_t)tile * P.KS + ks0) * TC_WBLOCK;
       const uint8_t* asrc = P.a + (size_t)ks0 * act_block;
@@ -179,11 +185,23 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         if (use > 0 && !mbar_wait(smem_u32(&S.empty[s]), (uint32_t)(use - 1) & 1u, abort)) break;
         const int nks = min(P.sk, ks1 - ks0 - it * P.sk);
         const uint32_t bar = smem_u32(&S.full[s]);
-        mbar_expect_tx(bar, (uint32_t)nks * (TC_WBLOCK + act_block));
-        bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w), wsrc, (uint32_t)nks * TC_WBLOCK, bar, pol);
-        bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a), asrc, (uint32_t)nks * act_block, bar);
-        wsrc += (size_t)nks * TC_WBLOCK;
-        asrc += (size_t)nks * act_block;
+        const uint32_t wbytes = (uint32_t)nks * TC_WBLOCK, abytes = (uint32_t)nks * act_block;
+        const uint32_t wp = (wbytes + TC_PIECE - 1) / TC_PIECE, ap = (abytes + TC_PIECE - 1) / TC_PIECE;
+        uint32_t mine = 0;
+        for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS)
+          mine += i < wp ? min(TC_PIECE, wbytes - i * TC_PIECE) : min(TC_PIECE, abytes - (i - wp) * TC_PIECE);
+        mbar_expect_tx(bar, mine);  // every issuing lane arrives once per stage, with its own byte count
+        for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS) {
+          if (i < wp) {
+            const uint32_t off = i * TC_PIECE;
+            bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w) + off, wsrc + off, min(TC_PIECE, wbytes - off), bar, pol);
+          } else {
+            const uint32_t off = (i - wp) * TC_PIECE;
+            bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a) + off, asrc + off, min(TC_PIECE, abytes - off), bar);
+          }
+        }
+        wsrc += wbytes;
+        asrc += abytes;
       }
       if (*abort) {
         // never leave with copies in flight into this CTA's shared memory: the last uses of the
@@ -202,15 +220,24 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         const uint32_t wb = smem_u32(smem_w + (size_t)s * stage_w), ab = smem_u32(smem_a + (size_t)s * stage_a);
         for (int j = 0; j < nks; ++j) {
           const uint64_t da = umma_desc(wb + (uint32_t)j * TC_WBLOCK, 2048u, 128u);
-#pragma unroll
-          for (int part = 0; part < 2; ++part) {
+          const uint32_t blk = ab + (uint32_t)j * act_block, lead = (uint32_t)P.Mpad * 32u;
+          if (P.wide) {
+            // the operand's 2 * Mpad rows (leading parts, then remainders) in ranges of <= 256:
+            // accumulator columns [0, Mpad) receive W x_hi, [Mpad, 2 Mpad) receive W x_lo
             for (int c = 0; c < P.nchunks; ++c) {
-              const int n = min(P.chunk_n, P.Mpad - c * P.chunk_n);
-              const uint64_t db = umma_desc(ab + (uint32_t)j * act_block + (uint32_t)part * (uint32_t)P.Mpad * 32u +
-                                                (uint32_t)(c * P.chunk_n) * 16u,
-                                            (uint32_t)P.Mpad * 16u, 128u);
-              umma_bf16(tmem + (uint32_t)(c * P.chunk_n), da, db, umma_idesc(n),
-                        (it > 0 || j > 0 || part > 0) ? 1u : 0u);
+              const int n = min(P.chunk_n, 2 * P.Mpad - c * P.chunk_n);
+              umma_bf16(tmem + (uint32_t)(c * P.chunk_n), da, umma_desc(blk + (uint32_t)(c * P.chunk_n) * 16u, lead, 128u),
+                        umma_idesc(n), (it > 0 || j > 0) ? 1u : 0u);
+            }
+          } else {
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+              for (int c = 0; c < P.nchunks; ++c) {
+                const int n = min(P.chunk_n, P.Mpad - c * P.chunk_n);
+                umma_bf16(tmem + (uint32_t)(c * P.chunk_n), da,
+                          umma_desc(blk + (uint32_t)(part * P.Mpad + c * P.chunk_n) * 16u, lead, 128u), umma_idesc(n),
+                          (it > 0 || j > 0 || part > 0) ? 1u : 0u);
+              }
             }
           }
         }
@@ -227,6 +254,12 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
       for (int c0 = 0; c0 < P.M; c0 += 32) {
         uint32_t v[32];
         tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        if (P.wide) {  // add the remainder part's products
+          uint32_t w[32];
+          tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(P.Mpad + c0), w);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(w[i]));
+        }
         if (P.epi == TC_EPI_PARTIAL) {
           float* dst = P.part + ((size_t)split * P.Mpad + c0) * P.ld_part + n;
 #pragma unroll
@@ -240,7 +273,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
           }
         } else {  // TC_EPI_SWIGLU: even lanes hold gate_j, odd lanes up_j, j = n / 2
           const int j = n >> 1;
-          uint8_t* dst = P.act_out + (size_t)(j >> 4) * ((size_t)P.Mpad * 64) + (size_t)((j >> 3) & 1) * ((size_t)P.Mpad * 16) +
+          uint8_t* dst = P.act_out + (size_t)(j >> 4) * ((size_t)P.Mpad * 64) + (size_t)((j >> 3) & 1) * ((size_t)P.Mpad * 32) +
                          (size_t)(j & 7) * 2;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -252,7 +285,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
               const bf16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
               uint8_t* e = dst + (size_t)(c0 + i) * 16;
               *reinterpret_cast<bf16*>(e) = hi;
-              *reinterpret_cast<bf16*>(e + (size_t)P.Mpad * 32) = lo;
+              *reinterpret_cast<bf16*>(e + (size_t)P.Mpad * 16) = lo;
             }
           }
         }
@@ -349,17 +382,19 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
       n_sm = 148;
   }
   const int ctas = tiles * g.ksplit;
-  const bool two_per_sm = p.Mpad <= 256 && ctas > n_sm && ctas <= 2 * n_sm;
+  const bool two_per_sm = p.Mpad <= 128 && ctas > n_sm && ctas <= 2 * n_sm;  // 2 x 256 columns
   const size_t budget = two_per_sm ? 100 * 1024 : 216 * 1024;
   p.sk = 4;
   while (p.sk > 1 && 3 * p.sk * per_ks > budget) p.sk >>= 1;
   p.stages = (int)(budget / (p.sk * per_ks));
   if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
   if (p.stages < 2) return cudaErrorInvalidValue;
-  p.nchunks = (p.Mpad + 255) / 256;
-  p.chunk_n = tc_round16((p.Mpad + p.nchunks - 1) / p.nchunks);
+  p.wide = p.Mpad <= 256;  // both parts' products fit the 512 tensor-memory columns side by side
+  const int op_rows = p.wide ? 2 * p.Mpad : p.Mpad;
+  p.nchunks = (op_rows + 255) / 256;
+  p.chunk_n = tc_round16((op_rows + p.nchunks - 1) / p.nchunks);
   p.tmem_cols = 32;
-  while (p.tmem_cols < p.Mpad) p.tmem_cols <<= 1;
+  while (p.tmem_cols < op_rows) p.tmem_cols <<= 1;
   const size_t smem = (size_t)p.stages * p.sk * per_ks + sizeof(TcShared) + 64;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;

@@ -11,8 +11,8 @@ namespace {
 
 // Byte offset of element (part, t, k) of a packed activation operand (tc.h).
 __device__ __forceinline__ size_t act_off(int Mpad, int part, int t, int k) {
-  return (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)part * ((size_t)Mpad * 32) +
-         (size_t)((k >> 3) & 1) * ((size_t)Mpad * 16) + (size_t)t * 16 + (size_t)(k & 7) * 2;
+  return (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mpad * 32) +
+         (size_t)part * ((size_t)Mpad * 16) + (size_t)t * 16 + (size_t)(k & 7) * 2;
 }
 // Columns (k, k + 1), k even, of token t: bf16 leading parts and remainders.
 __device__ __forceinline__ void store_pair(uint8_t* apack, int Mpad, int t, int k, float x0, float x1) {

@@ -73,9 +73,9 @@ def test_swiglu_epilogue_writes_a_packed_operand(M, F, K):
     Mpad = (M + 15) // 16 * 16
     t = np.arange(M)[:, None]
     j = np.arange(F)[None, :]
-    base = (j // 16) * (Mpad * 64) + ((j // 8) % 2) * (Mpad * 16) + t * 16 + (j % 8) * 2
+    base = (j // 16) * (Mpad * 64) + ((j // 8) % 2) * (Mpad * 32) + t * 16 + (j % 8) * 2
     hi = synth.from_bf16_bits(raw[(base // 2)]).astype(np.float64)
-    lo = synth.from_bf16_bits(raw[((base + Mpad * 32) // 2)]).astype(np.float64)
+    lo = synth.from_bf16_bits(raw[((base + Mpad * 16) // 2)]).astype(np.float64)
     assert np.abs(hi + lo - ref).max() <= 3e-5 * np.abs(ref).max() + 1e-6
     assert np.abs(hi - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6     # hi alone is the bf16 rounding
     assert np.abs(lo).max() > 0
