@@ -221,7 +221,7 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = synth.workload(args.config)
+    wl = synth.workload(args.config, gamma=args.gamma, prefix=args.prefix)
     shape = wl.target
     B, g, R, V = wl.batch, wl.gamma, wl.gamma + 1, shape.vocab_out
     w = synth.make_weights(shape, wl.model_seed)
@@ -419,6 +419,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--beta", type=float, default=0.4)
+    ap.add_argument("--gamma", type=int, default=None, help="draft length (config 2's sweep)")
+    ap.add_argument("--prefix", type=int, default=None, help="prefix length (config 2's sweep)")
     ap.add_argument("--draft-noise", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--loop-iterations", type=int, default=200,

@@ -30,6 +30,10 @@ int cuda_fail(cudaError_t e, const char* what) {
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 constexpr size_t PREFILL_ROWS = 64;  // least rows a bf16 streams object can run in one forward
+// Streams with room for this many tokens run the persistent kernel's key-split variant: from a
+// few hundred keys on, ten CTAs sharing a head's keys and meeting once costs less than each of
+// them walking all keys (0.8 us per 128 keys and layer against ~1.5 us for the exchange).
+constexpr int KEYSPLIT_MIN_CAPACITY = 768;
 
 bool cfg_ok(const ssd_model_config* c) {
   if (!c) return false;
@@ -140,6 +144,7 @@ struct WsPlan {
   size_t st_tokens, st_k, st_y, st_probs, st_uni;
   size_t hfix, flags, epoch_base, xa, xb, xd, xq, ssq_a, ssq_b;
   size_t tc_xa, tc_xattn, tc_xact, tc_part;
+  size_t attn_part, attn_cnt;
   size_t total;
   int max_rows, nsplit_max;
 };
@@ -186,6 +191,12 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
   p.ssq_b = take((d / 64 + 1) * FAST_MAX_T * 8);
   p.flags = take(64);
   p.epoch_base = take(2 * 4);
+  p.attn_part = p.attn_cnt = 0;
+  if (fast_supported(c)) {  // key-split attention of the persistent kernel
+    const int hps = c.n_q_heads / fast_o_split(c, fast_cta_count());
+    p.attn_part = take((size_t)FAST_MAX_CTAS * hps * FAST_MAX_T * (c.head_dim + 2) * 4);
+    p.attn_cnt = take((size_t)FAST_MAX_CTAS * 4);
+  }
   p.tc_xa = p.tc_xattn = p.tc_xact = p.tc_part = 0;
   if (c.weight_dtype == 1 && M > FAST_MAX_T && M <= TC_MAX_ROWS) {
     const int Mpad = tc_round16((int)M), n_sm = fast_cta_count();
@@ -278,6 +289,9 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.logits = logits_out;
   p.flags = s->flags;
   p.epoch_base = s->epoch_base;
+  p.attn_part = s->attn_part;
+  p.attn_cnt = s->attn_cnt;
+  p.key_split = s->key_split;
   p.split_act = s->split_act;
   p.trace = s->trace;
   p.trace_cap = s->trace_cap;
@@ -632,6 +646,9 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->ssq_b = (long long*)(W + p.ssq_b);
   s->flags = (uint32_t*)(W + p.flags);
   s->epoch_base = (uint32_t*)(W + p.epoch_base);
+  s->attn_part = p.attn_part ? (float*)(W + p.attn_part) : nullptr;
+  s->attn_cnt = p.attn_part ? (uint32_t*)(W + p.attn_cnt) : nullptr;
+  s->key_split = capacity_tokens >= KEYSPLIT_MIN_CAPACITY ? 1 : 0;
   s->tc_xa = p.tc_part ? (uint8_t*)(W + p.tc_xa) : nullptr;
   s->tc_xattn = p.tc_part ? (uint8_t*)(W + p.tc_xattn) : nullptr;
   s->tc_xact = p.tc_part ? (uint8_t*)(W + p.tc_xact) : nullptr;

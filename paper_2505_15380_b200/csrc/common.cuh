@@ -128,6 +128,9 @@ struct ssd_streams {
   uint32_t *xa, *xb, *xd, *xq;  // projection / attention inputs in tensor-core operand layout
   long long *ssq_a, *ssq_b;
   uint32_t *flags, *epoch_base;
+  float* attn_part;    // persistent kernel, key-split attention: per-CTA partials
+  uint32_t* attn_cnt;  // and the per-slice arrival counters
+  int key_split;       // 1: forwards on these streams use the key-split variant
   // batched tensor-core forward: packed operands (inputs of QKV / gate-up / head, of O, of down)
   // and the partial sums of the K-split projections
   uint8_t *tc_xa, *tc_xattn, *tc_xact;

@@ -146,6 +146,12 @@ struct FastParams {
   // per 64 columns and row the sums of squares that go with xa / xb.
   uint32_t *xa, *xb, *xd, *xq;  // xq: the rotated, scaled queries
   long long *ssq_a, *ssq_b;  // [ceil(d / 64)][FAST_MAX_T], 2^-32 fixed point
+  // key-split attention (long prefixes): per CTA the un-normalised partials of its heads' rows
+  // [n_cta][heads per slice][FAST_MAX_T][hd + 2], and one monotonic arrival counter per slice;
+  // key_split != 0 selects the kernel variant that uses them
+  float* attn_part;
+  uint32_t* attn_cnt;
+  int key_split;
   uint32_t* flags;       // [0] grid-barrier arrival counter, monotonic across launches
   uint32_t* epoch_base;  // [0] counter value at the start of the next launch, [1] nonzero after a failure
   // optional trace: thread 0 of CTA c stores clock64() at trace[c * trace_cap + i] for its i-th

@@ -667,9 +667,15 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 //
 // O projection: the warps split the CTA's tiles (tile u: warp u % 8), two tiles at a time so that
 // the residual adds of both are in flight together.
-template <int HD, bool T16, bool LO>
+//
+// KSPLIT (long prefixes): the CTAs of a slice do not repeat each other's work; CTA j of the J that
+// share the slice walks every J-th 128-key pass only, leaves its un-normalised partial (max, sum,
+// output) in global memory, and the J of them meet on the slice's own arrival counter - a wait of
+// about ten CTAs on one word, not a grid barrier - before each merges all J partials in a fixed
+// order.  Costs one more exchange through L2 per layer, saves (J - 1) / J of the key walk.
+template <int HD, bool T16, bool LO, bool KSPLIT>
 __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
-                                             const PhaseDesc& D, int layer) {
+                                             const PhaseDesc& D, int layer, uint32_t ks_base) {
   constexpr int ROWB = HD * 2 + 16;       // padded K / V row in bytes (conflict-free fragment loads)
   constexpr int NH = T16 ? 2 : 1;         // row halves: rows g and g + 8
   constexpr int W = Lay<T16, LO>::W;      // words per (k-step, lane) of an operand
@@ -681,10 +687,15 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
   constexpr int LPL = 16 * CH / 32;       // 16-byte loads per lane for 16 rows
   constexpr int NROW = 8 * NH;            // rows held
   const int cnt = M.ucnt[FOP_O];
-  if (cnt == 0) return;
+  if (cnt == 0 && !KSPLIT) return;  // key split: a CTA without tiles of W_o still takes its share of the keys
   const int R = P.R, nb = P.nb, Hq = P.Hq, G = Hq / P.Hkv, T = P.T;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   const int hps = Hq / P.m.o_split, slice = (int)blockIdx.x % P.m.o_split, KS = hps * KSTEPS;
+  // key split: this CTA's rank among the J CTAs of its slice
+  const int jr = KSPLIT ? (int)blockIdx.x / P.m.o_split : 0;
+  const int J = KSPLIT ? (P.m.n_cta - slice + P.m.o_split - 1) / P.m.o_split : 1;
+  const int key_step = 16 * FAST_WARPS * J;
+  float* my_part = KSPLIT ? P.attn_part + (size_t)blockIdx.x * hps * FAST_MAX_T * (HD + 2) : nullptr;
 
   uint32_t* qsm = reinterpret_cast<uint32_t*>(uni);                       // q operand, KSTEPS steps
   uint8_t* kv_w = uni + KSTEPS * 32 * W * 4 + warp * (2 * 16 * ROWB);     // this warp's K then V tile
@@ -708,7 +719,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
     const uint4* vg = reinterpret_cast<const uint4*>(kvl + (((size_t)stream * 2 + 1) * P.Hkv + gk) * (size_t)P.cap * HD);
 
     // first tile of this warp: loads in flight before anything else
-    int key0 = 16 * warp;
+    int key0 = 16 * warp + 16 * FAST_WARPS * jr;
     uint4 kq[LPL], vq[LPL];
 #pragma unroll
     for (int i = 0; i < LPL; ++i) {
@@ -744,7 +755,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
 #pragma unroll
     for (int dt = 0; dt < DT; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
 
-    for (; key0 < k1; key0 += 16 * FAST_WARPS) {
+    for (; key0 < k1; key0 += key_step) {
       __syncwarp();
 #pragma unroll
       for (int i = 0; i < LPL; ++i) {
@@ -754,7 +765,7 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
       }
       __syncwarp();
       {  // the next tile's loads, in flight during this tile's arithmetic
-        const int nkey0 = key0 + 16 * FAST_WARPS;
+        const int nkey0 = key0 + key_step;
 #pragma unroll
         for (int i = 0; i < LPL; ++i) {
           const int idx = lane + 32 * i, key = nkey0 + idx / CH;
@@ -897,11 +908,82 @@ __device__ __forceinline__ void attn_o_phase(const FastParams& P, FastMisc& M, u
         o0 = fmaf(ov.x, e, o0);
         o1 = fmaf(ov.y, e, o1);
       }
-      const float il = 1.f / l;
-      write_frag_pair<T16, LO>(osm, tok, hl * HD + dd, o0 * il, o1 * il);
+      if (KSPLIT) {  // this CTA's share of the keys only: leave (max, sum, output) for the merge
+        float* dst = my_part + ((size_t)hl * FAST_MAX_T + tok) * (HD + 2);
+        *reinterpret_cast<float2*>(dst + dd) = make_float2(o0, o1);
+        if (dd == 0) {
+          dst[HD] = m;
+          dst[HD + 1] = l;
+        }
+      } else {
+        const float il = 1.f / l;
+        write_frag_pair<T16, LO>(osm, tok, hl * HD + dd, o0 * il, o1 * il);
+      }
     }
   }
   __syncthreads();
+  if (KSPLIT) {
+    // the J CTAs of the slice meet: release arrival on the slice's monotonic counter, bounded poll
+    const uint32_t target = ks_base + (uint32_t)(layer + 1) * (uint32_t)J;
+    bool ok = true;
+    if (tid == 0) {
+      uint32_t* cnt = P.attn_cnt + slice;
+      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(cnt) : "memory");
+      const long long t0 = clock64();
+      uint32_t spins = 0;
+      while ((int32_t)(ld_acquire_u32(cnt) - target) < 0) {
+        if ((++spins & 63u) == 0u &&
+            (ld_acquire_u32(P.epoch_base + 1) != 0u || (unsigned long long)(clock64() - t0) > FAST_WAIT_CYCLES)) {
+          ok = false;
+          break;
+        }
+      }
+    }
+    if (__syncthreads_or(ok ? 0 : 1)) ring.dead = true;  // the next grid barrier spreads the failure
+    if (cnt == 0) return;
+    // (max, sum) of every (split, row): one round of independent loads into shared memory, then
+    // each split's weight exp(m_j - m) / sum, so that the pass over the outputs has no chain of
+    // dependent loads
+    float* wj = reinterpret_cast<float*>(uni + KSTEPS * 32 * W * 4);  // [hps * T][J], in the K / V staging area
+    const int nrow = hps * nb * R;
+    for (int idx = tid; idx < nrow * J; idx += FAST_THREADS) {
+      const int j = idx % J, row = idx / J, r = row % R, it2 = row / R, hl = it2 / nb, tok = (it2 % nb) * R + r;
+      const float* src = P.attn_part + ((size_t)((slice + j * P.m.o_split) * hps + hl) * FAST_MAX_T + tok) * (HD + 2);
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(src + HD));
+      wj[(size_t)row * 2 * J + j] = ml.x;
+      wj[(size_t)row * 2 * J + J + j] = ml.y;
+    }
+    __syncthreads();
+    for (int row = tid; row < nrow; row += FAST_THREADS) {
+      float* mrow = wj + (size_t)row * 2 * J;
+      float m = -CUDART_INF_F, l = 0.f;
+      for (int j = 0; j < J; ++j) m = fmaxf(m, mrow[j]);
+      for (int j = 0; j < J; ++j) {  // fixed order: bit-reproducible
+        const float e = mrow[j] == -CUDART_INF_F ? 0.f : __expf(mrow[j] - m);
+        l = fmaf(mrow[J + j], e, l);
+        mrow[j] = e;
+      }
+      const float il = 1.f / l;
+      for (int j = 0; j < J; ++j) mrow[j] *= il;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < nrow * (HD / 2); idx += FAST_THREADS) {
+      const int dd = (idx % (HD / 2)) * 2, row = idx / (HD / 2), r = row % R, it2 = row / R;
+      const int hl = it2 / nb, tok = (it2 % nb) * R + r;
+      const float* mrow = wj + (size_t)row * 2 * J;
+      const float* src = P.attn_part + ((size_t)(slice * hps + hl) * FAST_MAX_T + tok) * (HD + 2) + dd;
+      const size_t jstride = (size_t)P.m.o_split * hps * FAST_MAX_T * (HD + 2);
+      float o0 = 0.f, o1 = 0.f;
+#pragma unroll 4
+      for (int j = 0; j < J; ++j) {  // fixed order
+        const float2 ov = __ldcg(reinterpret_cast<const float2*>(src + (size_t)j * jstride));
+        o0 = fmaf(ov.x, mrow[j], o0);
+        o1 = fmaf(ov.y, mrow[j], o1);
+      }
+      write_frag_pair<T16, LO>(osm, tok, hl * HD + dd, o0, o1);
+    }
+    __syncthreads();
+  }
 
   // O projection of this CTA's tiles over the slice's KS k-steps
   const uint32_t o_lane = smem_u32(osm) + lane * (W * 4);
@@ -998,10 +1080,11 @@ struct PhaseCtx {
   float qscale;
   int dk0, dk1, dsl;  // K slice of the down projection this CTA works on
   int qd;
+  uint32_t ks_base;   // key-split variant: value of this slice's arrival counter at the launch's start
 };
 
 // Phase PH of layer l: 0 QKV, 1 attention + O projection, 2 gate/up, 3 down, 4 LM head.
-template <int PH, bool T16, bool LO>
+template <int PH, bool T16, bool LO, bool KSPLIT>
 __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint8_t* uni, Ring& ring,
                                           const PhaseCtx& C, int l, uint32_t& stage_parity) {
   const int d = P.d;
@@ -1022,9 +1105,9 @@ __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint
     D.op = FOP_O; D.epi = EPI_F_RESID;
     D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
     D.cinc = (int)blockIdx.x % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
-    if (P.hd == 64) attn_o_phase<64, T16, LO>(P, M, uni, ring, D, l);
-    else if (P.hd == 128) attn_o_phase<128, T16, LO>(P, M, uni, ring, D, l);
-    else attn_o_phase<32, T16, LO>(P, M, uni, ring, D, l);
+    if (P.hd == 64) attn_o_phase<64, T16, LO, KSPLIT>(P, M, uni, ring, D, l, C.ks_base);
+    else if (P.hd == 128) attn_o_phase<128, T16, LO, KSPLIT>(P, M, uni, ring, D, l, C.ks_base);
+    else attn_o_phase<32, T16, LO, KSPLIT>(P, M, uni, ring, D, l, C.ks_base);
     return;
   }
   if (PH == 0) {
@@ -1047,7 +1130,7 @@ __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint
 
 // ---- the kernel --------------------------------------------------------------------------------
 
-template <bool T16, bool LO, bool TRACE>
+template <bool T16, bool LO, bool TRACE, bool KSPLIT>
 __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __grid_constant__ FastParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, cta = blockIdx.x;
@@ -1102,6 +1185,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   __syncwarp();  // also orders this warp's chunk table before its first use
   for (int s = 0; s < P.nslot; ++s) ring_request(ring, (uint32_t)s, lane);
   const uint32_t epoch_base = ld_acquire_u32(P.epoch_base);
+  // key-split variant: the slice counters are quiet between launches, and no CTA gets past the
+  // first grid barrier before every CTA has read its slice's value here
+  const uint32_t ks_base = KSPLIT ? ld_acquire_u32(P.attn_cnt + cta % P.m.o_split) : 0u;
   uint32_t epoch = 0;
   __syncthreads();
   trace_mark<TRACE>(P, n_trace);
@@ -1159,7 +1245,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   // own call site, so that what a phase is (its projection, input, epilogue) is known at compile
   // time there: every instruction between two barriers is on the critical path.
   const int n_ssq = (d + SSQ_COLS - 1) / SSQ_COLS * FAST_MAX_T;
-  const PhaseCtx C{qscale, dk0, dk1, dsl, qd};
+  const PhaseCtx C{qscale, dk0, dk1, dsl, qd, ks_base};
 #pragma unroll 1
   for (int l = 0; l < P.L && ok; ++l) {
     if (l + 1 < P.L && cta == l % P.m.n_cta) {
@@ -1175,30 +1261,30 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
     // during the QKV phase, the one the down projection adds to during the attention + O phase.
     if (cta == P.m.n_cta - 1)
       for (int i = tid; i < n_ssq; i += FAST_THREADS) P.ssq_b[i] = 0;
-    run_phase<0, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    run_phase<0, T16, LO, KSPLIT>(P, M, uni, ring, C, l, stage_parity);
     trace_mark<TRACE>(P, n_trace);
     ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
     trace_mark<TRACE>(P, n_trace);
     if (!ok) break;
     if (cta == P.m.n_cta - 1)
       for (int i = tid; i < n_ssq; i += FAST_THREADS) P.ssq_a[i] = 0;
-    run_phase<1, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    run_phase<1, T16, LO, KSPLIT>(P, M, uni, ring, C, l, stage_parity);
     trace_mark<TRACE>(P, n_trace);
     ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
     trace_mark<TRACE>(P, n_trace);
     if (!ok) break;
-    run_phase<2, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    run_phase<2, T16, LO, KSPLIT>(P, M, uni, ring, C, l, stage_parity);
     trace_mark<TRACE>(P, n_trace);
     ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
     trace_mark<TRACE>(P, n_trace);
     if (!ok) break;
-    run_phase<3, T16, LO>(P, M, uni, ring, C, l, stage_parity);
+    run_phase<3, T16, LO, KSPLIT>(P, M, uni, ring, C, l, stage_parity);
     trace_mark<TRACE>(P, n_trace);
     ok = grid_sync(P, epoch_base + (++epoch) * (uint32_t)P.m.n_cta, ring.dead);
     trace_mark<TRACE>(P, n_trace);
   }
   if (ok && P.logits) {
-    run_phase<4, T16, LO>(P, M, uni, ring, C, 0, stage_parity);
+    run_phase<4, T16, LO, KSPLIT>(P, M, uni, ring, C, 0, stage_parity);
     trace_mark<TRACE>(P, n_trace);
     if (__syncthreads_or(ring.dead ? 1 : 0)) ok = false;
   }
@@ -1222,7 +1308,13 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
 // The kernel variant for a launch, from the translation unit that instantiates it.
 template <bool T16, bool LO>
 inline const void* fast_kernel_variant(bool trace) {
-  return trace ? (const void*)fast_forward_kernel<T16, LO, true> : (const void*)fast_forward_kernel<T16, LO, false>;
+  return trace ? (const void*)fast_forward_kernel<T16, LO, true, false>
+               : (const void*)fast_forward_kernel<T16, LO, false, false>;
+}
+// The key-split variant (long prefixes): split activations, no trace.
+template <bool T16>
+inline const void* fast_kernel_keysplit_variant() {
+  return (const void*)fast_forward_kernel<T16, true, false, true>;
 }
 
 }  // namespace

@@ -9,6 +9,7 @@ const void* fast_kernel_r8_split(bool trace);
 const void* fast_kernel_r8_bf16(bool trace);
 const void* fast_kernel_r16_split(bool trace);
 const void* fast_kernel_r16_bf16(bool trace);
+const void* fast_kernel_keysplit(bool t16);
 size_t fast_misc_bytes();  // per-CTA bookkeeping of the kernel in shared memory
 
 size_t fast_union_bytes(int stage_k, int hd, int T, int o_steps, bool split) {
@@ -45,6 +46,8 @@ cudaError_t launch_fast_forward(const FastParams& p_in, cudaStream_t st) {
   // the phase trace is a variant of its own: the common path carries no trace code
   const void* kern = p.split_act ? (t16 ? fast_kernel_r16_split(p.trace != nullptr) : fast_kernel_r8_split(p.trace != nullptr))
                                  : (t16 ? fast_kernel_r16_bf16(p.trace != nullptr) : fast_kernel_r8_bf16(p.trace != nullptr));
+  // long prefixes: the variant whose CTAs split the keys of a head instead of all walking them
+  if (p.key_split && p.split_act && !p.trace && p.attn_part && p.attn_cnt) kern = fast_kernel_keysplit(t16);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   void* args[] = {(void*)&p};

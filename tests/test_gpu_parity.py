@@ -208,6 +208,20 @@ def test_persistent_kernel_with_several_heads_per_o_slice():
     _case(_wl(shape, 3, 4, [17, 90, 33]), beta=0.0, sigma=0.5, path=0, logit_tol=2e-4)      # 15 rows
 
 
+@pytest.mark.parametrize("hd,hq,batch,gamma,lens", [
+    (64, 14, 1, 4, [900]), (64, 14, 2, 2, [5, 700]), (32, 32, 2, 3, [40, 650]), (128, 4, 3, 4, [1, 129, 1000]),
+    (64, 14, 1, 15, [333])])
+def test_persistent_kernel_key_split_variant(hd, hq, batch, gamma, lens):
+    """Streams created with room for >= 768 tokens run the variant whose CTAs share a head's keys
+    (each walks every J-th 128-key pass, partials merged after a meeting of the slice's CTAs):
+    long and very short prefixes (CTAs with no pass at all), one and two heads per slice, <= 8 and
+    <= 16 rows, with a commit and a second step on the same streams."""
+    shape = _fast_shape(hd, hq=hq, hkv=2 if hq != 32 else 4)
+    wl = _wl(shape, batch, gamma, lens)
+    _case(wl, beta=0.4, sigma=1.0, commit_and_repeat=True, path=0, logit_tol=2e-4, capacity=1100)
+    _case(wl, beta=0.0, sigma=0.5, path=0, logit_tol=2e-4, capacity=2048)
+
+
 def test_generic_kernels_still_cover_small_bf16_forwards():
     shape = _fast_shape(64, hq=14, hkv=2)
     _case(_wl(shape, 2, 4, [70, 129]), beta=0.0, sigma=0.5, path=1)
