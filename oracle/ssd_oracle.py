@@ -12,9 +12,11 @@ What is computed, and from which passage:
                    "Transformer adapted from Qwen2.5" of Sec. 3.1: pre-norm RMSNorm, grouped-query
                    attention with biased q/k/v projections and rotate-half RoPE, SiLU-gated
                    feed-forward, final RMSNorm, untied LM head.
-* `transform`    - temperature and top-k applied to a logit row before softmax.  The paper does
-                   not describe a sampler; this is the workload's (stated reading: z/T, keep the
-                   top_k largest with the lower id winning ties, softmax over what is kept).
+* `transform`    - temperature, top-k and nucleus (top-p) applied to a logit row before softmax.
+                   The paper does not describe a sampler; this is the workload's (stated reading:
+                   z/T, keep the top_k largest with the lower id winning ties, then the shortest
+                   prefix of those, most probable first, whose mass reaches top_p; softmax over
+                   what is kept).
 * `accept_step`  - the sequential tolerance test r_i < min(1, q_i(x_i)/p_i(x_i)) + beta (Eq. 5),
                    the residual resample from normalize(max(0, q_i - p_i)) at the first rejection
                    (Eq. 6), and the bonus token from q_{gamma+1} when nothing is rejected
@@ -168,16 +170,31 @@ def prefill(model: Model, stream: Stream, ids: np.ndarray, chunk: int = 64) -> N
 
 # ------------------------------------------------------------------ sampling transform
 
-def transform(logits_row: np.ndarray, temperature: float, top_k: int) -> np.ndarray:
-    """Logit row -> the distribution the target's sampler draws from (q_i in Eq. 5-6)."""
+def transform(logits_row: np.ndarray, temperature: float, top_k: int, top_p: float = 0.0) -> np.ndarray:
+    """Logit row -> the distribution the target's sampler draws from (q_i in Eq. 5-6).
+
+    z = logits / T; keep the top_k largest (lower id wins ties; top_k <= 0 or >= V: all); then,
+    with 0 < top_p < 1, the nucleus: walking the kept ids from the most to the least probable
+    (lower id first among equals), an id stays while the mass of the ids before it is below
+    top_p, i.e. the shortest such prefix whose mass reaches top_p; softmax over what is left.
+    """
     z = np.asarray(logits_row, F64) / float(temperature)
     V = z.shape[0]
+    order = np.argsort(-z, kind="stable")            # equal values: lower id first
+    keep = np.ones(V, dtype=bool)
     if 0 < top_k < V:
-        order = np.argsort(-z, kind="stable")        # equal values: lower id first
-        keep = np.zeros(V, dtype=bool)
+        keep[:] = False
         keep[order[:top_k]] = True
-    else:
-        keep = np.ones(V, dtype=bool)
+    if 0.0 < top_p < 1.0:
+        e = np.where(keep, np.exp(z - z[keep].max()), 0.0)
+        prob = e / e.sum()
+        before = 0.0
+        for t in order:                              # kept ids come first in this order
+            if not keep[t]:
+                break
+            if before >= top_p:
+                keep[t] = False
+            before += prob[t]
     e = np.where(keep, np.exp(z - z[keep].max()), 0.0)
     return e / e.sum()
 
@@ -234,12 +251,12 @@ def accept_step(q_rows: np.ndarray, p_rows: np.ndarray, draft_tokens: np.ndarray
 
 
 def verify(model: Model, stream: Stream, draft_tokens: np.ndarray, p_rows: np.ndarray,
-           uniforms: np.ndarray, *, temperature: float, top_k: int, beta: float
+           uniforms: np.ndarray, *, temperature: float, top_k: int, beta: float, top_p: float = 0.0
            ) -> Dict[str, object]:
     """One full verification step for one stream (forward, transform, accept); no commit."""
     ids = np.concatenate([[stream.pending], np.asarray(draft_tokens, np.int64)])
     logits = forward(model, stream, ids)
-    q_rows = np.stack([transform(row, temperature, top_k) for row in logits])
+    q_rows = np.stack([transform(row, temperature, top_k, top_p) for row in logits])
     res = accept_step(q_rows, p_rows, draft_tokens, uniforms, beta)
     res["logits"] = logits
     res["q_rows"] = q_rows

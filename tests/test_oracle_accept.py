@@ -203,6 +203,77 @@ def test_transform_against_torch_and_special_cases():
     assert orc.transform(z, 1e-3, 0).argmax() == z.argmax()
 
 
+def test_nucleus_transform_by_hand_brute_force_and_library():
+    """top-p keeps the shortest most-probable-first prefix whose mass reaches top_p."""
+    # by hand: probabilities 0.5, 0.3, 0.15, 0.05 (ids shuffled)
+    pr = np.array([0.15, 0.5, 0.05, 0.3])
+    z = np.log(pr)
+    assert list(np.nonzero(orc.transform(z, 1.0, 0, 0.79))[0]) == [1, 3]          # 0.5 + 0.3 reaches 0.79
+    assert list(np.nonzero(orc.transform(z, 1.0, 0, 0.81))[0]) == [0, 1, 3]       # needs the third
+    assert list(np.nonzero(orc.transform(z, 1.0, 0, 0.4))[0]) == [1]
+    q = orc.transform(z, 1.0, 0, 0.79)
+    assert np.allclose(q[[1, 3]], [0.5 / 0.8, 0.3 / 0.8]) and np.isclose(q.sum(), 1.0)
+    assert np.allclose(orc.transform(z, 1.0, 0, 0.0), pr) and np.allclose(orc.transform(z, 1.0, 0, 1.0), pr)
+    # ties: equal probabilities enter in id order
+    zt = np.log(np.array([0.25, 0.25, 0.25, 0.25]))
+    assert list(np.nonzero(orc.transform(zt, 1.0, 0, 0.5))[0]) == [0, 1]
+    assert list(np.nonzero(orc.transform(zt, 1.0, 0, 0.51))[0]) == [0, 1, 2]
+    # after top-k the nucleus is taken inside the kept set (mass relative to that set)
+    assert list(np.nonzero(orc.transform(z, 1.0, 2, 0.7))[0]) == [1, 3]            # 0.5/0.8 = 0.625 < 0.7
+    assert list(np.nonzero(orc.transform(z, 1.0, 2, 0.6))[0]) == [1]
+    # brute force: among all most-probable-first prefixes, the shortest with mass >= top_p
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        V = int(rng.integers(2, 9))
+        zz = rng.standard_normal(V) * 2
+        T = float(rng.uniform(0.5, 1.5))
+        top_p = float(rng.uniform(0.05, 0.98))
+        full = orc.transform(zz, T, 0)
+        order = np.argsort(-full, kind="stable")
+        n = next(i + 1 for i in range(V) if full[order[:i + 1]].sum() >= top_p or i == V - 1)
+        got = orc.transform(zz, T, 0, top_p)
+        assert set(np.nonzero(got)[0]) == set(order[:n].tolist())
+        assert np.allclose(got[order[:n]], full[order[:n]] / full[order[:n]].sum())
+    # library routine: the nucleus filter of `transformers`
+    from transformers.generation.logits_process import TopPLogitsWarper
+    for seed in range(20):
+        zz = np.random.default_rng(seed).standard_normal(64) * 2.5
+        tp = 0.3 + 0.03 * seed
+        kept_ref = torch.isfinite(TopPLogitsWarper(top_p=tp)(None, torch.from_numpy(zz)[None].clone()))[0].numpy()
+        assert np.array_equal(orc.transform(zz, 1.0, 0, tp) > 0, kept_ref)
+
+
+def test_accepted_length_grows_with_beta_as_in_table_3():
+    """Sec. 4.3 / Table 3: a larger tolerance accepts more.  For fixed distributions, tokens and
+    uniforms k(beta) never decreases, and its mean over draws follows the geometric closed form
+    with the per-position acceptance probability A = sum_x p(x) min(1, min(1, q/p) + beta)."""
+    rng = np.random.default_rng(5)
+    V, gamma, n = 12, 3, 4000
+    q = rng.dirichlet(np.ones(V) * 0.7)
+    p = rng.dirichlet(np.ones(V) * 0.7)
+    qs, ps = np.tile(q, (gamma + 1, 1)), np.tile(p, (gamma, 1))
+    means = []
+    for beta in (0.0, 0.1, 0.2, 0.3, 0.4):
+        ks = []
+        for i in range(n):
+            r = np.random.default_rng(1000 + i)
+            x = r.choice(V, size=gamma, p=p)
+            u = r.random((gamma + 1, 2))
+            ks.append(orc.accept_step(qs, ps, x, u, beta)["k"])
+        means.append(np.mean(ks))
+        A = float(np.sum(p * np.minimum(1.0, np.minimum(1.0, q / p) + beta)))
+        closed = sum(A ** j for j in range(1, gamma + 1))          # E[k] = A + A^2 + ... + A^gamma
+        assert abs(means[-1] - closed) < 4 * np.sqrt(gamma / n) + 0.02
+    assert all(b >= a for a, b in zip(means, means[1:])) and means[-1] > means[0] + 0.3
+    # same draws, larger beta: never fewer accepted
+    for i in range(200):
+        r = np.random.default_rng(i)
+        x = r.choice(V, size=gamma, p=p)
+        u = r.random((gamma + 1, 2))
+        kk = [orc.accept_step(qs, ps, x, u, b)["k"] for b in (0.0, 0.1, 0.2, 0.3, 0.4, 1.0)]
+        assert kk == sorted(kk) and kk[-1] == gamma
+
+
 def test_expected_tokens_per_iteration_geometric_identity():
     """With i.i.d. acceptance probability alpha, E[k+1] = (1 - alpha^(gamma+1)) / (1 - alpha)."""
     V, gamma, alpha = 4, 4, 0.5
