@@ -344,7 +344,8 @@ def run_cuda(args):
     assert np.array_equal(h_k.numpy(), k_timed), "host-buffer path disagrees with the device path"
     loop_stats = None
     if args.loop_iterations > 0:
-        loop_stats = {str(beta): run_loop(args, wl, model, dev, beta) for beta in (0.0, args.beta)}
+        betas = (0.0, 0.1, 0.2, 0.3, 0.4) if args.beta_sweep else (0.0, args.beta)
+        loop_stats = {str(beta): run_loop(args, wl, model, dev, beta) for beta in dict.fromkeys(betas + (args.beta,))}
 
     dev_ms, e2e_ms, fwd_ms = replicas.slowest([dev_ms, e2e_ms, fwd_ms], world, dev)   # max over ranks
     if rank != 0:
@@ -423,6 +424,8 @@ def main():
     ap.add_argument("--prefix", type=int, default=None, help="prefix length (config 2's sweep)")
     ap.add_argument("--draft-noise", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--beta-sweep", action="store_true",
+                    help="run the loop at beta = 0, 0.1 .. 0.4 (the sweep of the paper's Table 3, cost side)")
     ap.add_argument("--loop-iterations", type=int, default=200,
                     help="SSD iterations timed for the tokens/s figure (0: skip the loop)")
     ap.add_argument("--synthetic-kv", action="store_true",

@@ -86,6 +86,9 @@ typedef struct {
   float temperature; /* > 0; logits are divided by it */
   int32_t top_k;     /* <= 0 or >= vocab_out: off; else keep the top_k largest (lower id wins ties) */
   float beta;        /* tolerance factor of Eq. 5, >= 0 */
+  float top_p;       /* nucleus: 0 or >= 1: off; else, among the ids top_k kept, most probable first
+                        (lower id first among equals), an id stays while the mass before it is
+                        below top_p: the shortest such prefix whose mass reaches top_p */
 } ssd_verify_params;
 
 /* ---- model ------------------------------------------------------------------------------- */

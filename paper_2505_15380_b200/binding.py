@@ -41,7 +41,7 @@ class ModelConfig(ctypes.Structure):
 
 class VerifyParams(ctypes.Structure):
     _fields_ = [("gamma", ctypes.c_int32), ("temperature", ctypes.c_float),
-                ("top_k", ctypes.c_int32), ("beta", ctypes.c_float)]
+                ("top_k", ctypes.c_int32), ("beta", ctypes.c_float), ("top_p", ctypes.c_float)]
 
 
 class LoopIo(ctypes.Structure):

@@ -415,7 +415,7 @@ int draft_step_impl(ssd_model* draft, ssd_streams* ds, const int32_t* ids, int n
   if (rc != SSD_OK) return rc;
   launch_advance_all(ds->len, ds->B, n_in, ds->cap, ds->status, st);
   SSD_CUDA(launch_draft_sampler(ds->logits + (size_t)(n_in - 1) * V, n_in * V, V, uniform, ds->B,
-                                1.0f / params->temperature, params->top_k, out_token, tok_stride, out_prob,
+                                1.0f / params->temperature, params->top_k, params->top_p, out_token, tok_stride, out_prob,
                                 prob_stride, ds->pending, ds->status, st));
   return SSD_OK;
 }
@@ -425,6 +425,7 @@ int params_ok(const ssd_streams* s, const ssd_verify_params* p, bool need_gamma)
   if (need_gamma && (p->gamma < 1 || p->gamma > s->max_gamma)) return SSD_ERR_BAD_GAMMA;
   if (!(p->temperature > 0.f) || !isfinite(p->temperature)) return SSD_ERR_BAD_PARAM;
   if (!(p->beta >= 0.f) || !isfinite(p->beta)) return SSD_ERR_BAD_PARAM;
+  if (!(p->top_p >= 0.f) || !isfinite(p->top_p)) return SSD_ERR_BAD_PARAM;
   return SSD_OK;
 }
 
@@ -864,7 +865,7 @@ int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_token
   if (rc != SSD_OK) return rc;
   SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
                                  dev_uniforms, s->B, gamma, 1.0f / params->temperature,
-                                 params->top_k, params->beta, s->row_stats, s->accept_flags,
+                                 params->top_k, params->top_p, params->beta, s->row_stats, s->accept_flags,
                                  s->counters, dev_accepted_len, dev_next_token, s->status, st));
   return SSD_OK;
 }

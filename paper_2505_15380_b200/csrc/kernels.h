@@ -48,16 +48,17 @@ cudaError_t launch_attention_simt(int dtype, const float* qrot, const void* kv_l
 // sampler.cu
 cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* draft_tokens,
                                   const float* draft_probs, const float* uniforms, int B,
-                                  int gamma, float inv_temperature, int top_k, float beta,
+                                  int gamma, float inv_temperature, int top_k, float top_p, float beta,
                                   float* row_stats, int32_t* accept_flags, int32_t* counters,
                                   int32_t* accepted_len, int32_t* next_token, int32_t* status,
                                   cudaStream_t st);
 // out_token[b * tok_stride] and out_prob_row[b * prob_stride + t]: the strides let a loop write
 // step i of every stream straight into the [B, gamma] / [B, gamma, V] arrays the verifier reads.
 cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, const float* uniform,
-                                 int B, float inv_temperature, int top_k, int32_t* out_token,
-                                 int tok_stride, float* out_prob_row, size_t prob_stride,
-                                 int32_t* pending, int32_t* status, cudaStream_t st);
+                                 int B, float inv_temperature, int top_k, float top_p,
+                                 int32_t* out_token, int tok_stride, float* out_prob_row,
+                                 size_t prob_stride, int32_t* pending, int32_t* status,
+                                 cudaStream_t st);
 
 // loop.cu: bookkeeping kernels of the device-resident SSD iteration
 void launch_loop_stage_uniforms(const float* pool, int n_rows, const int32_t* iteration, int B, int gamma,

@@ -51,7 +51,24 @@ __device__ __forceinline__ double block_sum_d(double v, double* red) {
   return r;
 }
 
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long r = 0;
+  for (int i = 0; i < SAMP_THREADS / 32; ++i) r += red[i];
+  __syncthreads();
+  return r;
+}
+// Mass exp(x), x <= 0, in units of 2^-32: integer sums of these do not depend on the order of
+// the additions, so the nucleus cut is the same in every run.
+__device__ __forceinline__ unsigned long long mass_fx(float x) { return __float2ull_rn(expf(x) * 4294967296.f); }
+
 struct SampSmem {
+  unsigned long long hist_fx[256];
+  unsigned long long red_u[SAMP_THREADS / 32];
+  unsigned long long mass_above;
   double red_d[SAMP_THREADS / 32];
   double scan[SAMP_THREADS];
   float red_f[SAMP_THREADS / 32];
@@ -61,7 +78,7 @@ struct SampSmem {
 };
 
 // Row statistics of the sampling transform: z/T is already in `z` (shared).  Block-collective.
-__device__ RowStats compute_row_stats(const float* z, int V, int top_k, SampSmem& sm) {
+__device__ RowStats compute_row_stats(const float* z, int V, int top_k, float top_p, SampSmem& sm) {
   RowStats st;
   float mx = -CUDART_INF_F;
   for (int t = threadIdx.x; t < V; t += SAMP_THREADS) mx = fmaxf(mx, z[t]);
@@ -105,6 +122,74 @@ __device__ RowStats compute_row_stats(const float* z, int V, int top_k, SampSmem
       __syncthreads();
       st.tie_id_max = sm.tie_id;
     }
+    __syncthreads();
+  }
+  if (top_p > 0.f && top_p < 1.f) {
+    // Nucleus: walking the kept ids from the most to the least probable (lower id first among
+    // equals), an id stays while the mass before it is below top_p of the kept mass.  The id at
+    // which the running mass first reaches that target is found by a radix select over the
+    // ordered keys with histograms of mass instead of counts.
+    unsigned long long mine = 0;
+    for (int t = threadIdx.x; t < V; t += SAMP_THREADS)
+      if (is_kept(z[t], t, st)) mine += mass_fx(z[t] - st.zmax);
+    const unsigned long long total = block_sum_u64(mine, sm.red_u);
+    const double td = (double)top_p * (double)total;
+    unsigned long long target = (unsigned long long)td;
+    if ((double)target < td) ++target;  // an id stays iff (mass before it) < target
+    if (target < 1) target = 1;
+    if (threadIdx.x == 0) { sm.prefix = 0u; sm.mass_above = 0; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int i = threadIdx.x; i < 256; i += SAMP_THREADS) { sm.hist_fx[i] = 0; sm.hist[i] = 0; }
+      __syncthreads();
+      const uint32_t prefix = sm.prefix;
+      const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+      for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
+        const uint32_t k = order_key(z[t]);
+        if ((k & mask) == prefix && is_kept(z[t], t, st)) {
+          atomicAdd(&sm.hist_fx[(k >> shift) & 0xFF], mass_fx(z[t] - st.zmax));
+          atomicAdd(&sm.hist[(k >> shift) & 0xFF], 1);
+        }
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        unsigned long long acc = sm.mass_above;
+        int bin = 255;
+        for (; bin > 0; --bin) {
+          if (acc + sm.hist_fx[bin] >= target) break;
+          acc += sm.hist_fx[bin];
+        }
+        sm.prefix = prefix | ((uint32_t)bin << shift);
+        sm.mass_above = acc;
+        sm.eq_count = sm.hist[bin];
+      }
+      __syncthreads();
+    }
+    const uint32_t cut = sm.prefix;
+    int tie_id = st.thr_key == cut ? st.tie_id_max : V;  // ties already trimmed by the top-k cut
+    if (threadIdx.x == 0) {
+      // ids with the cut's value have equal mass: as many of them as it takes to reach the target
+      sm.tie_id = tie_id;
+      if (sm.eq_count > 1) {
+        unsigned long long each = 0;
+        int first = -1;
+        for (int t = 0; t < V && first < 0; ++t)
+          if (order_key(z[t]) == cut && is_kept(z[t], t, st)) first = t;
+        each = first >= 0 ? mass_fx(z[first] - st.zmax) : 1;
+        if (each < 1) each = 1;
+        unsigned long long need = (target - sm.mass_above + each - 1) / each;
+        if (need < 1) need = 1;
+        if (need < (unsigned long long)sm.eq_count) {
+          int t = first;
+          for (; t < V; ++t)
+            if (order_key(z[t]) == cut && is_kept(z[t], t, st) && --need == 0) break;
+          sm.tie_id = t;
+        }
+      }
+    }
+    __syncthreads();
+    st.thr_key = cut;
+    st.tie_id_max = sm.tie_id;
     __syncthreads();
   }
   double s = 0.0;
@@ -183,7 +268,7 @@ __global__ void __launch_bounds__(SAMP_THREADS)
 verify_sampler_kernel(const float* __restrict__ logits, int V,
                       const int32_t* __restrict__ draft_tokens,
                       const float* __restrict__ draft_probs, const float* __restrict__ uniforms,
-                      int gamma, float inv_t, int top_k, float beta, float* row_stats,
+                      int gamma, float inv_t, int top_k, float top_p, float beta, float* row_stats,
                       int32_t* accept_flags, int32_t* counters, int32_t* __restrict__ accepted_len,
                       int32_t* __restrict__ next_token, int32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -202,7 +287,7 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
   if (bad) sm.bad = 1;
   __syncthreads();
   if (sm.bad && threadIdx.x == 0) atomicOr(status, SSD_STATUS_NONFINITE);
-  RowStats st = compute_row_stats(z, V, top_k, sm);
+  RowStats st = compute_row_stats(z, V, top_k, top_p, sm);
   if (threadIdx.x == 0) {
     int flag = 0;
     if (r < gamma) {  // Eq. 5: accept x_i iff r_i < min(1, q_i(x_i) / p_i(x_i)) + beta
@@ -281,7 +366,7 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
 
 cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* draft_tokens,
                                   const float* draft_probs, const float* uniforms, int B,
-                                  int gamma, float inv_temperature, int top_k, float beta,
+                                  int gamma, float inv_temperature, int top_k, float top_p, float beta,
                                   float* row_stats, int32_t* accept_flags, int32_t* counters,
                                   int32_t* accepted_len, int32_t* next_token, int32_t* status,
                                   cudaStream_t st) {
@@ -294,7 +379,7 @@ cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* dra
   }
   dim3 grid(gamma + 1, B);
   verify_sampler_kernel<<<grid, SAMP_THREADS, smem, st>>>(
-      logits, V, draft_tokens, draft_probs, uniforms, gamma, inv_temperature, top_k, beta,
+      logits, V, draft_tokens, draft_probs, uniforms, gamma, inv_temperature, top_k, top_p, beta,
       row_stats, accept_flags, counters, accepted_len, next_token, status);
   count_launch();
   return cudaGetLastError();
@@ -304,7 +389,7 @@ cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* dra
 // because the verifier needs the whole row (Eq. 6).  One CTA per stream.
 __global__ void __launch_bounds__(SAMP_THREADS)
 draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
-                     const float* __restrict__ uniform, float inv_t, int top_k,
+                     const float* __restrict__ uniform, float inv_t, int top_k, float top_p,
                      int32_t* __restrict__ out_token, int tok_stride, float* __restrict__ out_prob,
                      size_t prob_stride, int32_t* pending, int32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -323,7 +408,7 @@ draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
   if (bad) sm.bad = 1;
   __syncthreads();
   if (sm.bad && threadIdx.x == 0) atomicOr(status, SSD_STATUS_NONFINITE);
-  RowStats st = compute_row_stats(z, V, top_k, sm);
+  RowStats st = compute_row_stats(z, V, top_k, top_p, sm);
   for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
     float p = is_kept(z[t], t, st) ? expf(z[t] - st.zmax) / st.sum : 0.f;
     z[t] = p;
@@ -340,9 +425,10 @@ draft_sampler_kernel(const float* __restrict__ logits, int ld_logits, int V,
 }
 
 cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, const float* uniform,
-                                 int B, float inv_temperature, int top_k, int32_t* out_token,
-                                 int tok_stride, float* out_prob_row, size_t prob_stride,
-                                 int32_t* pending, int32_t* status, cudaStream_t st) {
+                                 int B, float inv_temperature, int top_k, float top_p,
+                                 int32_t* out_token, int tok_stride, float* out_prob_row,
+                                 size_t prob_stride, int32_t* pending, int32_t* status,
+                                 cudaStream_t st) {
   size_t smem = sizeof(SampSmem) + (size_t)V * sizeof(float);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   if (smem > 48 * 1024) {
@@ -351,7 +437,7 @@ cudaError_t launch_draft_sampler(const float* logits, int ld_logits, int V, cons
     if (e != cudaSuccess) return e;
   }
   draft_sampler_kernel<<<B, SAMP_THREADS, smem, st>>>(logits, ld_logits, V, uniform,
-                                                      inv_temperature, top_k, out_token, tok_stride,
+                                                      inv_temperature, top_k, top_p, out_token, tok_stride,
                                                       out_prob_row, prob_stride, pending, status);
   count_launch();
   return cudaGetLastError();
@@ -458,7 +544,7 @@ extern "C" int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_dr
   if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: cudaMemsetAsync");
   e = ssd::launch_verify_sampler(dev_logits, vocab, dev_draft_tokens, dev_draft_probs, dev_uniforms,
                                  batch, params->gamma, 1.0f / params->temperature, params->top_k,
-                                 params->beta, sc->row_stats, sc->accept_flags, sc->counters,
+                                 params->top_p, params->beta, sc->row_stats, sc->accept_flags, sc->counters,
                                  dev_accepted_len, dev_next_token, &sc->status, st);
   if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: launch");
   return SSD_OK;

@@ -72,6 +72,16 @@ def _topk_gap_small(logits_row: np.ndarray, temperature: float, top_k: int) -> b
     return bool(z[top_k - 1] - z[top_k] < TOPK_GAP)
 
 
+def _nucleus_edge_close(logits_row: np.ndarray, temperature: float, top_k: int, top_p: float) -> bool:
+    """True when the running mass at the nucleus cut lies within 1e-5 of top_p: fp32 rounding of
+    the masses may then move the cut by one id."""
+    if not (0.0 < top_p < 1.0):
+        return False
+    full = np.sort(orc.transform(logits_row, temperature, top_k))[::-1]
+    cum = np.cumsum(full)
+    return bool(np.min(np.abs(cum - top_p)) < 1e-5)
+
+
 def _draw_interval(q_row: np.ndarray, p_row: Optional[np.ndarray], y: int):
     """[lo, hi) of token y in the normalised CDF the new token is drawn from: the residual
     max(0, q - p) after a rejection (q itself when that has no mass), q for the bonus token."""
@@ -98,7 +108,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
              oracle_streams: Optional[List[int]] = None, logit_tol: Optional[float] = None,
              uniform_seed: int = 0, commit_and_repeat: bool = False,
              capacity: Optional[int] = None, path: int = 0, split: bool = True,
-             max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34) -> CaseResult:
+             max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34, top_p: float = 0.0) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -156,7 +166,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
                 draft[b, i] = tok
             st.length = base_len
         # ---- GPU
-        params = binding.VerifyParams(gamma, wl.temperature, wl.top_k, beta)
+        params = binding.VerifyParams(gamma, wl.temperature, wl.top_k, beta, top_p)
         d_tok = torch.from_numpy(draft.astype(np.int32)).to(dev)
         d_p = torch.from_numpy(p_rows.astype(np.float32)).to(dev)
         d_u = torch.from_numpy(uni).to(dev)
@@ -177,13 +187,13 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
         for b in which:
             st = ostreams[b]
             o = orc.verify(omodel, st, draft[b], p_rows[b], uni[b], temperature=wl.temperature,
-                           top_k=wl.top_k, beta=beta)
+                           top_k=wl.top_k, beta=beta, top_p=top_p)
             err = float(np.abs(o["logits"] - g_logits[b]).max())
             res.max_logit_err = max(res.max_logit_err, err)
             assert err <= logit_tol, f"stream {b}: logits differ by {err}"
             # strict: oracle arithmetic on the GPU's logits
             gl = g_logits[b].astype(np.float64)
-            q_g = np.stack([orc.transform(r, wl.temperature, wl.top_k) for r in gl])
+            q_g = np.stack([orc.transform(r, wl.temperature, wl.top_k, top_p) for r in gl])
             o2 = orc.accept_step(q_g, p_rows[b], draft[b], uni[b], beta)
             res.n_streams += 1
             res.ks.append(int(g_k[b]))
@@ -191,13 +201,15 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
             n_eval = min(o2["k"] + 1, gamma)
             for i in range(n_eval):
                 if abs(o2["thresholds"][i] - float(uni[b, i, 0])) < WINDOW or \
-                        _topk_gap_small(gl[i], wl.temperature, wl.top_k):
+                        _topk_gap_small(gl[i], wl.temperature, wl.top_k) or \
+                        _nucleus_edge_close(gl[i], wl.temperature, wl.top_k, top_p):
                     strict_excl = True
                     break
             if not strict_excl:
                 assert g_k[b] == o2["k"], f"stream {b}: accepted length {g_k[b]} vs {o2['k']}"
-                if o2["draw_margin"] < DRAW_WINDOW or _topk_gap_small(gl[o2["k"]], wl.temperature,
-                                                                      wl.top_k):
+                if o2["draw_margin"] < DRAW_WINDOW or \
+                        _topk_gap_small(gl[o2["k"]], wl.temperature, wl.top_k) or \
+                        _nucleus_edge_close(gl[o2["k"]], wl.temperature, wl.top_k, top_p):
                     strict_excl = True
                 else:
                     assert g_y[b] == o2["y"], f"stream {b}: token {g_y[b]} vs {o2['y']}"

@@ -68,6 +68,48 @@ def test_top_k_and_temperature(top_k, temperature):
     _case(wl, beta=0.4, sigma=1.5)
 
 
+@pytest.mark.parametrize("top_p,top_k,temperature", [(0.8, 25, 0.8), (0.5, 0, 1.0), (0.95, 0, 0.7),
+                                                   (0.05, 10, 1.0)])
+def test_nucleus_sampling_in_the_fused_kernel(top_p, top_k, temperature):
+    """top-p inside the fused acceptance kernel (q rows still never leave the chip), alone and
+    after a top-k cut, down to a nucleus of a single id."""
+    shape = _small(synth.BF16, 64)
+    wl = _wl(shape, 6, 4, [50, 64, 100, 7, 33, 80], temperature=temperature, top_k=top_k)
+    _case(wl, beta=0.0, sigma=0.5, top_p=top_p)
+    _case(wl, beta=0.4, sigma=1.5, top_p=top_p, commit_and_repeat=True)
+    shape32 = _small(synth.F32, 32)
+    _case(_wl(shape32, 6, 3, [20, 30, 40, 50, 60, 70], temperature=temperature, top_k=top_k), beta=0.2,
+          sigma=1.0, top_p=top_p)
+
+
+def test_accepted_length_never_shrinks_with_beta():
+    """Table 3's mechanism on the GPU: with the inputs and uniforms held fixed, a larger
+    tolerance beta accepts at least as many draft tokens, and beta >= 1 accepts all of them."""
+    from paper_2505_15380_b200 import binding
+    shape = _small(synth.BF16, 64)
+    B, g, V = 16, 6, shape.vocab_out
+    model = binding.Model(shape, synth.weights_blob(shape, synth.make_weights(shape, 3)))
+    dev = model.device
+    gs = binding.Streams(model, B, 96, g)
+    lens = [10 + 3 * b for b in range(B)]
+    synth.fill_synthetic_kv(gs.kv, lens, seed=5)
+    gs.kv_truncate(lens, [b % V for b in range(B)])
+    p = synth.random_prob_rows(B * g, V, 4, sharpness=1.0).reshape(B, g, V)
+    x = synth.sample_from_rows(p.reshape(-1, V), 5).reshape(B, g).astype(np.int32)
+    u = synth.verify_uniforms(9, B, g + 1)
+    d_x, d_p, d_u = (torch.from_numpy(a).to(dev) for a in (x, p, u))
+    ks = []
+    for beta in (0.0, 0.1, 0.2, 0.3, 0.4, 1.0):
+        k = torch.zeros(B, dtype=torch.int32, device=dev)
+        y = torch.zeros(B, dtype=torch.int32, device=dev)
+        gs.verify(d_x, d_p, d_u, binding.VerifyParams(g, 1.0, 0, beta), k, y)
+        torch.cuda.synchronize()
+        ks.append(k.cpu().numpy())
+    for a, b in zip(ks, ks[1:]):
+        assert (b >= a).all()
+    assert (ks[-1] == g).all() and ks[0].sum() < ks[4].sum()
+
+
 def test_mha_no_grouping_and_single_kv_head():
     _case(_wl(_small(synth.F32, 32, hq=4, hkv=4), 2, 4, [30, 90]), beta=0.0, sigma=0.5)
     _case(_wl(_small(synth.BF16, 64, hq=8, hkv=1, d=128), 2, 4, [30, 90]), beta=0.0, sigma=0.5)
