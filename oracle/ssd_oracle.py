@@ -24,6 +24,9 @@ What is computed, and from which passage:
                    distribution, as in the paper (the reverse of the usual letters).
 * `commit`       - "append to T_in": the prefix grows by the accepted draft tokens plus the one
                    corrected / bonus token (Algorithm 1).
+* `PagedCache`   - a page pool with per-stream block tables: a layout, not arithmetic; pinned to
+                   give exactly the contiguous cache's results while streams grow, roll back,
+                   leave and join.
 
 State convention: a stream holding n tokens keeps K/V for tokens 0..n-2 (`length` = n-1) and the
 last token as `pending`.  A verify step feeds [pending, x_1..x_gamma] at positions
@@ -273,3 +276,76 @@ def truncate(stream: Stream, new_length: int, pending: int) -> None:
     """Roll the stream back to an earlier prefix; later cache rows become dead."""
     assert 0 <= new_length <= stream.length
     stream.length, stream.pending = int(new_length), int(pending)
+
+
+# ------------------------------------------------------------------ paged cache (layout only)
+
+PAGE_TOKENS = 64
+
+
+class PagedCache:
+    """A pool of fixed-size K/V pages shared by several streams, with a block table per stream.
+
+    The paper says nothing about memory layout: a paged cache must be indistinguishable from the
+    contiguous one (same logits, same decisions) while letting streams of very different lengths
+    share memory, join and leave.  Token t of stream b lives in page table[b][t // PAGE_TOKENS],
+    slot t % PAGE_TOKENS.  Rolling a stream back to `length` tokens returns the pages that lie
+    wholly beyond it to the free list: O(1) per page, no data moves.
+    """
+
+    def __init__(self, model: Model, n_streams: int, n_pages: int, max_pages_per_stream: int):
+        self.m = model
+        self.K = np.zeros((model.L, n_pages, PAGE_TOKENS, model.Hkv, model.hd), F64)
+        self.V = np.zeros((model.L, n_pages, PAGE_TOKENS, model.Hkv, model.hd), F64)
+        self.free = list(range(n_pages - 1, -1, -1))          # stack: pop() takes page 0 first
+        self.table = [[] for _ in range(n_streams)]
+        self.max_pages = max_pages_per_stream
+        self.length = [0] * n_streams
+        self.pending = [-1] * n_streams
+
+    def ensure(self, b: int, n_tokens: int) -> None:
+        """Make sure stream b owns pages for its first n_tokens slots."""
+        need = -(-n_tokens // PAGE_TOKENS)
+        assert need <= self.max_pages, "stream exceeds its block table"
+        while len(self.table[b]) < need:
+            assert self.free, "out of pages"
+            self.table[b].append(self.free.pop())
+
+    def release(self, b: int) -> None:
+        """Return the pages wholly beyond the committed length of stream b."""
+        keep = -(-self.length[b] // PAGE_TOKENS)
+        while len(self.table[b]) > keep:
+            self.free.append(self.table[b].pop())
+
+
+def forward_paged(model: Model, cache: PagedCache, b: int, ids: np.ndarray) -> np.ndarray:
+    """`forward` for stream b of a paged cache: gather its pages into a contiguous view, run the
+    same forward, scatter the appended rows back into the pages."""
+    ids = np.asarray(ids, dtype=np.int64)
+    n0, R = cache.length[b], len(ids)
+    cache.ensure(b, n0 + R)
+    view = Stream(model, len(cache.table[b]) * PAGE_TOKENS)
+    for l in range(model.L):
+        for i, pg in enumerate(cache.table[b]):
+            view.K[l][i * PAGE_TOKENS:(i + 1) * PAGE_TOKENS] = cache.K[l, pg]
+            view.V[l][i * PAGE_TOKENS:(i + 1) * PAGE_TOKENS] = cache.V[l, pg]
+    view.length, view.pending = n0, cache.pending[b]
+    logits = forward(model, view, ids)
+    for l in range(model.L):
+        for t in range(n0, n0 + R):
+            pg, slot = cache.table[b][t // PAGE_TOKENS], t % PAGE_TOKENS
+            cache.K[l, pg, slot] = view.K[l][t]
+            cache.V[l, pg, slot] = view.V[l][t]
+    return logits
+
+
+def commit_paged(cache: PagedCache, b: int, k: int, y: int) -> None:
+    cache.length[b] += 1 + int(k)
+    cache.pending[b] = int(y)
+    cache.release(b)
+
+
+def truncate_paged(cache: PagedCache, b: int, new_length: int, pending: int) -> None:
+    assert 0 <= new_length <= cache.length[b]
+    cache.length[b], cache.pending[b] = int(new_length), int(pending)
+    cache.release(b)

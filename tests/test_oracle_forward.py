@@ -209,3 +209,84 @@ def test_truncate_makes_verify_idempotent():
     orc.truncate(st, length, pending)
     b = orc.forward(m, st, ids)
     assert np.array_equal(a, b)
+
+
+def test_paged_cache_equals_contiguous_cache_under_churn():
+    """Three streams share a small page pool: prefill, verify-style forwards with commits and
+    rollbacks, one stream leaves and another prefix joins in its place.  Every forward must give
+    bit-identical logits to the same history on a private contiguous cache; pages are conserved,
+    never owned twice, and a rollback returns exactly the pages beyond the committed length."""
+    shape = small_shape()
+    w = synth.make_weights(shape, 21)
+    m = oracle_model(shape, w)
+    P = orc.PAGE_TOKENS
+    n_pages = 9
+    cache = orc.PagedCache(m, 3, n_pages, 4)
+    rng = np.random.default_rng(4)
+
+    def check_pages():
+        owned = [pg for t in cache.table for pg in t]
+        assert len(owned) == len(set(owned))
+        assert sorted(owned + cache.free) == list(range(n_pages))
+        for b in range(3):
+            assert len(cache.table[b]) == -(-cache.length[b] // P)
+
+    plain = [orc.Stream(m, 4 * P) for _ in range(3)]
+    lens = [70, 5, 130]
+    for b, n in enumerate(lens):
+        ids = rng.integers(0, shape.vocab_out, size=n)
+        for s0 in range(0, n - 1, 50):                     # chunked prefill on both
+            part = ids[s0:min(s0 + 50, n - 1)]
+            a = orc.forward_paged(m, cache, b, part)
+            cache.length[b] += len(part)
+            r = orc.forward(m, plain[b], part)
+            plain[b].length += len(part)
+            assert np.array_equal(a, r)
+        cache.pending[b] = plain[b].pending = int(ids[-1])
+    check_pages()
+    for step in range(6):
+        for b in range(3):
+            draft = rng.integers(0, shape.vocab_out, size=4)
+            ids = np.concatenate([[plain[b].pending], draft])
+            a = orc.forward_paged(m, cache, b, ids)
+            r = orc.forward(m, plain[b], ids)
+            assert np.array_equal(a, r)
+            k = int(rng.integers(0, 5))
+            y = int(rng.integers(0, shape.vocab_out))
+            orc.commit_paged(cache, b, k, y)               # releases the provisional pages
+            orc.commit(plain[b], k, y)
+        check_pages()
+    # rollback across a page boundary frees that page at once
+    before = len(cache.free)
+    b = 2
+    assert cache.length[b] > 2 * P
+    held = len(cache.table[b])
+    orc.truncate_paged(cache, b, P - 3, 7)
+    orc.truncate(plain[b], P - 3, 7)
+    assert len(cache.table[b]) == 1 and len(cache.free) == before + held - 1
+    check_pages()
+    ids = np.array([7, 1, 2])
+    assert np.array_equal(orc.forward_paged(m, cache, b, ids), orc.forward(m, plain[b], ids))
+    cache.release(b)
+    # stream 0 leaves; a new, longer prefix joins in its place and reuses the freed pages
+    orc.truncate_paged(cache, 0, 0, -1)
+    assert cache.table[0] == []
+    plain[0] = orc.Stream(m, 4 * P)
+    ids = rng.integers(0, shape.vocab_out, size=150)
+    a = orc.forward_paged(m, cache, 0, ids[:-1])
+    cache.length[0] += 149
+    r = orc.forward(m, plain[0], ids[:-1])
+    plain[0].length += 149
+    assert np.array_equal(a, r)
+    check_pages()
+    # the other streams' data survived the churn
+    for b in (1, 2):
+        ids = np.array([plain[b].pending, 3, 4])
+        assert np.array_equal(orc.forward_paged(m, cache, b, ids), orc.forward(m, plain[b], ids))
+        cache.release(b)
+    check_pages()
+    # the pool is finite: asking for more than it holds fails loudly
+    with pytest.raises(AssertionError):
+        cache.ensure(1, 4 * P)
+        cache.ensure(2, 4 * P)
+        cache.ensure(0, 4 * P)
