@@ -121,6 +121,31 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
                        size_t ws_bytes, ssd_streams** out);
 void ssd_streams_destroy(ssd_streams* s);
 
+/* Paged form of the cache (bf16 models): instead of one slice of `capacity` slots per stream, all
+ * streams draw 64-token pages from one pool, so that short and long utterances share memory and a
+ * stream that ends hands its pages to the next one.  Pool layout (caller-owned, ssd_paged_kv_bytes):
+ *     kv[layer][page][2 (0 = K, 1 = V)][kv_head][64][head_dim]
+ * Token t of stream b lives in page table[b][t / 64], slot t % 64; the tables and the free-page
+ * stack are device arrays inside the workspace, maintained by the library's kernels: a forward
+ * first takes pages for the rows it appends, and every call that can lower a length (ssd_kv_commit,
+ * ssd_kv_truncate, ssd_kv_restore) returns the pages that lie wholly beyond the new length - the
+ * O(1) rollback of rejected positions, without moving data.  A stream leaves by being truncated to
+ * length 0 and joins by a prefill (ssd_prefill accepts streams with no ids: they keep their state).
+ * A stream may hold at most max_pages_per_stream pages (its capacity is 64 times that); if the pool
+ * or a table is exhausted the rows that found no page are dropped and SSD_STATUS_KV_OVERFLOW is set.
+ * All forwards of paged streams run on the batched tensor-core path; batch * (max_gamma + 1) must
+ * not exceed 512 rows.  Everything else (verify, draft step, commit, the loop) is called as usual. */
+size_t ssd_paged_kv_bytes(const ssd_model_config* cfg, int32_t n_pages);
+size_t ssd_paged_workspace_bytes(const ssd_model_config* cfg, int32_t batch, int32_t max_gamma,
+                                 int32_t n_pages, int32_t max_pages_per_stream);
+int ssd_streams_create_paged(const ssd_model* m, int32_t batch, int32_t n_pages,
+                             int32_t max_pages_per_stream, int32_t max_gamma, void* dev_kv,
+                             size_t kv_bytes, void* dev_workspace, size_t ws_bytes, ssd_streams** out);
+/* Pages each stream holds (int32 [B]), pages on the free stack, and the block tables
+ * (int32 [B, max_pages_per_stream], -1 = none); any output may be NULL.  Synchronises `stream`. */
+int ssd_paged_state(ssd_streams* s, int32_t* host_pages_used, int32_t* host_free_pages,
+                    int32_t* host_page_table, void* stream);
+
 /* Which kernels run the decoder forward (Eq. 4) for these streams.  path 0 (default): forwards of
  * at most 16 rows over a bf16 model run in one persistent kernel (one CTA per SM, weights streamed
  * through shared-memory rings), larger ones in the generic per-operation kernels; path 1: generic
@@ -155,8 +180,8 @@ int ssd_kv_restore(ssd_streams* s, const int32_t* dev_len, const int32_t* dev_pe
 int ssd_streams_get_state(ssd_streams* s, int32_t* host_len, int32_t* host_pending, void* stream);
 
 /* Loads prefixes T_in through the model: stream b receives ids dev_ids[host_offsets[b] ..
- * host_offsets[b+1]) (>= 1 id each), appended after its current len.  K/V are written for all
- * but the last id, which becomes `pending`.  Enqueues work only. */
+ * host_offsets[b+1]), appended after its current len.  K/V are written for all but the last id,
+ * which becomes `pending`; a stream with no ids is left as it is.  Enqueues work only. */
 int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int32_t* host_offsets,
                 void* stream);
 

@@ -25,7 +25,8 @@ EXPORTS = [
     "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_streams_inject_failure",
-    "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check", "ssd_iteration",
+    "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check", "ssd_iteration", "ssd_paged_kv_bytes",
+    "ssd_paged_workspace_bytes", "ssd_streams_create_paged", "ssd_paged_state",
     "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
@@ -97,6 +98,12 @@ def lib() -> ctypes.CDLL:
     L.ssd_accept_noalloc.argtypes = [vp, vp, vp, vp, parp, i32, i32, vp, vp, vp]
     L.ssd_streams_inject_failure.argtypes = [vp, vp]
     L.ssd_iteration.argtypes = [vp, vp, vp, vp, parp, ctypes.POINTER(LoopIo), vp]
+    L.ssd_paged_kv_bytes.restype = sz
+    L.ssd_paged_kv_bytes.argtypes = [cfgp, i32]
+    L.ssd_paged_workspace_bytes.restype = sz
+    L.ssd_paged_workspace_bytes.argtypes = [cfgp, i32, i32, i32, i32]
+    L.ssd_streams_create_paged.argtypes = [vp, i32, i32, i32, i32, vp, sz, vp, sz, ctypes.POINTER(vp)]
+    L.ssd_paged_state.argtypes = [vp, vp, vp, vp, vp]
     L.ssd_tc_gemm_scratch_bytes.restype = sz
     L.ssd_tc_gemm_scratch_bytes.argtypes = [i32, i32, i32]
     L.ssd_tc_gemm_check.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, sz, vp, vp, vp]
@@ -310,6 +317,47 @@ class Streams:
         check(lib().ssd_draft_step(self.model.handle, self.handle, in_ids.data_ptr(), n_in,
                                    uniform.data_ptr(), ctypes.byref(params), out_token.data_ptr(),
                                    out_prob_row.data_ptr(), _stream_ptr(stream)))
+
+
+class PagedStreams(Streams):
+    """Streams whose K/V live in 64-token pages drawn from one pool (ssd_streams_create_paged)."""
+
+    PAGE_TOKENS = 64
+
+    def __init__(self, model: Model, batch: int, n_pages: int, max_pages_per_stream: int, max_gamma: int):
+        L = lib()
+        self.model, self.B, self.max_gamma = model, batch, max_gamma
+        self.n_pages, self.max_pages = n_pages, max_pages_per_stream
+        self.capacity = max_pages_per_stream * self.PAGE_TOKENS
+        cfg, dev = model.cfg, model.device
+        kvb = L.ssd_paged_kv_bytes(ctypes.byref(cfg), n_pages)
+        wsb = L.ssd_paged_workspace_bytes(ctypes.byref(cfg), batch, max_gamma, n_pages, max_pages_per_stream)
+        if kvb == 0 or wsb == 0:
+            raise SsdError("unsupported paged stream configuration")
+        with torch.cuda.device(dev):
+            self.kv_raw = _alloc(kvb, dev)
+            self.ws = _alloc(wsb, dev)
+            h = ctypes.c_void_p()
+            check(L.ssd_streams_create_paged(model.handle, batch, n_pages, max_pages_per_stream, max_gamma,
+                                             self.kv_raw.data_ptr(), kvb, self.ws.data_ptr(), wsb,
+                                             ctypes.byref(h)))
+        self.handle = h
+        s = model.shape
+        self.kv = self.kv_raw[:kvb].view(torch.bfloat16).view(s.n_layers, n_pages, 2, s.n_kv_heads,
+                                                              self.PAGE_TOKENS, s.head_dim)
+
+    def paged_state(self, stream=None):
+        """(pages held by each stream, free pages, block tables [B, max_pages] with -1 = none)."""
+        used = np.zeros(self.B, np.int32)
+        free = np.zeros(1, np.int32)
+        table = np.zeros((self.B, self.max_pages), np.int32)
+        check(lib().ssd_paged_state(self.handle, used.ctypes.data, free.ctypes.data, table.ctypes.data,
+                                    _stream_ptr(stream)))
+        return used, int(free[0]), table
+
+    def prefill_some(self, prefixes: Sequence[Optional[np.ndarray]], stream=None) -> None:
+        """Prefill only the streams whose entry is not None (the others keep their state)."""
+        self.prefill([p if p is not None else np.zeros(0, np.int32) for p in prefixes], stream)
 
 
 def accept_noalloc(logits: torch.Tensor, draft_tokens: torch.Tensor, draft_probs: torch.Tensor,

@@ -145,11 +145,12 @@ struct WsPlan {
   size_t hfix, flags, epoch_base, xa, xb, xd, xq, ssq_a, ssq_b;
   size_t tc_xa, tc_xattn, tc_xact, tc_part;
   size_t attn_part, attn_cnt;
+  size_t page_table, pages_used, free_stack, free_top;
   size_t total;
   int max_rows, nsplit_max;
 };
 
-WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
+WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap, int n_pages = 0, int max_pages = 0) {
   WsPlan p;
   size_t off = 0;
   size_t d = c.d_model, qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
@@ -197,6 +198,13 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap) {
     p.attn_part = take((size_t)FAST_MAX_CTAS * hps * FAST_MAX_T * (c.head_dim + 2) * 4);
     p.attn_cnt = take((size_t)FAST_MAX_CTAS * 4);
   }
+  p.page_table = p.pages_used = p.free_stack = p.free_top = 0;
+  if (n_pages > 0) {
+    p.page_table = take((size_t)B * max_pages * 4);
+    p.pages_used = take((size_t)B * 4);
+    p.free_stack = take((size_t)n_pages * 4);
+    p.free_top = take(4);
+  }
   p.tc_xa = p.tc_xattn = p.tc_xact = p.tc_part = 0;
   if (c.weight_dtype == 1 && M > FAST_MAX_T && M <= TC_MAX_ROWS) {
     const int Mpad = tc_round16((int)M), n_sm = fast_cta_count();
@@ -232,7 +240,7 @@ bool same_shape(const ssd_model_config& a, const ssd_model_config& b) {
 // rows' K/V at len + r; when logits_out is non-null also runs the final norm and the LM head.
 // The persistent kernel covers forwards of at most FAST_MAX_T rows over a bf16 model.
 bool use_fast(const ssd_model* m, const ssd_streams* s, RowMap rm) {
-  return m->fast.enabled && s->path == 0 && rm.nb * rm.R <= FAST_MAX_T;
+  return m->fast.enabled && s->path == 0 && !s->paged && rm.nb * rm.R <= FAST_MAX_T;
 }
 
 int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* row_ids,
@@ -303,6 +311,7 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
 // (each weight byte read once), attention on the warp-level tensor-core instruction.
 bool use_tc(const ssd_model* m, const ssd_streams* s, RowMap rm) {
   const int M = rm.nb * rm.R;
+  if (s->paged) return true;  // the paged cache exists on this path only (sizes checked at creation)
   return m->tc.enabled && s->path == 0 && s->tc_part && M > FAST_MAX_T && M <= TC_MAX_ROWS && M <= s->max_rows;
 }
 
@@ -321,6 +330,10 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
   if (kps < 64) kps = 64;
   while ((s->cap + kps - 1) / kps > 128) kps += 64;  // the merge kernel's table of splits
   const int nsplit = (int)((s->cap + kps - 1) / kps);
+  if (M > s->max_rows || M > TC_MAX_ROWS) return SSD_ERR_BAD_PARAM;
+  if (s->paged)  // every stream of this forward owns pages for the rows it is about to append
+    launch_page_ensure(s->len, rm, s->page_table, s->pages_used, s->free_stack, s->free_top, s->max_pages,
+                       s->status, st);
   launch_embed(1, m->embed, c.vocab_out + c.vocab_text, d, s->row_ids, M, s->h, s->status, st);
   launch_rope_table(s->len, rm, m->inv_freq, c.head_dim / 2, s->rope_cs, st);
   const float* part = nullptr;
@@ -336,9 +349,10 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
     g.w = t.w_qkv; g.a = s->tc_xa; g.n_rows = nq; g.K = d; g.ksplit = ks_qkv; g.epi = TC_EPI_PARTIAL; g.part = s->tc_part;
     SSD_CUDA(launch_tc_gemm(g, st));
     launch_tc_qkv_post(s->tc_part, ks_qkv, ld_of(nq), Mpad, (const bf16*)w.b_qkv, s->rope_cs, s->qrot, kv_layer,
-                       s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim, s->status, st);
+                       s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim, s->page_table, s->max_pages,
+                       s->status, st);
     SSD_CUDA(launch_tc_attention(s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim,
-                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, st));
+                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, s->page_table, s->max_pages, st));
     g.w = t.w_o; g.a = s->tc_xattn; g.n_rows = d; g.K = qd; g.ksplit = ks_o;
     SSD_CUDA(launch_tc_gemm(g, st));
     launch_tc_norm_pack(s->h, s->tc_part, ks_o, ld_of(d), M, d, (const bf16*)w.norm2, c.rms_eps, s->tc_xa, st);
@@ -361,6 +375,7 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
 }
 
 int forward(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out, cudaStream_t st) {
+  if (s->paged) return forward_tc(m, s, rm, logits_out, st);
   if (use_fast(m, s, rm)) return forward_fast(m, s, rm, s->row_ids, nullptr, logits_out, st);
   if (use_tc(m, s, rm)) return forward_tc(m, s, rm, logits_out, st);
   const ssd_model_config& c = m->cfg;
@@ -591,17 +606,93 @@ size_t ssd_workspace_bytes(const ssd_model_config* cfg, int32_t batch, int32_t m
   return plan_ws(*cfg, batch, max_gamma, capacity_tokens).total;
 }
 
+}  // extern "C"
+
+namespace {
+
+// Shared by the contiguous (n_pages = 0) and the paged form.
+int streams_create_impl(const ssd_model* m, int32_t batch, int32_t capacity_tokens, int32_t max_gamma,
+                        int32_t n_pages, int32_t max_pages, void* dev_kv, size_t kv_bytes,
+                        void* dev_workspace, size_t ws_bytes, ssd_streams** out);
+
+}  // namespace
+
+extern "C" {
+
 int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_tokens,
                        int32_t max_gamma, void* dev_kv, size_t kv_bytes, void* dev_workspace,
                        size_t ws_bytes, ssd_streams** out) {
+  return streams_create_impl(m, batch, capacity_tokens, max_gamma, 0, 0, dev_kv, kv_bytes, dev_workspace,
+                             ws_bytes, out);
+}
+
+size_t ssd_paged_kv_bytes(const ssd_model_config* cfg, int32_t n_pages) {
+  if (!cfg_ok(cfg) || cfg->weight_dtype != 1 || n_pages < 1) return 0;
+  return (size_t)cfg->n_layers * n_pages * 2 * cfg->n_kv_heads * TC_PAGE_TOKENS * cfg->head_dim * 2;
+}
+
+size_t ssd_paged_workspace_bytes(const ssd_model_config* cfg, int32_t batch, int32_t max_gamma,
+                                 int32_t n_pages, int32_t max_pages_per_stream) {
+  if (!cfg || cfg->weight_dtype != 1 || n_pages < 1 || max_pages_per_stream < 1 ||
+      max_pages_per_stream > (1 << 14) ||
+      !streams_args_ok(cfg, batch, max_gamma, max_pages_per_stream * TC_PAGE_TOKENS))
+    return 0;
+  const WsPlan p = plan_ws(*cfg, batch, max_gamma, max_pages_per_stream * TC_PAGE_TOKENS, n_pages,
+                           max_pages_per_stream);
+  return p.max_rows <= TC_MAX_ROWS ? p.total : 0;
+}
+
+int ssd_streams_create_paged(const ssd_model* m, int32_t batch, int32_t n_pages,
+                             int32_t max_pages_per_stream, int32_t max_gamma, void* dev_kv,
+                             size_t kv_bytes, void* dev_workspace, size_t ws_bytes, ssd_streams** out) {
+  if (!m) return SSD_ERR_NULL;
+  if (!m->tc.enabled || n_pages < 1 || max_pages_per_stream < 1 || max_pages_per_stream > (1 << 14))
+    return SSD_ERR_BAD_CONFIG;
+  return streams_create_impl(m, batch, max_pages_per_stream * TC_PAGE_TOKENS, max_gamma, n_pages,
+                             max_pages_per_stream, dev_kv, kv_bytes, dev_workspace, ws_bytes, out);
+}
+
+int ssd_paged_state(ssd_streams* s, int32_t* host_pages_used, int32_t* host_free_pages,
+                    int32_t* host_page_table, void* stream) {
+  if (!s) return SSD_ERR_NULL;
+  if (!s->paged) return SSD_ERR_BAD_CONFIG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (host_pages_used)
+    SSD_CUDA(cudaMemcpyAsync(host_pages_used, s->pages_used, (size_t)s->B * 4, cudaMemcpyDeviceToHost, st));
+  if (host_free_pages) SSD_CUDA(cudaMemcpyAsync(host_free_pages, s->free_top, 4, cudaMemcpyDeviceToHost, st));
+  if (host_page_table)
+    SSD_CUDA(cudaMemcpyAsync(host_page_table, s->page_table, (size_t)s->B * s->max_pages * 4,
+                             cudaMemcpyDeviceToHost, st));
+  SSD_CUDA(cudaStreamSynchronize(st));
+  return SSD_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int streams_create_impl(const ssd_model* m, int32_t batch, int32_t capacity_tokens, int32_t max_gamma,
+                        int32_t n_pages, int32_t max_pages, void* dev_kv, size_t kv_bytes,
+                        void* dev_workspace, size_t ws_bytes, ssd_streams** out) {
   if (!m || !dev_kv || !dev_workspace || !out) return SSD_ERR_NULL;
   if (!streams_args_ok(&m->cfg, batch, max_gamma, capacity_tokens)) return SSD_ERR_BAD_CONFIG;
   if (((uintptr_t)dev_kv & 255) || ((uintptr_t)dev_workspace & 255)) return SSD_ERR_MISALIGNED;
   const ssd_model_config& c = m->cfg;
-  if (kv_bytes < ssd_kv_bytes(&c, batch, capacity_tokens)) return SSD_ERR_TOO_SMALL;
-  WsPlan p = plan_ws(c, batch, max_gamma, capacity_tokens);
+  const bool paged = n_pages > 0;
+  if (kv_bytes < (paged ? ssd_paged_kv_bytes(&c, n_pages) : ssd_kv_bytes(&c, batch, capacity_tokens)))
+    return SSD_ERR_TOO_SMALL;
+  WsPlan p = plan_ws(c, batch, max_gamma, capacity_tokens, n_pages, max_pages);
+  if (paged && (p.max_rows > TC_MAX_ROWS || !p.tc_part)) return SSD_ERR_BAD_CONFIG;
   if (ws_bytes < p.total) return SSD_ERR_TOO_SMALL;
   SSD_CUDA(cudaMemset(dev_workspace, 0, p.total));
+  if (paged) {  // all pages free (page 0 on top of the stack), block tables empty (-1)
+    std::vector<int32_t> stack(n_pages);
+    for (int i = 0; i < n_pages; ++i) stack[i] = n_pages - 1 - i;
+    SSD_CUDA(cudaMemcpy((char*)dev_workspace + p.free_stack, stack.data(), (size_t)n_pages * 4,
+                        cudaMemcpyHostToDevice));
+    SSD_CUDA(cudaMemcpy((char*)dev_workspace + p.free_top, &n_pages, 4, cudaMemcpyHostToDevice));
+    SSD_CUDA(cudaMemset((char*)dev_workspace + p.page_table, 0xFF, (size_t)batch * max_pages * 4));
+  }
   SSD_CUDA(cudaDeviceSynchronize());
   ssd_streams* s = new (std::nothrow) ssd_streams();
   if (!s) return SSD_ERR_CUDA;
@@ -613,7 +704,11 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->max_rows = p.max_rows;
   s->nsplit_max = p.nsplit_max;
   s->kv = (char*)dev_kv;
-  s->kv_layer_elems = (size_t)batch * 2 * c.n_kv_heads * (size_t)capacity_tokens * c.head_dim;
+  s->kv_layer_elems = paged ? (size_t)n_pages * 2 * c.n_kv_heads * (size_t)TC_PAGE_TOKENS * c.head_dim
+                            : (size_t)batch * 2 * c.n_kv_heads * (size_t)capacity_tokens * c.head_dim;
+  s->paged = paged ? 1 : 0;
+  s->n_pages = n_pages;
+  s->max_pages = max_pages;
   char* W = (char*)dev_workspace;
   s->ws = W;
   s->ws_bytes = p.total;
@@ -654,6 +749,11 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   s->tc_xattn = p.tc_part ? (uint8_t*)(W + p.tc_xattn) : nullptr;
   s->tc_xact = p.tc_part ? (uint8_t*)(W + p.tc_xact) : nullptr;
   s->tc_part = p.tc_part ? (float*)(W + p.tc_part) : nullptr;
+  s->page_table = paged ? (int32_t*)(W + p.page_table) : nullptr;
+  s->pages_used = paged ? (int32_t*)(W + p.pages_used) : nullptr;
+  s->free_stack = paged ? (int32_t*)(W + p.free_stack) : nullptr;
+  s->free_top = paged ? (int32_t*)(W + p.free_top) : nullptr;
+  if (paged) s->key_split = 0;
   s->path = 0;
   s->split_act = 1;
   s->trace = nullptr;
@@ -661,6 +761,16 @@ int ssd_streams_create(const ssd_model* m, int32_t batch, int32_t capacity_token
   *out = s;
   return SSD_OK;
 }
+
+// Paged cache: after anything that may have lowered a length, the pages beyond it are returned.
+void release_pages(ssd_streams* s, cudaStream_t st) {
+  if (s->paged)
+    launch_page_release(s->len, s->B, s->page_table, s->pages_used, s->free_stack, s->free_top, s->max_pages, st);
+}
+
+}  // namespace
+
+extern "C" {
 
 void ssd_streams_destroy(ssd_streams* s) { delete s; }
 
@@ -742,6 +852,7 @@ int ssd_kv_truncate(ssd_streams* s, const int32_t* host_len, const int32_t* host
   cudaStream_t st = (cudaStream_t)stream;
   SSD_CUDA(cudaMemcpyAsync(s->len, host_len, s->B * 4, cudaMemcpyHostToDevice, st));
   SSD_CUDA(cudaMemcpyAsync(s->pending, host_pending, s->B * 4, cudaMemcpyHostToDevice, st));
+  release_pages(s, st);
   SSD_CUDA(cudaStreamSynchronize(st));
   return SSD_OK;
 }
@@ -749,6 +860,7 @@ int ssd_kv_truncate(ssd_streams* s, const int32_t* host_len, const int32_t* host
 int ssd_kv_restore(ssd_streams* s, const int32_t* dev_len, const int32_t* dev_pending, void* stream) {
   if (!s || !dev_len || !dev_pending) return SSD_ERR_NULL;
   launch_kv_restore(s->len, s->pending, dev_len, dev_pending, s->B, s->cap, (cudaStream_t)stream);
+  release_pages(s, (cudaStream_t)stream);
   SSD_CUDA(cudaGetLastError());
   return SSD_OK;
 }
@@ -769,7 +881,7 @@ int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int3
   if (!same_shape(m->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
   for (int b = 0; b < s->B; ++b) {
     int n = host_offsets[b + 1] - host_offsets[b];
-    if (n < 1) return SSD_ERR_BAD_PARAM;
+    if (n < 0) return SSD_ERR_BAD_PARAM;  // 0: this stream takes no part (it keeps its state)
     if (n - 1 > s->cap) return SSD_ERR_KV_OVERFLOW;
   }
   cudaStream_t st = (cudaStream_t)stream;
@@ -781,6 +893,7 @@ int ssd_prefill(ssd_model* m, ssd_streams* s, const int32_t* dev_ids, const int3
   for (int b = 0; b < s->B; ++b) {
     const int32_t* ids = dev_ids + host_offsets[b];
     int n = host_offsets[b + 1] - host_offsets[b];
+    if (n == 0) continue;
     for (int done = 0; done < n - 1; done += chunk) {
       int rows = n - 1 - done < chunk ? n - 1 - done : chunk;
       SSD_CUDA(cudaMemcpyAsync(s->row_ids, ids + done, rows * 4, cudaMemcpyDeviceToDevice, st));
@@ -838,6 +951,7 @@ int ssd_iteration(ssd_model* target, ssd_streams* ts, ssd_model* draft, ssd_stre
   launch_loop_finish(ds->len, ds->pending, ds->cap, io->dev_in_ids, io->dev_draft_tokens, gamma,
                      io->dev_accepted_len, io->dev_next_token, B, io->dev_out_tokens, io->out_capacity,
                      io->dev_out_count, io->dev_accept_log, io->n_iterations, io->dev_iteration, ts->status, st);
+  release_pages(ds, st);
   SSD_CUDA(cudaGetLastError());
   return SSD_OK;
 }
@@ -875,6 +989,7 @@ int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t
   if (!s || !dev_accepted_len || !dev_next_token) return SSD_ERR_NULL;
   launch_kv_commit(s->len, s->pending, dev_accepted_len, dev_next_token, s->B, s->cap, s->max_gamma, s->status,
                    (cudaStream_t)stream);
+  release_pages(s, (cudaStream_t)stream);  // the rejected positions' pages, if they filled any
   SSD_CUDA(cudaGetLastError());
   return SSD_OK;
 }

@@ -131,6 +131,10 @@ struct ssd_streams {
   float* attn_part;    // persistent kernel, key-split attention: per-CTA partials
   uint32_t* attn_cnt;  // and the per-slice arrival counters
   int key_split;       // 1: forwards on these streams use the key-split variant
+  // paged cache (ssd_streams_create_paged): pool kv[layer][page][2][Hkv][64][hd], block tables and
+  // the free stack in the workspace; cap = max_pages * 64
+  int paged, n_pages, max_pages;
+  int32_t *page_table, *pages_used, *free_stack, *free_top;
   // batched tensor-core forward: packed operands (inputs of QKV / gate-up / head, of O, of down)
   // and the partial sums of the K-split projections
   uint8_t *tc_xa, *tc_xattn, *tc_xact;

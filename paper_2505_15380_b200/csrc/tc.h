@@ -93,14 +93,27 @@ void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, i
 void launch_tc_pack_rows(const float* x, int M, int K, uint8_t* apack, cudaStream_t st);
 // q/k/v = sum of partials + bias; rotary embedding; q (scaled) to qrot [M, Hq * hd] fp32, K and V
 // appended to the cache at len + r.
+// Paged cache (page_table non-null): kv_layer is the layer's page pool [page][2][Hkv][64][hd] and
+// token t of stream b lives in page page_table[b * max_pages + t / 64], slot t % 64.
+constexpr int TC_PAGE_TOKENS = 64;
 void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, const bf16* bias,
                         const float* cs, float* qrot, bf16* kv_layer, const int32_t* len, RowMap rm,
-                        int cap, int Hq, int Hkv, int hd, int32_t* status, cudaStream_t st);
+                        int cap, int Hq, int Hkv, int hd, const int32_t* page_table, int max_pages,
+                        int32_t* status, cudaStream_t st);
+// Page bookkeeping of a paged cache.  ensure: every stream of the forward owns pages for its
+// first len + R slots (taken from the free stack).  release: pages wholly beyond a stream's
+// committed length go back to the free stack - the O(1) rollback of a paged cache.
+void launch_page_ensure(const int32_t* len, RowMap rm, int32_t* page_table, int32_t* pages_used,
+                        int32_t* free_stack, int32_t* free_top, int max_pages, int32_t* status,
+                        cudaStream_t st);
+void launch_page_release(const int32_t* len, int B, int32_t* page_table, int32_t* pages_used,
+                         int32_t* free_stack, int32_t* free_top, int max_pages, cudaStream_t st);
 
 // tc_attention.cu: verify attention for all streams of the forward (causal inside the block, GQA),
 // split over the keys; the merged result is written as the packed operand of the O projection.
 cudaError_t launch_tc_attention(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm,
                                 int cap, int Hq, int Hkv, int hd, float* part, int nsplit,
-                                int keys_per_split, uint8_t* apack_out, int Mpad, cudaStream_t st);
+                                int keys_per_split, uint8_t* apack_out, int Mpad,
+                                const int32_t* page_table, int max_pages, cudaStream_t st);
 
 }  // namespace ssd

@@ -25,6 +25,7 @@ namespace {
 
 constexpr int TA_WARPS = 4;
 constexpr int TA_TILE = 64;  // keys per tile
+static_assert(TA_TILE == TC_PAGE_TOKENS, "a key tile of the batched attention is one page of a paged cache");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -57,7 +58,7 @@ template <int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32)
 tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer, const int32_t* __restrict__ len,
                RowMap rm, int cap, int Hq, int Hkv, int n_rowgroups, float* __restrict__ part, int nsplit,
-               int keys_per_split) {
+               int keys_per_split, const int32_t* __restrict__ page_table, int max_pages) {
   constexpr int ROWB = HD * 2 + 16;   // padded K / V row: conflict-free matrix loads
   constexpr int KSTEPS = HD / 16;
   constexpr int DT = HD / 8;
@@ -79,12 +80,21 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
 
   auto stage_tile = [&](int stage, int key0) {
     uint8_t* ks = kv_s + (size_t)stage * 2 * TILE_BYTES;
+    const bf16 *kt = kbase, *vt = vbase;
+    int first = 0;  // key index of the tile's base pointers
+    if (page_table) {
+      // a tile is one page: key splits start at multiples of the page size, which is the tile size
+      const int pg = max(page_table[(size_t)b * max_pages + key0 / TC_PAGE_TOKENS], 0);
+      kt = kv_layer + (((size_t)pg * 2 + 0) * Hkv + gk) * (size_t)TC_PAGE_TOKENS * HD;
+      vt = kv_layer + (((size_t)pg * 2 + 1) * Hkv + gk) * (size_t)TC_PAGE_TOKENS * HD;
+      first = key0;
+    }
     for (int i = tid; i < TA_TILE * CH; i += TA_WARPS * 32) {
       const int key = i / CH, c = i % CH;
       // keys past the range repeat the last valid one: finite data, masked out below
-      const size_t src = (size_t)min(key0 + key, k_end - 1) * HD + c * 8;
-      cp_async16(smem_u32(ks + key * ROWB + c * 16), kbase + src);
-      cp_async16(smem_u32(ks + TILE_BYTES + key * ROWB + c * 16), vbase + src);
+      const size_t src = (size_t)(min(key0 + key, k_end - 1) - first) * HD + c * 8;
+      cp_async16(smem_u32(ks + key * ROWB + c * 16), kt + src);
+      cp_async16(smem_u32(ks + TILE_BYTES + key * ROWB + c * 16), vt + src);
     }
     cp_async_commit();
   };
@@ -298,14 +308,15 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
 template <int HD>
 cudaError_t launch_t(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm, int cap, int Hq,
                      int Hkv, float* part, int nsplit, int keys_per_split, uint8_t* apack_out, int Mpad,
-                     cudaStream_t st) {
+                     const int32_t* page_table, int max_pages, cudaStream_t st) {
   const int NQ = (Hq / Hkv) * rm.R, n_rowgroups = (NQ + TA_WARPS * 16 - 1) / (TA_WARPS * 16);
   const size_t smem = (size_t)4 * TA_TILE * (HD * 2 + 16) + (size_t)TA_WARPS * (HD / 16) * 32 * 32;
   auto kern = tc_attn_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<dim3(nsplit, Hkv * n_rowgroups, rm.nb), TA_WARPS * 32, smem, st>>>(qrot, kv_layer, len, rm, cap, Hq, Hkv,
-                                                                             n_rowgroups, part, nsplit, keys_per_split);
+                                                                             n_rowgroups, part, nsplit, keys_per_split,
+                                                                             page_table, max_pages);
   count_launch();
   tc_attn_merge_kernel<HD><<<dim3(Hq, rm.nb * rm.R), HD / 2 < 32 ? 32 : HD / 2, 0, st>>>(
       part, len, rm, cap, Hq, nsplit, keys_per_split, apack_out, Mpad);
@@ -317,11 +328,13 @@ cudaError_t launch_t(const float* qrot, const bf16* kv_layer, const int32_t* len
 
 cudaError_t launch_tc_attention(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm,
                                 int cap, int Hq, int Hkv, int hd, float* part, int nsplit,
-                                int keys_per_split, uint8_t* apack_out, int Mpad, cudaStream_t st) {
+                                int keys_per_split, uint8_t* apack_out, int Mpad,
+                                const int32_t* page_table, int max_pages, cudaStream_t st) {
+  if (page_table && keys_per_split % TC_PAGE_TOKENS) return cudaErrorInvalidValue;
   switch (hd) {
-    case 32: return launch_t<32>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, st);
-    case 64: return launch_t<64>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, st);
-    case 128: return launch_t<128>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, st);
+    case 32: return launch_t<32>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, st);
+    case 64: return launch_t<64>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, st);
+    case 128: return launch_t<128>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, st);
   }
   return cudaErrorInvalidValue;
 }

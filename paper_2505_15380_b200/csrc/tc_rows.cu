@@ -88,7 +88,8 @@ __global__ void __launch_bounds__(256)
 tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
                    const bf16* __restrict__ bias, const float* __restrict__ cs, float* __restrict__ qrot,
                    bf16* __restrict__ kv_layer, const int32_t* __restrict__ len, RowMap rm, int cap, int Hq,
-                   int Hkv, int hd, float scale, int32_t* status) {
+                   int Hkv, int hd, float scale, const int32_t* __restrict__ page_table, int max_pages,
+                   int32_t* status) {
   extern __shared__ float row[];  // [(Hq + 2 Hkv) * hd]
   const int m = blockIdx.x, tid = threadIdx.x;
   const int bi = m / rm.R, r = m % rm.R, b = rm.b0 + bi;
@@ -113,16 +114,27 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
   }
   const float* krow = row + Hq * hd;
   const float* vrow = krow + Hkv * hd;
+  // where this row's K and V live: the stream's slice of a contiguous cache, or its page
+  size_t owner = (size_t)b, rows_per = (size_t)cap, slot = (size_t)pos;
+  if (page_table) {
+    const int pg = page_table[(size_t)b * max_pages + pos / TC_PAGE_TOKENS];
+    if (pg < 0) {  // no page was granted (pool exhausted): flagged by the page kernel
+      return;
+    }
+    owner = (size_t)pg;
+    rows_per = TC_PAGE_TOKENS;
+    slot = (size_t)(pos % TC_PAGE_TOKENS);
+  }
   for (int i = tid; i < Hkv * half; i += 256) {
     const int g = i / half, j = i % half;
     const float x1 = krow[g * hd + j], x2 = krow[g * hd + j + half], co = c[2 * j], si = c[2 * j + 1];
-    bf16* kdst = kv_layer + (((size_t)b * 2 + 0) * Hkv + g) * (size_t)cap * hd + (size_t)pos * hd;
+    bf16* kdst = kv_layer + ((owner * 2 + 0) * Hkv + g) * rows_per * hd + slot * hd;
     kdst[j] = __float2bfloat16_rn(x1 * co - x2 * si);
     kdst[j + half] = __float2bfloat16_rn(x2 * co + x1 * si);
   }
   for (int i = tid; i < Hkv * hd; i += 256) {
     const int g = i / hd, j = i % hd;
-    bf16* vdst = kv_layer + (((size_t)b * 2 + 1) * Hkv + g) * (size_t)cap * hd + (size_t)pos * hd;
+    bf16* vdst = kv_layer + ((owner * 2 + 1) * Hkv + g) * rows_per * hd + slot * hd;
     vdst[j] = __float2bfloat16_rn(vrow[g * hd + j]);
   }
 }
@@ -143,11 +155,71 @@ void launch_tc_pack_rows(const float* x, int M, int K, uint8_t* apack, cudaStrea
 
 void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, const bf16* bias,
                         const float* cs, float* qrot, bf16* kv_layer, const int32_t* len, RowMap rm,
-                        int cap, int Hq, int Hkv, int hd, int32_t* status, cudaStream_t st) {
+                        int cap, int Hq, int Hkv, int hd, const int32_t* page_table, int max_pages,
+                        int32_t* status, cudaStream_t st) {
   const int M = rm.nb * rm.R;
   const size_t smem = (size_t)(Hq + 2 * Hkv) * hd * 4;
   tc_qkv_post_kernel<<<M, 256, smem, st>>>(part, nsplit, ld_part, Mpad, bias, cs, qrot, kv_layer, len, rm, cap, Hq,
-                                           Hkv, hd, 1.0f / sqrtf((float)hd), status);
+                                           Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
+  count_launch();
+}
+
+namespace {
+
+__global__ void page_ensure_kernel(const int32_t* __restrict__ len, RowMap rm, int32_t* page_table,
+                                   int32_t* pages_used, const int32_t* __restrict__ free_stack, int32_t* free_top,
+                                   int max_pages, int32_t* status) {
+  const int bi = blockIdx.x * blockDim.x + threadIdx.x;
+  if (bi >= rm.nb) return;
+  const int b = rm.b0 + bi;
+  int need = (len[b] + rm.R + TC_PAGE_TOKENS - 1) / TC_PAGE_TOKENS;
+  if (need > max_pages) {  // rows beyond the block table are not written (flagged as an overflow)
+    atomicOr(status, SSD_STATUS_KV_OVERFLOW);
+    need = max_pages;
+  }
+  int used = pages_used[b];
+  while (used < need) {
+    const int idx = atomicSub(free_top, 1) - 1;  // pops from different streams race only on this counter
+    if (idx < 0) {
+      atomicAdd(free_top, 1);
+      atomicOr(status, SSD_STATUS_KV_OVERFLOW);  // the pool is exhausted: the rows of this page are dropped
+      break;
+    }
+    page_table[(size_t)b * max_pages + used] = free_stack[idx];
+    ++used;
+  }
+  pages_used[b] = used;
+}
+
+__global__ void page_release_kernel(const int32_t* __restrict__ len, int B, int32_t* page_table, int32_t* pages_used,
+                                    int32_t* free_stack, int32_t* free_top, int max_pages) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int keep = (max(len[b], 0) + TC_PAGE_TOKENS - 1) / TC_PAGE_TOKENS;
+  int used = pages_used[b];
+  while (used > keep) {
+    --used;
+    const int idx = atomicAdd(free_top, 1);
+    free_stack[idx] = page_table[(size_t)b * max_pages + used];
+    page_table[(size_t)b * max_pages + used] = -1;
+  }
+  pages_used[b] = used;
+}
+
+}  // namespace
+
+void launch_page_ensure(const int32_t* len, RowMap rm, int32_t* page_table, int32_t* pages_used,
+                        int32_t* free_stack, int32_t* free_top, int max_pages, int32_t* status,
+                        cudaStream_t st) {
+  page_ensure_kernel<<<(rm.nb + 127) / 128, 128, 0, st>>>(len, rm, page_table, pages_used, free_stack, free_top,
+                                                         max_pages, status);
+  count_launch();
+}
+
+void launch_page_release(const int32_t* len, int B, int32_t* page_table, int32_t* pages_used,
+                         int32_t* free_stack, int32_t* free_top, int max_pages, cudaStream_t st) {
+  page_release_kernel<<<(B + 127) / 128, 128, 0, st>>>(len, B, page_table, pages_used, free_stack, free_top,
+                                                      max_pages);
   count_launch();
 }
 

@@ -98,9 +98,9 @@ def check_exclusions(res: "CaseResult", max_strict_frac: float = 0.10,
     """A parity case must have compared something, and may skip only a small share."""
     n = res.n_streams
     assert n >= 1 and n - res.n_strict_excluded >= 1, "no decision was compared"
-    assert res.n_strict_excluded <= max(1, int(max_strict_frac * n)), \
+    assert res.n_strict_excluded <= max(1, int(np.ceil(max_strict_frac * n))), \
         f"{res.n_strict_excluded} of {n} stream-steps excluded from the strict comparison"
-    assert res.n_e2e_excluded <= max(1, int(max_e2e_frac * n)), \
+    assert res.n_e2e_excluded <= max(1, int(np.ceil(max_e2e_frac * n))), \
         f"{res.n_e2e_excluded} of {n} stream-steps excluded from the end-to-end comparison"
 
 
@@ -108,7 +108,8 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
              oracle_streams: Optional[List[int]] = None, logit_tol: Optional[float] = None,
              uniform_seed: int = 0, commit_and_repeat: bool = False,
              capacity: Optional[int] = None, path: int = 0, split: bool = True,
-             max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34, top_p: float = 0.0) -> CaseResult:
+             max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34, top_p: float = 0.0,
+             paged: Optional[tuple] = None) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -119,7 +120,11 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
     omodel = oracle_model(shape, w)
     gmodel = binding.Model(shape, synth.weights_blob(shape, w))
     cap = capacity or (max(wl.prefix_lens) + 2 * R + 8)
-    gs = binding.Streams(gmodel, B, cap, gamma)
+    if paged:          # (pages in the pool, pages per stream): K/V in 64-token pages
+        gs = binding.PagedStreams(gmodel, B, paged[0], paged[1], gamma)
+        cap = gs.capacity
+    else:
+        gs = binding.Streams(gmodel, B, cap, gamma)
     gs.set_path(path)          # 0: persistent kernel where the forward fits it, 1: generic kernels
     gs.set_activation_split(split)   # persistent kernel: bf16 activations, or bf16 hi + lo pairs
     which = list(range(B)) if oracle_streams is None else list(oracle_streams)
