@@ -107,6 +107,16 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
                      void* dev_arena, size_t arena_bytes, ssd_model** out);
 void ssd_model_destroy(ssd_model* m);
 
+/* A model made of layers of another one, WITHOUT copying them: layer i of the new model is layer
+ * host_layer_map[i] of `source`; embedding, final norm and LM head are the source's.  This is the
+ * shape of the paper's draft model (Sec. 2.3: a shallower copy of the target built from its own
+ * layers - in the experiments the target's lower two and upper six of 24 - before fine-tuning):
+ * the draft pass then re-reads weights the verify pass has just pulled through L2 and adds no
+ * weight memory.  dev_arena (256-byte aligned, at least 256 bytes per 64 layers) receives the map;
+ * `source` and its arena must outlive the new handle.  Streams for it are created as for any model. */
+int ssd_model_create_inherited(const ssd_model* source, const int32_t* host_layer_map, int32_t n_layers,
+                               void* dev_arena, size_t arena_bytes, ssd_model** out);
+
 /* ---- streams ----------------------------------------------------------------------------- */
 
 size_t ssd_kv_bytes(const ssd_model_config* cfg, int32_t batch, int32_t capacity_tokens);

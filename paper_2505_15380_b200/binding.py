@@ -27,6 +27,7 @@ EXPORTS = [
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_streams_inject_failure",
     "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check", "ssd_iteration", "ssd_paged_kv_bytes",
     "ssd_paged_workspace_bytes", "ssd_streams_create_paged", "ssd_paged_state",
+    "ssd_model_create_inherited",
     "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
@@ -72,6 +73,7 @@ def lib() -> ctypes.CDLL:
     L.ssd_model_arena_bytes.restype = sz
     L.ssd_model_arena_bytes.argtypes = [cfgp]
     L.ssd_model_create.argtypes = [cfgp, vp, sz, vp, sz, ctypes.POINTER(vp)]
+    L.ssd_model_create_inherited.argtypes = [vp, vp, i32, vp, sz, ctypes.POINTER(vp)]
     L.ssd_model_destroy.restype = None
     L.ssd_model_destroy.argtypes = [vp]
     L.ssd_kv_bytes.restype = sz
@@ -174,6 +176,27 @@ class Model:
         if getattr(self, "handle", None) is not None and _lib is not None:
             _lib.ssd_model_destroy(self.handle)
             self.handle = None
+
+
+class InheritedModel(Model):
+    """A model made of some of another model's layers (ssd_model_create_inherited): no weights are
+    copied.  `shape` is the source's shape with the new number of layers."""
+
+    def __init__(self, source: Model, layer_map: Sequence[int]):
+        import dataclasses
+        L = lib()
+        self.source = source                      # keeps the source's arena alive
+        self.layer_map = [int(x) for x in layer_map]
+        self.shape = dataclasses.replace(source.shape, n_layers=len(self.layer_map))
+        self.cfg = make_config(self.shape)
+        self.device = source.device
+        m = np.ascontiguousarray(self.layer_map, dtype=np.int32)
+        with torch.cuda.device(self.device):
+            self.arena = _alloc(max(256, 4 * len(m)), self.device)
+            h = ctypes.c_void_p()
+            check(L.ssd_model_create_inherited(source.handle, m.ctypes.data, len(m), self.arena.data_ptr(),
+                                               self.arena.numel(), ctypes.byref(h)))
+        self.handle = h
 
 
 class Streams:

@@ -262,6 +262,8 @@ int forward_fast(const ssd_model* m, ssd_streams* s, RowMap rm, const int32_t* r
   p.m.down_split = f.down_split;
   p.m.o_split = f.o_split;
   p.m.max_stage_k = f.max_stage_k;
+  p.layer_map = f.layer_map;
+  p.n_src_layers = f.n_src_layers;
   p.embed = (const bf16*)m->embed;
   p.inv_freq = m->inv_freq;
   p.L = c.n_layers;
@@ -548,6 +550,7 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
     f.bias_qkv = (const float*)(A + p.f_bias);
     f.gains = (const float*)(A + p.f_gains);
     f.n_cta = fplan.n_cta;
+    f.n_src_layers = c.n_layers;
     f.down_split = fplan.ops[FOP_DOWN].ksplit;
     f.o_split = fplan.ops[FOP_O].ksplit;
     f.max_units = 0;
@@ -588,6 +591,34 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
     delete m;
     return cuda_fail(e, "ssd_model_create copy");
   }
+  *out = m;
+  return SSD_OK;
+}
+
+int ssd_model_create_inherited(const ssd_model* source, const int32_t* host_layer_map, int32_t n_layers,
+                               void* dev_arena, size_t arena_bytes, ssd_model** out) {
+  if (!source || !host_layer_map || !dev_arena || !out) return SSD_ERR_NULL;
+  if (n_layers < 1 || n_layers > 4096) return SSD_ERR_BAD_CONFIG;
+  for (int i = 0; i < n_layers; ++i)
+    if (host_layer_map[i] < 0 || host_layer_map[i] >= source->cfg.n_layers) return SSD_ERR_BAD_CONFIG;
+  if ((uintptr_t)dev_arena & 255) return SSD_ERR_MISALIGNED;
+  if (arena_bytes < align_up((size_t)n_layers * 4)) return SSD_ERR_TOO_SMALL;
+  ssd_model* m = new (std::nothrow) ssd_model(*source);  // same pointers: nothing is copied
+  if (!m) return SSD_ERR_CUDA;
+  m->cfg.n_layers = n_layers;
+  m->arena = (char*)dev_arena;
+  m->layers.resize(n_layers);
+  if (source->tc.enabled) m->tc.layers.resize(n_layers);
+  for (int i = 0; i < n_layers; ++i) {
+    m->layers[i] = source->layers[host_layer_map[i]];
+    if (source->tc.enabled) m->tc.layers[i] = source->tc.layers[host_layer_map[i]];
+  }
+  cudaError_t e = cudaMemcpy(dev_arena, host_layer_map, (size_t)n_layers * 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    delete m;
+    return cuda_fail(e, "ssd_model_create_inherited copy");
+  }
+  m->fast.layer_map = (const int32_t*)dev_arena;  // n_src_layers stays the source's
   *out = m;
   return SSD_OK;
 }

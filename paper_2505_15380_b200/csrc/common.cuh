@@ -83,6 +83,8 @@ struct ssd_fast_model {
   const int32_t *chunk_cnt = nullptr, *unit_cnt = nullptr, *unit_off = nullptr, *unit_tile = nullptr;
   const float *bias_qkv = nullptr, *gains = nullptr;
   int n_cta = 0, max_units = 0, down_split = 1, o_split = 1, max_stage_k = 0;
+  const int32_t* layer_map = nullptr;  // device: layer -> layer of the packed streams (null: identity)
+  int n_src_layers = 0;                // layers in the packed streams
 };
 
 // Device-side view of the weights packed for the tensor-core projections of batched forwards (tc.h).

@@ -125,6 +125,10 @@ struct FastParams {
   const bf16* embed;
   const double* inv_freq;
   int L, d, Hq, Hkv, hd, hd_shift, F, V, vocab_in;  // hd = 1 << hd_shift
+  // A model that inherits layers of another: layer l runs the packed weights of source layer
+  // layer_map[l] (null: identity); n_src_layers = layers in the packed streams, before the head.
+  const int32_t* layer_map;
+  int n_src_layers;
   float eps;
   // streams
   bf16* kv;
