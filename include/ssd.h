@@ -112,8 +112,10 @@ void ssd_model_destroy(ssd_model* m);
  * shape of the paper's draft model (Sec. 2.3: a shallower copy of the target built from its own
  * layers - in the experiments the target's lower two and upper six of 24 - before fine-tuning):
  * the draft pass then re-reads weights the verify pass has just pulled through L2 and adds no
- * weight memory.  dev_arena (256-byte aligned, at least 256 bytes per 64 layers) receives the map;
- * `source` and its arena must outlive the new handle.  Streams for it are created as for any model. */
+ * weight memory.  dev_arena (256-byte aligned, ssd_model_inherited_arena_bytes) receives the map and
+ * the new model's own copies of the small per-layer vectors (q/k/v biases, norm gains); `source`
+ * and its arena must outlive the new handle.  Streams for it are created as for any model. */
+size_t ssd_model_inherited_arena_bytes(const ssd_model* source, int32_t n_layers);
 int ssd_model_create_inherited(const ssd_model* source, const int32_t* host_layer_map, int32_t n_layers,
                                void* dev_arena, size_t arena_bytes, ssd_model** out);
 

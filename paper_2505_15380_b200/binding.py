@@ -27,7 +27,7 @@ EXPORTS = [
     "ssd_kv_commit", "ssd_kv_restore", "ssd_accept_noalloc", "ssd_streams_inject_failure",
     "ssd_tc_gemm_scratch_bytes", "ssd_tc_gemm_check", "ssd_iteration", "ssd_paged_kv_bytes",
     "ssd_paged_workspace_bytes", "ssd_streams_create_paged", "ssd_paged_state",
-    "ssd_model_create_inherited",
+    "ssd_model_create_inherited", "ssd_model_inherited_arena_bytes",
     "ssd_kernel_launch_count",
     "ssd_last_status", "ssd_last_cuda_error", "ssd_strerror",
 ]
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
     L.ssd_model_arena_bytes.argtypes = [cfgp]
     L.ssd_model_create.argtypes = [cfgp, vp, sz, vp, sz, ctypes.POINTER(vp)]
     L.ssd_model_create_inherited.argtypes = [vp, vp, i32, vp, sz, ctypes.POINTER(vp)]
+    L.ssd_model_inherited_arena_bytes.restype = sz
+    L.ssd_model_inherited_arena_bytes.argtypes = [vp, i32]
     L.ssd_model_destroy.restype = None
     L.ssd_model_destroy.argtypes = [vp]
     L.ssd_kv_bytes.restype = sz
@@ -192,7 +194,7 @@ class InheritedModel(Model):
         self.device = source.device
         m = np.ascontiguousarray(self.layer_map, dtype=np.int32)
         with torch.cuda.device(self.device):
-            self.arena = _alloc(max(256, 4 * len(m)), self.device)
+            self.arena = _alloc(L.ssd_model_inherited_arena_bytes(source.handle, len(m)), self.device)
             h = ctypes.c_void_p()
             check(L.ssd_model_create_inherited(source.handle, m.ctypes.data, len(m), self.arena.data_ptr(),
                                                self.arena.numel(), ctypes.byref(h)))

@@ -595,15 +595,24 @@ int ssd_model_create(const ssd_model_config* cfg, const void* host_weights, size
   return SSD_OK;
 }
 
+size_t ssd_model_inherited_arena_bytes(const ssd_model* source, int32_t n_layers) {
+  if (!source || n_layers < 1 || n_layers > 4096) return 0;
+  const ssd_model_config& c = source->cfg;
+  const size_t nq = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, d = c.d_model;
+  return align_up((size_t)n_layers * 4) + align_up((size_t)n_layers * nq * 4) +
+         align_up(((size_t)n_layers * 2 + 1) * d * 4);
+}
+
 int ssd_model_create_inherited(const ssd_model* source, const int32_t* host_layer_map, int32_t n_layers,
                                void* dev_arena, size_t arena_bytes, ssd_model** out) {
   if (!source || !host_layer_map || !dev_arena || !out) return SSD_ERR_NULL;
   if (n_layers < 1 || n_layers > 4096) return SSD_ERR_BAD_CONFIG;
+  const ssd_model_config& c = source->cfg;
   for (int i = 0; i < n_layers; ++i)
-    if (host_layer_map[i] < 0 || host_layer_map[i] >= source->cfg.n_layers) return SSD_ERR_BAD_CONFIG;
+    if (host_layer_map[i] < 0 || host_layer_map[i] >= c.n_layers) return SSD_ERR_BAD_CONFIG;
   if ((uintptr_t)dev_arena & 255) return SSD_ERR_MISALIGNED;
-  if (arena_bytes < align_up((size_t)n_layers * 4)) return SSD_ERR_TOO_SMALL;
-  ssd_model* m = new (std::nothrow) ssd_model(*source);  // same pointers: nothing is copied
+  if (arena_bytes < ssd_model_inherited_arena_bytes(source, n_layers)) return SSD_ERR_TOO_SMALL;
+  ssd_model* m = new (std::nothrow) ssd_model(*source);  // same pointers: no weight is copied
   if (!m) return SSD_ERR_CUDA;
   m->cfg.n_layers = n_layers;
   m->arena = (char*)dev_arena;
@@ -613,12 +622,34 @@ int ssd_model_create_inherited(const ssd_model* source, const int32_t* host_laye
     m->layers[i] = source->layers[host_layer_map[i]];
     if (source->tc.enabled) m->tc.layers[i] = source->tc.layers[host_layer_map[i]];
   }
-  cudaError_t e = cudaMemcpy(dev_arena, host_layer_map, (size_t)n_layers * 4, cudaMemcpyHostToDevice);
+  char* A = (char*)dev_arena;
+  cudaError_t e = cudaMemcpy(A, host_layer_map, (size_t)n_layers * 4, cudaMemcpyHostToDevice);
+  m->fast.layer_map = (const int32_t*)A;  // n_src_layers stays the source's
+  if (source->fast.enabled) {
+    // The persistent kernel indexes q/k/v biases and norm gains by the model's own layer number:
+    // small arrays, gathered here in the new model's layer order (the weights themselves are walked
+    // in place through the layer map).
+    const size_t nq = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, d = c.d_model;
+    float* bias = (float*)(A + align_up((size_t)n_layers * 4));
+    float* gains = (float*)((char*)bias + align_up((size_t)n_layers * nq * 4));
+    for (int i = 0; i < n_layers && e == cudaSuccess; ++i) {
+      const int src = host_layer_map[i];
+      e = cudaMemcpy(bias + (size_t)i * nq, source->fast.bias_qkv + (size_t)src * nq, nq * 4, cudaMemcpyDeviceToDevice);
+      if (e == cudaSuccess)
+        e = cudaMemcpy(gains + (size_t)i * 2 * d, source->fast.gains + (size_t)src * 2 * d, 2 * d * 4,
+                       cudaMemcpyDeviceToDevice);
+    }
+    if (e == cudaSuccess)  // the final norm follows the last source layer
+      e = cudaMemcpy(gains + (size_t)n_layers * 2 * d, source->fast.gains + (size_t)source->fast.n_src_layers * 2 * d,
+                     d * 4, cudaMemcpyDeviceToDevice);
+    m->fast.bias_qkv = bias;
+    m->fast.gains = gains;
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete m;
     return cuda_fail(e, "ssd_model_create_inherited copy");
   }
-  m->fast.layer_map = (const int32_t*)dev_arena;  // n_src_layers stays the source's
   *out = m;
   return SSD_OK;
 }

@@ -126,11 +126,24 @@ __device__ __forceinline__ float fix_to_float(long long v) {
   return fmaf(__uint2float_rn(lo), FIX_INV_SCALE, __int2float_rn(hi));
 }
 
+// Where each layer's part of a warp's stream starts: base + (source layer) * layer_bytes.  A model
+// that inherits layers of another (a draft made of some of the target's layers) walks the same
+// stream in the order of its layer map, so the source pointer jumps at layer boundaries.  Touched
+// once per layer only, hence kept in shared memory (behind the warp's chunk table), not in the
+// ring's registers.
+struct RingSide {
+  const uint8_t* base;
+  const int32_t* map;   // layer -> source layer, or null: identity
+  uint32_t layer_bytes;
+  uint32_t cur, n_src;  // layer being requested; layers in the packed stream (the head follows them)
+};
+
 // Per-CTA bookkeeping in shared memory.
 struct FastMisc {
   unsigned long long bars[FAST_WARPS][FAST_MAX_SLOTS];
   unsigned long long sbar[FAST_WARPS];          // per warp: arrival of its slice of the A operand
-  uint8_t chunks[FAST_WARPS][FAST_MAX_CHUNKS];  // chunk sizes (tiles) of each warp's stream
+  // chunk sizes (tiles) of each warp's stream, followed by the warp's RingSide record
+  alignas(8) uint8_t chunks[FAST_WARPS][FAST_MAX_CHUNKS + sizeof(RingSide)];
   int32_t ucnt[FOP_COUNT];
   int32_t utile[FOP_COUNT][FAST_MAX_UNITS];
   float inv_rms[FAST_MAX_T];
@@ -142,12 +155,6 @@ struct FastMisc {
 
 __device__ __forceinline__ void prefetch_l2(const void* p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
-
-// Layer of the packed weights (and of the bias / gain arrays) that the model's layer l uses;
-// l = number of layers addresses what follows the last source layer (final norm, LM head).
-__device__ __forceinline__ int src_layer(const FastParams& P, int l) {
-  return l >= P.L ? P.n_src_layers : (P.layer_map ? P.layer_map[l] : l);
 }
 
 // A warp's private weight stream and shared-memory ring; every lane keeps an identical copy in
@@ -163,38 +170,41 @@ struct Ring {
   uint32_t nslot;
   uint32_t outstanding;     // copies issued and not yet waited for
   bool dead;                // a bounded wait ran out
-  // Where each layer's part of the stream starts: base + (source layer) * layer_bytes.  A model
-  // that inherits layers of another (a draft made of some of the target's layers) walks the same
-  // stream in the order of its layer map, so the source pointer jumps at layer boundaries.
-  const uint8_t* base;
-  uint32_t layer_bytes;
-  const int32_t* map;       // draft layer -> source layer, or null: identity
-  uint32_t cur, n_src;      // layer being requested; layers in the packed stream (the head follows them)
-  bool jump;                // the next request starts at jump_src
-  const uint8_t* jump_src;
+  bool mapped;              // the model walks another model's stream by a layer map (see RingSide)
   uint64_t policy;          // L2 eviction priority of the stream's copies, made once (making it
                             // anew for every copy cost 11 us per forward)
 };
 
-// Tiles of the next chunk to request (0: the stream is exhausted).
-__device__ __forceinline__ uint32_t ring_next_chunk(Ring& r) {
+// A mapped stream (a model that inherits layers of another) at a layer boundary: where the next
+// layer's chunks start.  Out of line: once per layer and warp, and only for such models.
+__device__ __noinline__ const uint8_t* ring_boundary_src(const uint8_t* tab, bool more_layers) {
+  RingSide* sd = reinterpret_cast<RingSide*>(const_cast<uint8_t*>(tab) + FAST_MAX_CHUNKS);
+  uint32_t next = sd->n_src;  // the head's chunks follow the last source layer
+  if (more_layers) {
+    const uint32_t cur = sd->cur + 1;
+    next = (uint32_t)sd->map[cur];
+    __syncwarp();
+    sd->cur = cur;            // every lane writes the same value
+    __syncwarp();
+  }
+  return sd->base + (size_t)next * sd->layer_bytes;
+}
+// Tiles of the next chunk to request (0: the stream is exhausted); `boundary`: it was the last
+// chunk of a layer.
+__device__ __forceinline__ uint32_t ring_next_chunk(Ring& r, bool& boundary) {
+  boundary = false;
   if (r.pc >= r.nend) return 0u;
   const uint32_t n = r.tab[r.pc];
   ++r.pc;
   if (r.layers_left > 0 && r.pc == r.ncl) {
-    uint32_t next = r.n_src;            // the head's chunks follow the last source layer
-    if (--r.layers_left > 0) {
-      r.pc = 0;                         // next layer: same chunk sizes; else fall through to the head
-      ++r.cur;
-      next = r.map ? (uint32_t)r.map[r.cur] : r.cur;
-    }
-    r.jump = true;
-    r.jump_src = r.base + (size_t)next * r.layer_bytes;
+    if (--r.layers_left > 0) r.pc = 0;  // next layer: same chunk sizes; else fall through to the head
+    boundary = true;
   }
   return n;
 }
 __device__ __forceinline__ void ring_request(Ring& r, uint32_t slot, int lane) {
-  const uint32_t n = ring_next_chunk(r);
+  bool boundary;
+  const uint32_t n = ring_next_chunk(r, boundary);
   if (n) {
     if (lane == 0) {
       const uint32_t bar = r.bars + slot * 8;
@@ -202,10 +212,7 @@ __device__ __forceinline__ void ring_request(Ring& r, uint32_t slot, int lane) {
       bulk_g2s_hint(r.ring + slot * FAST_SLOT_BYTES, r.src, n * FAST_TILE_BYTES, bar, r.policy);
     }
     r.src += n * FAST_TILE_BYTES;
-    if (r.jump) {
-      r.src = r.jump_src;
-      r.jump = false;
-    }
+    if (boundary && r.mapped) r.src = ring_boundary_src(r.tab, r.layers_left > 0);
     r.outstanding++;
   }
 }
@@ -1115,7 +1122,7 @@ __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint
                                           const PhaseCtx& C, int l, uint32_t& stage_parity) {
   const int d = P.d;
   PhaseDesc D;
-  D.layer = src_layer(P, l);  // of the weights' side arrays; the cache is indexed by l
+  D.layer = l;
   D.qscale = C.qscale;
   D.kv_layer = P.kv + (size_t)l * P.kv_layer_elems;
   D.xin = nullptr;
@@ -1129,7 +1136,7 @@ __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint
   D.n_rows = d;
   if (PH == 1) {
     D.op = FOP_O; D.epi = EPI_F_RESID;
-    D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)D.layer * 2 * d + d;
+    D.xout = P.xb; D.ssq_out = P.ssq_b; D.gain_next = P.m.gains + (size_t)l * 2 * d + d;
     D.cinc = (int)blockIdx.x % P.m.o_split == 0 ? 1 - P.m.o_split : 1;
     if (P.hd == 64) attn_o_phase<64, T16, LO, KSPLIT>(P, M, uni, ring, D, l, C.ks_base);
     else if (P.hd == 128) attn_o_phase<128, T16, LO, KSPLIT>(P, M, uni, ring, D, l, C.ks_base);
@@ -1146,7 +1153,7 @@ __device__ __forceinline__ void run_phase(const FastParams& P, FastMisc& M, uint
     D.op = FOP_DOWN; D.epi = EPI_F_RESID;
     D.xin = P.xd + (size_t)(C.dk0 >> 4) * (32 * Lay<T16, LO>::W); D.kc = C.dk1 - C.dk0;
     D.xout = P.xa; D.ssq_out = P.ssq_a; D.cinc = C.dsl == 0 ? 1 - P.m.down_split : 1;
-    D.gain_next = P.m.gains + (size_t)src_layer(P, l + 1) * 2 * d;  // next layer's input norm, or the final norm
+    D.gain_next = P.m.gains + (size_t)(l + 1) * 2 * d;  // next layer's input norm, or the final norm
   } else {
     D.op = FOP_HEAD; D.epi = EPI_F_LOGITS; D.in_fix = 1; D.xin = P.xa; D.ssq_in = P.ssq_a;
     D.layer = 0; D.kc = d; D.n_rows = P.V;
@@ -1191,7 +1198,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   Ring ring;
   ring.ring = smem_u32(smem) + warp * P.ring_warp_bytes;
   ring.bars = smem_u32(&M.bars[warp][0]);
-  ring.base = P.m.wstream + P.m.stream_off[wi];
   ring.tab = M.chunks[warp];
   ring.ncl = (uint32_t)P.m.chunk_cnt[wi * 2];
   ring.nend = ring.ncl + (P.logits ? (uint32_t)P.m.chunk_cnt[wi * 2 + 1] : 0u);
@@ -1212,13 +1218,20 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
   {
     uint32_t lb = 0;
     for (uint32_t i = 0; i < ring.ncl; ++i) lb += ring.tab[i];
-    ring.layer_bytes = lb * FAST_TILE_BYTES;
-    ring.map = P.layer_map;
-    ring.n_src = (uint32_t)P.n_src_layers;
-    ring.cur = 0;
-    ring.jump = false;
-    ring.jump_src = nullptr;
-    ring.src = ring.base + (size_t)(ring.ncl ? src_layer(P, 0) : P.n_src_layers) * ring.layer_bytes;
+    lb *= FAST_TILE_BYTES;
+    const uint8_t* base = P.m.wstream + P.m.stream_off[wi];
+    if (lane == 0) {
+      RingSide* sd = reinterpret_cast<RingSide*>(M.chunks[warp] + FAST_MAX_CHUNKS);
+      sd->base = base;
+      sd->map = P.layer_map;
+      sd->layer_bytes = lb;
+      sd->cur = 0;
+      sd->n_src = (uint32_t)P.n_src_layers;
+    }
+    __syncwarp();
+    ring.mapped = P.layer_map != nullptr;
+    ring.src = base;
+    if (ring.mapped) ring.src = base + (size_t)(ring.ncl ? P.layer_map[0] : P.n_src_layers) * lb;
   }
   for (int s = 0; s < P.nslot; ++s) ring_request(ring, (uint32_t)s, lane);
   const uint32_t epoch_base = ld_acquire_u32(P.epoch_base);
@@ -1241,7 +1254,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       id = min(max(id, 0), P.vocab_in - 1);
     }
     const __nv_bfloat162* src = reinterpret_cast<const __nv_bfloat162*>(P.embed + (size_t)id * d);
-    const float2* g0 = reinterpret_cast<const float2*>(P.m.gains + (size_t)src_layer(P, 0) * 2 * d);  // first layer's input norm
+    const float2* g0 = reinterpret_cast<const float2*>(P.m.gains);  // first layer's input norm
     for (int kk0 = 0; kk0 < (d >> 1); kk0 += FAST_THREADS) {         // column pairs; a warp = 64 columns
       const int kk = kk0 + tid;
       long long ss = 0;
@@ -1289,9 +1302,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) fast_forward_kernel(const __g
       // the small per-layer constants are read once per forward, so they would miss all the way
       // to HBM in the middle of an epilogue: one CTA pulls the next layer's into L2 ahead of time
       const int nq = (P.Hq + 2 * P.Hkv) * P.hd;
-      const int ls = src_layer(P, l + 1);
-      const uint8_t* bq = reinterpret_cast<const uint8_t*>(P.m.bias_qkv + (size_t)ls * nq);
-      const uint8_t* gq = reinterpret_cast<const uint8_t*>(P.m.gains + (size_t)ls * 2 * d);
+      const uint8_t* bq = reinterpret_cast<const uint8_t*>(P.m.bias_qkv + (size_t)(l + 1) * nq);
+      const uint8_t* gq = reinterpret_cast<const uint8_t*>(P.m.gains + (size_t)(l + 1) * 2 * d);
       for (int i = tid; i < ((nq * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(bq + (size_t)i * 128);
       for (int i = tid; i < ((3 * d * 4 + 127) >> 7); i += FAST_THREADS) prefetch_l2(gq + (size_t)i * 128);
     }
