@@ -28,9 +28,37 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent forward kernel, from
-# the ncu capture summarised under profiles/ (null once the kernel has changed since)
-TRAFFIC_BYTES = {"cfg1_qwen2style_b1": 735782400}
+KERNEL_SOURCES = ("fast_kernel.cuh", "fast.h", "fast_verify.cu", "fast_pack.cu")
+
+
+def kernel_sources_sha1():
+    """Hash of the persistent forward kernel's sources: ties a profile summary to the code it measured."""
+    import hashlib
+    h = hashlib.sha1()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2505_15380_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def profiled_traffic(workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent forward kernel,
+    read from the ncu summary under profiles/; None when there is no summary for this workload or
+    the kernel's sources have changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", f"fast_forward_kernel_{workload}_ncu_sections.md")
+    if not os.path.exists(path):
+        return None
+    fields = {}
+    for line in open(path):
+        if ":" in line:
+            k, v = line.split(":", 1)
+            fields[k.strip().strip("`*- ")] = v.strip().strip("`")
+    if fields.get("kernel_sources_sha1") != kernel_sources_sha1():
+        return None
+    try:
+        return int(fields["dram_bytes_per_launch"])
+    except (KeyError, ValueError):
+        return None
 
 
 def _measured_peaks():
@@ -393,7 +421,7 @@ def run_cuda(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_step": alg_bytes, "traffic": TRAFFIC_BYTES.get(wl.name) if persistent else None,
+                     "algorithmic_bytes_per_step": alg_bytes, "traffic": profiled_traffic(wl.name) if persistent else None,
                      "kernel": ("fast_forward_kernel (persistent decoder forward, one launch)" if persistent
                                 else "whole verify step (all launches of one graph replay)"),
                      "kernel_us": kern_us, "kernel_share_of_step": kern_us / us,
@@ -430,7 +458,12 @@ def main():
                     help="SSD iterations timed for the tokens/s figure (0: skip the loop)")
     ap.add_argument("--synthetic-kv", action="store_true",
                     help="seed the prefix K/V with noise instead of running a prefill (short profiling runs)")
+    ap.add_argument("--print-kernel-hash", action="store_true",
+                    help="print the hash of the persistent kernel's sources (for a profile summary) and exit")
     args = ap.parse_args()
+    if args.print_kernel_hash:
+        print(kernel_sources_sha1())
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -327,8 +327,9 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
   // key splits of the attention: whole 64-key tiles, and at most two CTAs per SM in all, which
   // is what fits at once (a second, partly filled wave would cost as much as the first)
   const int G = c.n_q_heads / c.n_kv_heads, rowgroups = (G * rm.R + 63) / 64;
-  long long kps = ((long long)s->cap * rm.nb * c.n_kv_heads * rowgroups + 2LL * n_sm - 1) / (2LL * n_sm);
-  kps = (kps + 63) / 64 * 64;
+  long long want = (2LL * n_sm) / ((long long)rm.nb * c.n_kv_heads * rowgroups);  // splits that still fit one wave
+  if (want < 1) want = 1;
+  long long kps = ((s->cap + want - 1) / want + 63) / 64 * 64;
   if (kps < 64) kps = 64;
   while ((s->cap + kps - 1) / kps > 128) kps += 64;  // the merge kernel's table of splits
   const int nsplit = (int)((s->cap + kps - 1) / kps);
@@ -834,7 +835,15 @@ void release_pages(ssd_streams* s, cudaStream_t st) {
 
 extern "C" {
 
-void ssd_streams_destroy(ssd_streams* s) { delete s; }
+void ssd_streams_destroy(ssd_streams* s) {
+  if (!s) return;
+  if (s->copy_stream) {
+    cudaStreamDestroy(s->copy_stream);
+    cudaEventDestroy(s->ev_free);
+    cudaEventDestroy(s->ev_probs);
+  }
+  delete s;
+}
 
 int ssd_fast_plan_host(const ssd_model_config* cfg, int32_t n_cta, int64_t* out8) {
   if (!cfg || !out8) return SSD_ERR_NULL;
@@ -1018,6 +1027,40 @@ int ssd_iteration(ssd_model* target, ssd_streams* ts, ssd_model* draft, ssd_stre
   return SSD_OK;
 }
 
+}  // extern "C"
+
+namespace {
+
+// ssd_verify's body; `probs_ready` (may be null) is an event the acceptance kernel waits for: the
+// host-buffer entry uploads the draft rows on a side stream while the forward, which does not
+// read them, is already running.
+int verify_impl(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens,
+                const float* dev_draft_probs, const float* dev_uniforms, const ssd_verify_params* params,
+                int32_t* dev_accepted_len, int32_t* dev_next_token, float* dev_logits_or_null,
+                cudaStream_t st, cudaEvent_t probs_ready) {
+  const int gamma = params->gamma;
+  float* logits = dev_logits_or_null ? dev_logits_or_null : s->logits;
+  const RowMap rm{0, s->B, gamma + 1};
+  int rc;
+  if (use_fast(target, s, rm)) {
+    rc = forward_fast(target, s, rm, nullptr, dev_draft_tokens, logits, st);
+  } else {
+    launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
+    rc = forward(target, s, rm, logits, st);
+  }
+  if (rc != SSD_OK) return rc;
+  if (probs_ready) SSD_CUDA(cudaStreamWaitEvent(st, probs_ready, 0));
+  SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
+                                 dev_uniforms, s->B, gamma, 1.0f / params->temperature,
+                                 params->top_k, params->top_p, params->beta, s->row_stats, s->accept_flags,
+                                 s->counters, dev_accepted_len, dev_next_token, s->status, st));
+  return SSD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens,
                const float* dev_draft_probs, const float* dev_uniforms,
                const ssd_verify_params* params, int32_t* dev_accepted_len,
@@ -1028,22 +1071,8 @@ int ssd_verify(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_token
   if (!same_shape(target->cfg, s->cfg)) return SSD_ERR_BAD_CONFIG;
   int rc = params_ok(s, params, true);
   if (rc != SSD_OK) return rc;
-  cudaStream_t st = (cudaStream_t)stream;
-  const int gamma = params->gamma;
-  float* logits = dev_logits_or_null ? dev_logits_or_null : s->logits;
-  const RowMap rm{0, s->B, gamma + 1};
-  if (use_fast(target, s, rm)) {
-    rc = forward_fast(target, s, rm, nullptr, dev_draft_tokens, logits, st);
-  } else {
-    launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
-    rc = forward(target, s, rm, logits, st);
-  }
-  if (rc != SSD_OK) return rc;
-  SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
-                                 dev_uniforms, s->B, gamma, 1.0f / params->temperature,
-                                 params->top_k, params->top_p, params->beta, s->row_stats, s->accept_flags,
-                                 s->counters, dev_accepted_len, dev_next_token, s->status, st));
-  return SSD_OK;
+  return verify_impl(target, s, dev_draft_tokens, dev_draft_probs, dev_uniforms, params, dev_accepted_len,
+                     dev_next_token, dev_logits_or_null, (cudaStream_t)stream, nullptr);
 }
 
 int ssd_kv_commit(ssd_streams* s, const int32_t* dev_accepted_len, const int32_t* dev_next_token,
@@ -1070,11 +1099,22 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
   if (rc != SSD_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t B = s->B, g = params->gamma, V = s->cfg.vocab_out;
+  if (!s->copy_stream) {  // side stream and events of the overlapped upload, made on first use
+    SSD_CUDA(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
+    SSD_CUDA(cudaEventCreateWithFlags(&s->ev_free, cudaEventDisableTiming));
+    SSD_CUDA(cudaEventCreateWithFlags(&s->ev_probs, cudaEventDisableTiming));
+  }
+  // The draft rows are by far the largest input and only the acceptance kernel reads them: they
+  // travel on the side stream (after whatever still reads the staging buffer on `stream`) while
+  // the small inputs go ahead and the forward starts.
+  SSD_CUDA(cudaEventRecord(s->ev_free, st));
+  SSD_CUDA(cudaStreamWaitEvent(s->copy_stream, s->ev_free, 0));
+  SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, s->copy_stream));
+  SSD_CUDA(cudaEventRecord(s->ev_probs, s->copy_stream));
   SSD_CUDA(cudaMemcpyAsync(s->st_tokens, host_draft_tokens, B * g * 4, cudaMemcpyHostToDevice, st));
-  SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, st));
   SSD_CUDA(cudaMemcpyAsync(s->st_uni, host_uniforms, B * (g + 1) * 2 * 4, cudaMemcpyHostToDevice, st));
-  rc = ssd_verify(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr,
-                  stream);
+  rc = verify_impl(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr, st,
+                   s->ev_probs);
   if (rc != SSD_OK) return rc;
   rc = ssd_kv_commit(s, s->st_k, s->st_y, stream);
   if (rc != SSD_OK) return rc;

@@ -141,6 +141,9 @@ struct ssd_streams {
   // and the partial sums of the K-split projections
   uint8_t *tc_xa, *tc_xattn, *tc_xact;
   float* tc_part;
+  // host-buffer entry: side stream for the upload of the draft rows, and its two events
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_free = nullptr, ev_probs = nullptr;
   int split_act;     // persistent kernel: activations as bf16 hi + lo pairs (1) or plain bf16 (0)
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)

@@ -49,6 +49,33 @@ enum TcEpilogue {
   TC_EPI_SWIGLU = 2    // rows interleaved (gate_j, up_j): packed[token, j] = SiLU(gate) * up
 };
 
+// Programmatic dependent launch: the kernels of the batched forward form one dependency chain
+// of ~200 short launches.  Each lets its successor start launching at once (tc_pdl_trigger) and
+// waits for its predecessor's results only where it first needs them (tc_pdl_wait, which returns
+// when the whole preceding grid has completed and its writes are visible), so launch latency and
+// set-up - and, in the projections, the first weight copies, which depend on nothing - overlap the
+// predecessor's tail.  Nothing that blocks on a shared resource (tensor memory) is taken before
+// the wait.  Without the launch attribute both instructions do nothing.
+#ifdef __CUDACC__
+__device__ __forceinline__ void tc_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void tc_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t tc_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 inline int tc_round16(int m) { return (m + 15) / 16 * 16; }
 inline size_t tc_weight_bytes(int n_rows, int K) {
   return (size_t)((n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS) * ((K + 15) / 16) * TC_WBLOCK;

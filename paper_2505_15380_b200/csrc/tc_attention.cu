@@ -24,6 +24,11 @@ namespace ssd {
 namespace {
 
 constexpr int TA_WARPS = 4;
+// The softmax weights P enter the second contraction as bf16 leading part + remainder.  Rounding
+// them to bf16 instead (one instruction fewer in four) was measured: the logits of the 24- and
+// 28-layer models then differ from the float64 oracle by 2.0e-2 and 1.4e-2, against 1e-4 with the
+// split - too close to the 3e-2 bound to be the default.
+constexpr bool TA_SPLIT_P = true;
 constexpr int TA_TILE = 64;  // keys per tile
 static_assert(TA_TILE == TC_PAGE_TOKENS, "a key tile of the batched attention is one page of a paged cache");
 
@@ -70,6 +75,8 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
 
   const int sp = blockIdx.x, gk = blockIdx.y / n_rowgroups, rg = blockIdx.y % n_rowgroups, bi = blockIdx.z;
   const int b = rm.b0 + bi, R = rm.R, G = Hq / Hkv, NQ = G * R;
+  tc_pdl_trigger();
+  tc_pdl_wait();
   const int L = len[b], total = min(L + R, cap);
   const int k_begin = sp * keys_per_split;
   if (k_begin >= total) return;
@@ -223,9 +230,9 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
           uint32_t b0, b1, b2, b3;
           ldmatrix_x4_trans(v_addr + kk * 16 * ROWB + dt * 16, b0, b1, b2, b3);
           mma_bf16(o[dt], phi, b0, b1);
-          mma_bf16(o[dt], plo, b0, b1);
+          if (TA_SPLIT_P) mma_bf16(o[dt], plo, b0, b1);
           mma_bf16(o[dt + 1], phi, b2, b3);
-          mma_bf16(o[dt + 1], plo, b2, b3);
+          if (TA_SPLIT_P) mma_bf16(o[dt + 1], plo, b2, b3);
         }
       }
     }
@@ -265,6 +272,8 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
                                      uint8_t* __restrict__ apack, int Mpad) {
   const int h = blockIdx.x, m = blockIdx.y;
   const int bi = m / rm.R, b = rm.b0 + bi;
+  tc_pdl_trigger();
+  tc_pdl_wait();
   const int total = min(len[b] + rm.R, cap);
   const int ns = (total + keys_per_split - 1) / keys_per_split;
   const float* src = part + ((size_t)m * Hq + h) * nsplit * (HD + 2);
@@ -314,12 +323,13 @@ cudaError_t launch_t(const float* qrot, const bf16* kv_layer, const int32_t* len
   auto kern = tc_attn_kernel<HD>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(nsplit, Hkv * n_rowgroups, rm.nb), TA_WARPS * 32, smem, st>>>(qrot, kv_layer, len, rm, cap, Hq, Hkv,
-                                                                             n_rowgroups, part, nsplit, keys_per_split,
-                                                                             page_table, max_pages);
+  e = tc_launch_pdl(kern, dim3(nsplit, Hkv * n_rowgroups, rm.nb), dim3(TA_WARPS * 32), smem, st, qrot, kv_layer, len, rm,
+                    cap, Hq, Hkv, n_rowgroups, part, nsplit, keys_per_split, page_table, max_pages);
+  if (e != cudaSuccess) return e;
   count_launch();
-  tc_attn_merge_kernel<HD><<<dim3(Hq, rm.nb * rm.R), HD / 2 < 32 ? 32 : HD / 2, 0, st>>>(
-      part, len, rm, cap, Hq, nsplit, keys_per_split, apack_out, Mpad);
+  e = tc_launch_pdl(tc_attn_merge_kernel<HD>, dim3(Hq, rm.nb * rm.R), dim3(HD / 2 < 32 ? 32 : HD / 2), 0, st,
+                    (const float*)part, len, rm, cap, Hq, nsplit, keys_per_split, apack_out, Mpad);
+  if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
 }

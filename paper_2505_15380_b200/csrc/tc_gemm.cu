@@ -163,6 +163,11 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     S.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  tc_pdl_trigger();
+  // The copy warp does not wait here: the first weight copies depend on nothing and go out at
+  // once.  Everyone else needs the predecessor's results (or tensor memory, which must not be
+  // held while the predecessor may still want it).
+  if (warp != 0) tc_pdl_wait();
   if (warp == 1) {  // tensor memory: one warp allocates, the same warp frees
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(&S.tmem_base)), "r"((uint32_t)P.tmem_cols) : "memory");
@@ -175,33 +180,49 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
   volatile int* abort = &S.abort;
 
   if (warp == 0) {
+    if (lane >= TC_ISSUERS) tc_pdl_wait();
     if (lane < TC_ISSUERS) {  // ---- operand copies: piece i of a stage is issued by lane i % TC_ISSUERS
       const uint64_t pol = policy_evict_first();
       const uint8_t* wsrc = P.w + ((size_t)tile * P.KS + ks0) * TC_WBLOCK;
       const uint8_t* asrc = P.a + (size_t)ks0 * act_block;
-      int it = 0;
-      for (; it < n_iter; ++it) {
-        const int s = it % P.stages, use = it / P.stages;
-        if (use > 0 && !mbar_wait(smem_u32(&S.empty[s]), (uint32_t)(use - 1) & 1u, abort)) break;
+      // One stage's pieces; which = 1: weights, 2: activations, 3: both.  A lane arrives once per
+      // stage (with the weights, or with `both`), announcing all the bytes it will bring.
+      auto issue = [&](int it, int which) {
+        const int s = it % P.stages;
         const int nks = min(P.sk, ks1 - ks0 - it * P.sk);
         const uint32_t bar = smem_u32(&S.full[s]);
         const uint32_t wbytes = (uint32_t)nks * TC_WBLOCK, abytes = (uint32_t)nks * act_block;
         const uint32_t wp = (wbytes + TC_PIECE - 1) / TC_PIECE, ap = (abytes + TC_PIECE - 1) / TC_PIECE;
-        uint32_t mine = 0;
-        for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS)
-          mine += i < wp ? min(TC_PIECE, wbytes - i * TC_PIECE) : min(TC_PIECE, abytes - (i - wp) * TC_PIECE);
-        mbar_expect_tx(bar, mine);  // every issuing lane arrives once per stage, with its own byte count
+        const uint8_t* ws = wsrc + (size_t)it * P.sk * TC_WBLOCK;
+        const uint8_t* as = asrc + (size_t)it * P.sk * act_block;
+        if (which & 1) {
+          uint32_t mine = 0;
+          for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS)
+            mine += i < wp ? min(TC_PIECE, wbytes - i * TC_PIECE) : min(TC_PIECE, abytes - (i - wp) * TC_PIECE);
+          mbar_expect_tx(bar, mine);
+        }
         for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS) {
           if (i < wp) {
             const uint32_t off = i * TC_PIECE;
-            bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w) + off, wsrc + off, min(TC_PIECE, wbytes - off), bar, pol);
+            if (which & 1)
+              bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w) + off, ws + off, min(TC_PIECE, wbytes - off), bar, pol);
           } else {
             const uint32_t off = (i - wp) * TC_PIECE;
-            bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a) + off, asrc + off, min(TC_PIECE, abytes - off), bar);
+            if (which & 2)
+              bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a) + off, as + off, min(TC_PIECE, abytes - off), bar);
           }
         }
-        wsrc += wbytes;
-        asrc += abytes;
+      };
+      // first fill of the ring: the weights at once, the activations when the predecessor is done
+      const int first = min(n_iter, P.stages);
+      for (int it = 0; it < first; ++it) issue(it, 1);
+      tc_pdl_wait();
+      for (int it = 0; it < first; ++it) issue(it, 2);
+      int it = first;
+      for (; it < n_iter; ++it) {
+        const int s = it % P.stages, use = it / P.stages;
+        if (!mbar_wait(smem_u32(&S.empty[s]), (uint32_t)(use - 1) & 1u, abort)) break;
+        issue(it, 3);
       }
       if (*abort) {
         // never leave with copies in flight into this CTA's shared memory: the last uses of the
@@ -398,7 +419,8 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   const size_t smem = (size_t)p.stages * p.sk * per_ks + sizeof(TcShared) + 64;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
-  tc_gemm_kernel<<<dim3(tiles, g.ksplit), TC_THREADS, smem, st>>>(p);
+  e = tc_launch_pdl(tc_gemm_kernel, dim3(tiles, g.ksplit), dim3(TC_THREADS), smem, st, p);
+  if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
 }

@@ -51,6 +51,8 @@ tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int n
   extern __shared__ float row[];
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
+  tc_pdl_trigger();
+  tc_pdl_wait();
   float ss = 0.f;
   for (int j = tid * 2; j < d; j += 512) {
     float2 v = *reinterpret_cast<const float2*>(h + (size_t)m * d + j);
@@ -92,6 +94,8 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
                    int32_t* status) {
   extern __shared__ float row[];  // [(Hq + 2 Hkv) * hd]
   const int m = blockIdx.x, tid = threadIdx.x;
+  tc_pdl_trigger();
+  tc_pdl_wait();
   const int bi = m / rm.R, r = m % rm.R, b = rm.b0 + bi;
   const int pos = len[b] + r, half = hd >> 1, nq = (Hq + 2 * Hkv) * hd;
   for (int j = tid * 2; j < nq; j += 512) {
@@ -143,8 +147,8 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
 
 void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, int M, int d,
                          const bf16* gain, float eps, uint8_t* apack, cudaStream_t st) {
-  tc_norm_pack_kernel<<<M, 256, (size_t)d * 4, st>>>(h, part, part ? nsplit : 0, ld_part, tc_round16(M), d, gain,
-                                                     eps, apack);
+  tc_launch_pdl(tc_norm_pack_kernel, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0, ld_part,
+                tc_round16(M), d, gain, eps, apack);
   count_launch();
 }
 
@@ -159,8 +163,8 @@ void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, co
                         int32_t* status, cudaStream_t st) {
   const int M = rm.nb * rm.R;
   const size_t smem = (size_t)(Hq + 2 * Hkv) * hd * 4;
-  tc_qkv_post_kernel<<<M, 256, smem, st>>>(part, nsplit, ld_part, Mpad, bias, cs, qrot, kv_layer, len, rm, cap, Hq,
-                                           Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
+  tc_launch_pdl(tc_qkv_post_kernel, dim3(M), dim3(256), smem, st, part, nsplit, ld_part, Mpad, bias, cs, qrot,
+                kv_layer, len, rm, cap, Hq, Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
   count_launch();
 }
 
