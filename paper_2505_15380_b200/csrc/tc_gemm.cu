@@ -390,7 +390,8 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   p.act_out = g.act_out;
   p.status = g.status;
   if (g.ksplit > p.KS || (g.epi != TC_EPI_PARTIAL && g.ksplit != 1)) return cudaErrorInvalidValue;
-  // pipeline: at least four stages (when one k-step fits four times) of as many k-steps as fit.  A grid that exceeds the SM count
+  // pipeline: at least three stages of as many k-steps as fit (measured at 448 rows: six stages
+  // of one k-step are 12 % slower than three of two - fewer, larger copies win).  A grid that exceeds the SM count
   // by a little leaves room for a second CTA per SM so that it still runs in one wave; any other
   // grid takes the whole shared memory: with few token rows the weight stream is latency-bound,
   // and what a CTA keeps in flight is what it gets.
@@ -406,7 +407,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   const bool two_per_sm = p.Mpad <= 128 && ctas > n_sm && ctas <= 2 * n_sm;  // 2 x 256 columns
   const size_t budget = two_per_sm ? 100 * 1024 : 216 * 1024;
   p.sk = 4;
-  while (p.sk > 1 && 4 * p.sk * per_ks > budget) p.sk >>= 1;  // at least four stages in flight
+  while (p.sk > 1 && 3 * p.sk * per_ks > budget) p.sk >>= 1;
   p.stages = (int)(budget / (p.sk * per_ks));
   if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
   if (p.stages < 2) return cudaErrorInvalidValue;
