@@ -234,8 +234,11 @@ int ssd_forward(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_toke
                 float* dev_logits, void* stream);
 
 /* Same step with HOST buffers: copies the three inputs to the device, runs ssd_verify and
- * ssd_kv_commit, copies accepted_len / next_token back and synchronises `stream`.  Host
- * buffers should be pinned for the copies to be asynchronous. */
+ * ssd_kv_commit, copies accepted_len / next_token back and synchronises `stream`.  The draft rows
+ * (by far the largest input, read only by the acceptance step) are uploaded on a side stream
+ * while the forward runs, so host_draft_probs should be pinned; the small arrays travel through
+ * a pinned staging buffer of a few hundred bytes.  The first call on a streams object creates
+ * that side stream, two events and the staging buffer (host memory; no device allocation). */
 int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft_tokens,
                     const float* host_draft_probs, const float* host_uniforms,
                     const ssd_verify_params* params, int32_t* host_accepted_len,

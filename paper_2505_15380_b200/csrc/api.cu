@@ -177,11 +177,13 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap, int n_p
   p.xn = take(M * d * 4);
   p.attn_out = take(M * qd * 4);
   p.act = take(M * F * 4);
-  p.st_tokens = take((size_t)B * max_gamma * 4);
-  p.st_k = take(B * 4);
-  p.st_y = take(B * 4);
+  // host-call staging: [tokens | uniforms] and [k | y] are each one contiguous run, so that the
+  // host-buffer entry moves them with one copy each way
+  p.st_tokens = take((size_t)B * max_gamma * 4 + M * 2 * 4);
+  p.st_k = take((size_t)2 * B * 4);
+  p.st_y = p.st_k + (size_t)B * 4;
   p.st_probs = take((size_t)B * max_gamma * V * 4);
-  p.st_uni = take(M * 2 * 4);
+  p.st_uni = p.st_tokens + (size_t)B * max_gamma * 4;
   p.hfix = take((size_t)FAST_MAX_T * d * 8);
   // operand-layout activations: per 16 columns 32 lanes x 32 bytes (16 rows, bf16 hi + lo)
   p.xa = take(d * 64);
@@ -841,6 +843,7 @@ void ssd_streams_destroy(ssd_streams* s) {
     cudaStreamDestroy(s->copy_stream);
     cudaEventDestroy(s->ev_free);
     cudaEventDestroy(s->ev_probs);
+    if (s->h_stage) cudaFreeHost(s->h_stage);
   }
   delete s;
 }
@@ -1103,6 +1106,9 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
     SSD_CUDA(cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking));
     SSD_CUDA(cudaEventCreateWithFlags(&s->ev_free, cudaEventDisableTiming));
     SSD_CUDA(cudaEventCreateWithFlags(&s->ev_probs, cudaEventDisableTiming));
+    // pinned host staging for the small inputs and the two result arrays (host memory, not device)
+    s->h_stage_in = (size_t)((char*)s->st_uni - (char*)s->st_tokens) + (size_t)s->max_rows * 2 * 4;
+    SSD_CUDA(cudaHostAlloc((void**)&s->h_stage, s->h_stage_in + 2 * B * 4, cudaHostAllocDefault));
   }
   // The draft rows are by far the largest input and only the acceptance kernel reads them: they
   // travel on the side stream (after whatever still reads the staging buffer on `stream`) while
@@ -1111,16 +1117,21 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
   SSD_CUDA(cudaStreamWaitEvent(s->copy_stream, s->ev_free, 0));
   SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, s->copy_stream));
   SSD_CUDA(cudaEventRecord(s->ev_probs, s->copy_stream));
-  SSD_CUDA(cudaMemcpyAsync(s->st_tokens, host_draft_tokens, B * g * 4, cudaMemcpyHostToDevice, st));
-  SSD_CUDA(cudaMemcpyAsync(s->st_uni, host_uniforms, B * (g + 1) * 2 * 4, cudaMemcpyHostToDevice, st));
+  // tokens and uniforms: gathered in the pinned staging buffer (a few hundred bytes), one copy
+  const size_t uni_off = (size_t)((char*)s->st_uni - (char*)s->st_tokens), uni_bytes = B * (g + 1) * 2 * 4;
+  memcpy(s->h_stage, host_draft_tokens, B * g * 4);
+  memcpy(s->h_stage + uni_off, host_uniforms, uni_bytes);
+  SSD_CUDA(cudaMemcpyAsync(s->st_tokens, s->h_stage, uni_off + uni_bytes, cudaMemcpyHostToDevice, st));
   rc = verify_impl(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr, st,
                    s->ev_probs);
   if (rc != SSD_OK) return rc;
   rc = ssd_kv_commit(s, s->st_k, s->st_y, stream);
   if (rc != SSD_OK) return rc;
-  SSD_CUDA(cudaMemcpyAsync(host_accepted_len, s->st_k, B * 4, cudaMemcpyDeviceToHost, st));
-  SSD_CUDA(cudaMemcpyAsync(host_next_token, s->st_y, B * 4, cudaMemcpyDeviceToHost, st));
+  char* h_out = s->h_stage + s->h_stage_in;  // [k | y] come back with one copy
+  SSD_CUDA(cudaMemcpyAsync(h_out, s->st_k, 2 * B * 4, cudaMemcpyDeviceToHost, st));
   SSD_CUDA(cudaStreamSynchronize(st));
+  memcpy(host_accepted_len, h_out, B * 4);
+  memcpy(host_next_token, h_out + B * 4, B * 4);
   return SSD_OK;
 }
 

@@ -144,6 +144,8 @@ struct ssd_streams {
   // host-buffer entry: side stream for the upload of the draft rows, and its two events
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_free = nullptr, ev_probs = nullptr;
+  char* h_stage = nullptr;  // pinned host staging of that entry: [tokens | uniforms] then [k | y]
+  size_t h_stage_in = 0;
   int split_act;     // persistent kernel: activations as bf16 hi + lo pairs (1) or plain bf16 (0)
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)
