@@ -17,6 +17,8 @@ What is computed, and from which passage:
                    z/T, keep the top_k largest with the lower id winning ties, then the shortest
                    prefix of those, most probable first, whose mass reaches top_p; softmax over
                    what is kept).
+* `transform_ras`- repetition-aware sampling (a nucleus draw that is redrawn from the full softmax
+                   when it repeats a recent token) written as the one distribution it samples from.
 * `accept_step`  - the sequential tolerance test r_i < min(1, q_i(x_i)/p_i(x_i)) + beta (Eq. 5),
                    the residual resample from normalize(max(0, q_i - p_i)) at the first rejection
                    (Eq. 6), and the bonus token from q_{gamma+1} when nothing is rejected
@@ -202,6 +204,31 @@ def transform(logits_row: np.ndarray, temperature: float, top_k: int, top_p: flo
     return e / e.sum()
 
 
+def transform_ras(logits_row: np.ndarray, temperature: float, top_k: int, top_p: float,
+                  window: np.ndarray, win_size: int, tau_r: float) -> np.ndarray:
+    """Repetition-aware sampling as ONE distribution (the paper is silent on samplers; this is the
+    sampler of the CosyVoice family the paper builds on, restated).
+
+    The procedure: draw a token from the nucleus / top-k distribution q_nuc; if it occurs at least
+    win_size * tau_r times among the last win_size tokens (`window`, any -1 entries ignored), throw
+    it away and draw from the full softmax q_full instead.  Its output law is
+        q(x) = q_nuc(x) * [x not repeated] + R * q_full(x),   R = sum of q_nuc over repeated ids,
+    which is the target distribution q_i that Eq. 5-6 then use.
+    """
+    q_nuc = transform(logits_row, temperature, top_k, top_p)
+    if win_size <= 0:
+        return q_nuc
+    q_full = transform(logits_row, temperature, 0, 0.0)
+    w = np.asarray(window, dtype=np.int64)[-win_size:]
+    w = w[w >= 0]
+    ids, counts = np.unique(w, return_counts=True)
+    repeated = ids[counts >= win_size * tau_r]
+    mask = np.zeros(len(q_nuc), dtype=bool)
+    mask[repeated[repeated < len(q_nuc)]] = True
+    R = float(q_nuc[mask].sum())
+    return np.where(mask, 0.0, q_nuc) + R * q_full
+
+
 # ------------------------------------------------------------------ acceptance (Eq. 5, 6)
 
 def categorical_draw(weights: np.ndarray, u: float) -> Tuple[int, float]:
@@ -254,12 +281,23 @@ def accept_step(q_rows: np.ndarray, p_rows: np.ndarray, draft_tokens: np.ndarray
 
 
 def verify(model: Model, stream: Stream, draft_tokens: np.ndarray, p_rows: np.ndarray,
-           uniforms: np.ndarray, *, temperature: float, top_k: int, beta: float, top_p: float = 0.0
+           uniforms: np.ndarray, *, temperature: float, top_k: int, beta: float, top_p: float = 0.0,
+           recent: Optional[np.ndarray] = None, win_size: int = 0, tau_r: float = 0.0
            ) -> Dict[str, object]:
-    """One full verification step for one stream (forward, transform, accept); no commit."""
+    """One full verification step for one stream (forward, transform, accept); no commit.
+
+    With win_size > 0 the target samples repetition-aware: `recent` holds the last tokens of T_in
+    (the pending token last); row i's window is the last win_size tokens of recent + x_1..x_{i-1}.
+    """
     ids = np.concatenate([[stream.pending], np.asarray(draft_tokens, np.int64)])
     logits = forward(model, stream, ids)
-    q_rows = np.stack([transform(row, temperature, top_k, top_p) for row in logits])
+    if win_size > 0:
+        hist = np.concatenate([np.asarray(recent, np.int64), np.asarray(draft_tokens, np.int64)])
+        n0 = len(recent)
+        q_rows = np.stack([transform_ras(row, temperature, top_k, top_p, hist[:n0 + i], win_size, tau_r)
+                           for i, row in enumerate(logits)])
+    else:
+        q_rows = np.stack([transform(row, temperature, top_k, top_p) for row in logits])
     res = accept_step(q_rows, p_rows, draft_tokens, uniforms, beta)
     res["logits"] = logits
     res["q_rows"] = q_rows

@@ -243,6 +243,68 @@ def test_nucleus_transform_by_hand_brute_force_and_library():
         assert np.array_equal(orc.transform(zz, 1.0, 0, tp) > 0, kept_ref)
 
 
+def test_repetition_aware_law_by_enumerating_the_two_stage_procedure():
+    """The closed form of transform_ras against a literal enumeration of the procedure: first draw
+    from the nucleus row; if that id is repeated in the window, second draw from the full row."""
+    rng = np.random.default_rng(8)
+    for trial in range(60):
+        V = int(rng.integers(4, 10))
+        z = rng.standard_normal(V) * 2
+        T = float(rng.uniform(0.6, 1.4))
+        top_k = int(rng.integers(0, V + 1))
+        top_p = float(rng.choice([0.0, 0.5, 0.8, 0.95]))
+        win = int(rng.integers(1, 8))
+        tau = float(rng.choice([0.1, 0.3, 0.5]))
+        window = rng.integers(-1, V, size=int(rng.integers(0, 12)))
+        q_nuc, q_full = orc.transform(z, T, top_k, top_p), orc.transform(z, T, 0)
+        tail = [int(t) for t in window[-win:] if t >= 0]
+        law = np.zeros(V)
+        for first in range(V):
+            if q_nuc[first] == 0:
+                continue
+            if tail.count(first) >= win * tau:
+                law += q_nuc[first] * q_full                 # thrown away, redrawn from the full row
+            else:
+                law[first] += q_nuc[first]
+        got = orc.transform_ras(z, T, top_k, top_p, window, win, tau)
+        assert np.allclose(got, law, atol=1e-14) and np.isclose(got.sum(), 1.0)
+    z = np.log(np.array([0.5, 0.3, 0.15, 0.05]))
+    # by hand: nucleus {0, 1} = (0.625, 0.375); id 0 repeated -> 0.625 of the mass is redrawn from the full row
+    got = orc.transform_ras(z, 1.0, 0, 0.79, np.array([3, 0, 2]), 10, 0.1)
+    assert np.allclose(got, [0.625 * 0.5, 0.375 + 0.625 * 0.3, 0.625 * 0.15, 0.625 * 0.05])
+    # no window, an empty window, or a threshold no count reaches: the nucleus row itself
+    nuc = orc.transform(z, 1.0, 0, 0.8)
+    assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 0]), 0, 0.1), nuc)
+    assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([-1, -1]), 4, 0.1), nuc)
+    assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 1]), 4, 0.9), nuc)
+    # only the last win_size tokens count
+    assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 2, 2, 3]), 3, 0.3), nuc)
+    # every kept id repeated: the full row
+    assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 1]), 2, 0.5), orc.transform(z, 1.0, 0))
+
+
+def test_verify_builds_each_rows_window_from_recent_tokens_and_the_draft():
+    from tests.helpers import oracle_model, small_shape
+    from paper_2505_15380_b200 import synth
+    shape = small_shape()
+    m = oracle_model(shape, synth.make_weights(shape, 2))
+    st = orc.Stream(m, 64)
+    orc.prefill(m, st, np.array([5, 9, 3, 9, 7]))
+    draft = np.array([9, 9, 4])
+    V = shape.vocab_out
+    p = np.full((3, V), 1.0 / V)
+    u = np.zeros((4, 2))
+    recent = np.array([3, 9, 7])
+    o = orc.verify(m, st, draft, p, u, temperature=1.0, top_k=5, beta=0.0, top_p=0.9, recent=recent,
+                   win_size=4, tau_r=0.5)
+    lg = o["logits"]
+    for i in range(4):
+        window = np.concatenate([recent, draft[:i]])        # row i sees x_1..x_{i-1}, not x_i
+        assert np.allclose(o["q_rows"][i], orc.transform_ras(lg[i], 1.0, 5, 0.9, window, 4, 0.5))
+    # row 2's window is [9, 7, 9, 9]: id 9 occurs 3 >= 2 times, so its nucleus mass is spread
+    assert not np.allclose(o["q_rows"][2], orc.transform(lg[2], 1.0, 5, 0.9)) or orc.transform(lg[2], 1.0, 5, 0.9)[9] == 0
+
+
 def test_accepted_length_grows_with_beta_as_in_table_3():
     """Sec. 4.3 / Table 3: a larger tolerance accepts more.  For fixed distributions, tokens and
     uniforms k(beta) never decreases, and its mean over draws follows the geometric closed form
