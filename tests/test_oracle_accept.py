@@ -273,7 +273,7 @@ def test_repetition_aware_law_by_enumerating_the_two_stage_procedure():
     got = orc.transform_ras(z, 1.0, 0, 0.79, np.array([3, 0, 2]), 10, 0.1)
     assert np.allclose(got, [0.625 * 0.5, 0.375 + 0.625 * 0.3, 0.625 * 0.15, 0.625 * 0.05])
     # no window, an empty window, or a threshold no count reaches: the nucleus row itself
-    nuc = orc.transform(z, 1.0, 0, 0.8)
+    nuc = orc.transform(z, 1.0, 0, 0.79)
     assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 0]), 0, 0.1), nuc)
     assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([-1, -1]), 4, 0.1), nuc)
     assert np.allclose(orc.transform_ras(z, 1.0, 0, 0.79, np.array([0, 1]), 4, 0.9), nuc)
