@@ -89,6 +89,18 @@ typedef struct {
   float top_p;       /* nucleus: 0 or >= 1: off; else, among the ids top_k kept, most probable first
                         (lower id first among equals), an id stays while the mass before it is
                         below top_p: the shortest such prefix whose mass reaches top_p */
+  /* Repetition-aware sampling of the TARGET (the sampler of the CosyVoice family; the paper is
+   * silent): a nucleus / top-k draw that occurs at least ras_window * ras_tau times among the last
+   * ras_window tokens is thrown away and redrawn from the full softmax.  The acceptance step uses
+   * the distribution this procedure samples from, q(x) = q_nuc(x) [x not repeated] + R q_full(x)
+   * with R = the nucleus mass of the repeated ids, as q_i in Eq. 5-6.  ras_window 0: off (at
+   * most 32).  dev_recent_tokens: int32 [B, ras_window], the last tokens of each stream's T_in,
+   * oldest first, the pending token last, -1 where the history is shorter; row i of a verify step
+   * uses the last ras_window tokens of that followed by x_1..x_{i-1}.  ssd_iteration keeps the
+   * array up to date (it appends the emitted tokens); ssd_draft_step ignores these fields. */
+  int32_t ras_window;
+  float ras_tau;
+  const int32_t* dev_recent_tokens;
 } ssd_verify_params;
 
 /* ---- model ------------------------------------------------------------------------------- */
@@ -304,7 +316,7 @@ int ssd_iteration(ssd_model* target, ssd_streams* target_streams, ssd_model* dra
  * bonus draw of Eq. 6 exactly as ssd_verify does, and writes the same two outputs.
  *   in  dev_logits float [batch, gamma+1, vocab]; dev_draft_tokens, dev_draft_probs, dev_uniforms
  *       as in ssd_verify;  out dev_accepted_len, dev_next_token int32 [batch].
- * The kernel's scratch lives in a fixed array inside the library (about 84 KB, held by every GPU
+ * The kernel's scratch lives in a fixed array inside the library (about 148 KB, held by every GPU
  * that loads the library until the process exits), sized for at most 256 streams and
  * gamma + 1 <= 16 rows: larger batches return SSD_ERR_TOO_SMALL, larger gamma SSD_ERR_BAD_GAMMA.
  * No cudaMalloc / cudaFree or allocating library routine is called.  The first call on a device

@@ -43,7 +43,9 @@ class ModelConfig(ctypes.Structure):
 
 class VerifyParams(ctypes.Structure):
     _fields_ = [("gamma", ctypes.c_int32), ("temperature", ctypes.c_float),
-                ("top_k", ctypes.c_int32), ("beta", ctypes.c_float), ("top_p", ctypes.c_float)]
+                ("top_k", ctypes.c_int32), ("beta", ctypes.c_float), ("top_p", ctypes.c_float),
+                ("ras_window", ctypes.c_int32), ("ras_tau", ctypes.c_float),
+                ("dev_recent_tokens", ctypes.c_void_p)]
 
 
 class LoopIo(ctypes.Structure):
@@ -439,7 +441,7 @@ class Loop:
     the draft streams back by one token and keeps the last two prefix ids, as the call expects."""
 
     def __init__(self, target: Streams, draft: Streams, prefixes: Sequence[np.ndarray], gamma: int,
-                 uniform_pool: np.ndarray, out_capacity: int):
+                 uniform_pool: np.ndarray, out_capacity: int, ras_window: int = 0):
         B, V = target.B, target.model.shape.vocab_out
         assert draft.B == B and len(prefixes) == B and all(len(p) >= 2 for p in prefixes)
         per = gamma + 2 * (gamma + 1)
@@ -456,6 +458,14 @@ class Loop:
         self.out_tokens = torch.zeros((B, out_capacity), dtype=torch.int32, device=dev)
         self.out_count = torch.zeros(B, dtype=torch.int32, device=dev)
         self.accept_log = torch.full((uniform_pool.shape[0], B), -9, dtype=torch.int32, device=dev)
+        # window of the repetition-aware sampler: the last tokens of each prefix, pending token last
+        self.recent = None
+        if ras_window > 0:
+            rec = np.full((B, ras_window), -1, dtype=np.int32)
+            for b, p in enumerate(prefixes):
+                tail = np.asarray(p[-ras_window:], np.int32)
+                rec[b, ras_window - len(tail):] = tail
+            self.recent = torch.from_numpy(rec).to(dev)
         lens, pend = draft.get_state()
         draft.kv_truncate(lens - 1, pend)
         self.io = LoopIo(self.pool.data_ptr(), uniform_pool.shape[0], self.iteration.data_ptr(),

@@ -173,7 +173,7 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap, int n_p
   p.rope_cs = take(M * c.head_dim * 4);
   p.part = take(M * c.n_q_heads * (size_t)p.nsplit_max * (c.head_dim + 2) * 4);
   p.logits = take(M * V * 4);
-  p.row_stats = take(M * 4 * 4);
+  p.row_stats = take(M * 8 * 4);  // eight statistics words per row (sampler.cu)
   p.xn = take(M * d * 4);
   p.attn_out = take(M * qd * 4);
   p.act = take(M * F * 4);
@@ -446,6 +446,8 @@ int params_ok(const ssd_streams* s, const ssd_verify_params* p, bool need_gamma)
   if (!(p->temperature > 0.f) || !isfinite(p->temperature)) return SSD_ERR_BAD_PARAM;
   if (!(p->beta >= 0.f) || !isfinite(p->beta)) return SSD_ERR_BAD_PARAM;
   if (!(p->top_p >= 0.f) || !isfinite(p->top_p)) return SSD_ERR_BAD_PARAM;
+  if (p->ras_window < 0 || p->ras_window > 32 || (p->ras_window > 0 && (!p->dev_recent_tokens || !(p->ras_tau >= 0.f))))
+    return SSD_ERR_BAD_PARAM;
   return SSD_OK;
 }
 
@@ -1024,7 +1026,9 @@ int ssd_iteration(ssd_model* target, ssd_streams* ts, ssd_model* draft, ssd_stre
   if (rc != SSD_OK) return rc;
   launch_loop_finish(ds->len, ds->pending, ds->cap, io->dev_in_ids, io->dev_draft_tokens, gamma,
                      io->dev_accepted_len, io->dev_next_token, B, io->dev_out_tokens, io->out_capacity,
-                     io->dev_out_count, io->dev_accept_log, io->n_iterations, io->dev_iteration, ts->status, st);
+                     io->dev_out_count, io->dev_accept_log, io->n_iterations, io->dev_iteration,
+                     params->ras_window > 0 ? const_cast<int32_t*>(params->dev_recent_tokens) : nullptr,
+                     params->ras_window, ts->status, st);
   release_pages(ds, st);
   SSD_CUDA(cudaGetLastError());
   return SSD_OK;
@@ -1055,7 +1059,8 @@ int verify_impl(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_toke
   if (probs_ready) SSD_CUDA(cudaStreamWaitEvent(st, probs_ready, 0));
   SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
                                  dev_uniforms, s->B, gamma, 1.0f / params->temperature,
-                                 params->top_k, params->top_p, params->beta, s->row_stats, s->accept_flags,
+                                 params->top_k, params->top_p, params->beta, params->ras_window, params->ras_tau,
+                                 params->dev_recent_tokens, s->row_stats, s->accept_flags,
                                  s->counters, dev_accepted_len, dev_next_token, s->status, st));
   return SSD_OK;
 }

@@ -49,6 +49,7 @@ cudaError_t launch_attention_simt(int dtype, const float* qrot, const void* kv_l
 cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* draft_tokens,
                                   const float* draft_probs, const float* uniforms, int B,
                                   int gamma, float inv_temperature, int top_k, float top_p, float beta,
+                                  int ras_window, float ras_tau, const int32_t* recent_tokens,
                                   float* row_stats, int32_t* accept_flags, int32_t* counters,
                                   int32_t* accepted_len, int32_t* next_token, int32_t* status,
                                   cudaStream_t st);
@@ -67,7 +68,7 @@ void launch_loop_finish(int32_t* draft_len, int32_t* draft_pending, int cap, int
                         const int32_t* draft_tokens, int gamma, const int32_t* accepted_len,
                         const int32_t* next_token, int B, int32_t* out_tokens, int out_capacity,
                         int32_t* out_count, int32_t* accept_log, int n_rows, int32_t* iteration,
-                        int32_t* status, cudaStream_t st);
+                        int32_t* recent_tokens, int ras_window, int32_t* status, cudaStream_t st);
 void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_len,
                       const int32_t* next_token, int B, int cap, int max_gamma, int32_t* status,
                       cudaStream_t st);

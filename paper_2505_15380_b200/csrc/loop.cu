@@ -42,7 +42,7 @@ __global__ void loop_finish_kernel(int32_t* draft_len, int32_t* draft_pending, i
                                    const int32_t* __restrict__ accepted_len,
                                    const int32_t* __restrict__ next_token, int B, int32_t* out_tokens,
                                    int out_capacity, int32_t* out_count, int32_t* accept_log, int n_rows,
-                                   int32_t* iteration, int32_t* status) {
+                                   int32_t* iteration, int32_t* recent, int win, int32_t* status) {
   const int it = ((*iteration % n_rows) + n_rows) % n_rows;
   for (int b = threadIdx.x; b < B; b += blockDim.x) {  // launched as one block
     int k = accepted_len[b];
@@ -59,6 +59,14 @@ __global__ void loop_finish_kernel(int32_t* draft_len, int32_t* draft_pending, i
         ++n;
       }
       out_count[b] = n;
+      if (recent) {  // the window of the repetition-aware sampler: the last `win` tokens of T_in
+        const int e = k + 1;
+        for (int i = 0; i < win; ++i) {  // in place: entry i takes a value from at or beyond i
+          const int src = i + e;
+          recent[(size_t)b * win + i] = src < win ? recent[(size_t)b * win + src]
+                                                  : (src - win < k ? draft_tokens[b * gamma + src - win] : y);
+        }
+      }
       const int prev = k > 0 ? draft_tokens[b * gamma + k - 1] : in_ids[2 * b + 1];
       in_ids[2 * b] = prev;
       in_ids[2 * b + 1] = y;
@@ -74,11 +82,11 @@ void launch_loop_finish(int32_t* draft_len, int32_t* draft_pending, int cap, int
                         const int32_t* draft_tokens, int gamma, const int32_t* accepted_len,
                         const int32_t* next_token, int B, int32_t* out_tokens, int out_capacity,
                         int32_t* out_count, int32_t* accept_log, int n_rows, int32_t* iteration,
-                        int32_t* status, cudaStream_t st) {
+                        int32_t* recent_tokens, int ras_window, int32_t* status, cudaStream_t st) {
   // one block: every thread reads the iteration counter before the last thread advances it
   loop_finish_kernel<<<1, 1024, 0, st>>>(draft_len, draft_pending, cap, in_ids, draft_tokens, gamma, accepted_len,
                                          next_token, B, out_tokens, out_capacity, out_count, accept_log, n_rows,
-                                         iteration, status);
+                                         iteration, recent_tokens, ras_window, status);
   count_launch();
 }
 

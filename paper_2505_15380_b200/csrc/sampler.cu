@@ -65,7 +65,23 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
 // the additions, so the nucleus cut is the same in every run.
 __device__ __forceinline__ unsigned long long mass_fx(float x) { return __float2ull_rn(expf(x) * 4294967296.f); }
 
+// Repetition-aware sampling: a nucleus draw that repeats one of the last `win` tokens at least
+// win * tau times is thrown away and redrawn from the full softmax.  As one distribution:
+//   q(x) = q_nuc(x) [x not repeated] + R q_full(x),  R = mass of q_nuc on the repeated ids.
+constexpr int RAS_MAX_WIN = 32;
+constexpr int RS_STRIDE = 8;  // floats of row statistics per row: the four of RowStats, sum_full, R
+struct Ras {
+  int win;               // 0: off
+  float thresh;          // win * tau
+  const int32_t* recent; // [B, win]: last tokens of T_in, oldest first, pending token last, -1 = none
+};
+struct RasRow {
+  float sum_full;  // sum of exp(z - zmax) over all ids
+  float R;
+};
+
 struct SampSmem {
+  int rep_ids[RAS_MAX_WIN];  // repeated ids of this row's window (-1: none)
   unsigned long long hist_fx[256];
   unsigned long long red_u[SAMP_THREADS / 32];
   unsigned long long mass_above;
@@ -263,12 +279,71 @@ __device__ int block_inverse_cdf(const float* w, int V, float u, SampSmem& sm, d
   return y;
 }
 
+// The repeated ids of row r's window: the last `win` tokens of recent[b] ++ x_1..x_r (row r's
+// own token x_{r+1} is not part of it).  Block-collective; leaves them in sm.rep_ids.
+__device__ void ras_window(const Ras& ras, const int32_t* __restrict__ draft_tokens, int gamma, int b, int r, int V,
+                           SampSmem& sm) {
+  const int j = threadIdx.x;
+  if (j < RAS_MAX_WIN) {
+    int rep = -1;
+    if (j < ras.win) {
+      auto at = [&](int i) {  // i-th token of the window
+        const int c = r + i;
+        return c < ras.win ? ras.recent[(size_t)b * ras.win + c] : draft_tokens[b * gamma + c - ras.win];
+      };
+      const int t = at(j);
+      if (t >= 0 && t < V) {
+        int cnt = 0;
+        bool first = true;
+        for (int i = 0; i < ras.win; ++i) {
+          const bool same = at(i) == t;
+          cnt += same;
+          if (same && i < j) first = false;
+        }
+        if (first && (float)cnt >= ras.thresh) rep = t;
+      }
+    }
+    sm.rep_ids[j] = rep;
+  }
+  __syncthreads();
+}
+__device__ __forceinline__ bool ras_is_rep(const SampSmem& sm, int win, int t) {
+  bool rep = false;
+  for (int j = 0; j < win; ++j) rep |= sm.rep_ids[j] == t;
+  return rep;
+}
+// sum_full and R of a row whose nucleus statistics are `st`.  Block-collective.
+__device__ RasRow ras_row(const float* z, int V, const RowStats& st, int win, SampSmem& sm) {
+  double s = 0.0;
+  for (int t = threadIdx.x; t < V; t += SAMP_THREADS) s += (double)expf(z[t] - st.zmax);
+  RasRow rr;
+  rr.sum_full = (float)block_sum_d(s, sm.red_d);
+  float R = 0.f;
+  for (int j = 0; j < win; ++j) {  // fixed order
+    const int t = sm.rep_ids[j];
+    if (t >= 0 && is_kept(z[t], t, st)) R += expf(z[t] - st.zmax) / st.sum;
+  }
+  rr.R = R;
+  return rr;
+}
+// q(t) of the target's sampler: the (top-k, top-p) softmax, or the repetition-aware mixture.
+__device__ __forceinline__ float q_value(float zz, int t, const RowStats& st, int win, const RasRow& rr,
+                                         const SampSmem& sm) {
+  const float e = expf(zz - st.zmax);
+  float q = is_kept(zz, t, st) ? e / st.sum : 0.f;
+  if (win > 0) {
+    if (q > 0.f && ras_is_rep(sm, win, t)) q = 0.f;
+    q += rr.R * (e / rr.sum_full);
+  }
+  return q;
+}
+
 // Grid (R, B), R = gamma + 1.
 __global__ void __launch_bounds__(SAMP_THREADS)
 verify_sampler_kernel(const float* __restrict__ logits, int V,
                       const int32_t* __restrict__ draft_tokens,
                       const float* __restrict__ draft_probs, const float* __restrict__ uniforms,
-                      int gamma, float inv_t, int top_k, float top_p, float beta, float* row_stats,
+                      int gamma, float inv_t, int top_k, float top_p, float beta, Ras ras, float* row_stats,
                       int32_t* accept_flags, int32_t* counters, int32_t* __restrict__ accepted_len,
                       int32_t* __restrict__ next_token, int32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -288,6 +363,11 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
   __syncthreads();
   if (sm.bad && threadIdx.x == 0) atomicOr(status, SSD_STATUS_NONFINITE);
   RowStats st = compute_row_stats(z, V, top_k, top_p, sm);
+  RasRow rr{1.f, 0.f};
+  if (ras.win > 0) {
+    ras_window(ras, draft_tokens, gamma, b, r, V, sm);
+    rr = ras_row(z, V, st, ras.win, sm);
+  }
   if (threadIdx.x == 0) {
     int flag = 0;
     if (r < gamma) {  // Eq. 5: accept x_i iff r_i < min(1, q_i(x_i) / p_i(x_i)) + beta
@@ -298,7 +378,7 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
         atomicOr(status, SSD_STATUS_BAD_TOKEN);
         valid = false;
       } else {
-        if (is_kept(z[x], x, st)) qx = expf(z[x] - st.zmax) / st.sum;
+        qx = q_value(z[x], x, st, ras.win, rr, sm);
         px = draft_probs[((size_t)b * gamma + r) * V + x];
         if (!(px >= 0.f) || !isfinite(px)) {
           atomicOr(status, SSD_STATUS_BAD_PROB);
@@ -308,11 +388,13 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
       float ratio = px <= qx ? 1.f : qx / px;
       flag = valid && uniforms[((size_t)b * R + r) * 2] < ratio + beta;
     }
-    float* rs = row_stats + ((size_t)b * R + r) * 4;
+    float* rs = row_stats + ((size_t)b * R + r) * RS_STRIDE;
     rs[0] = st.zmax;
     rs[1] = st.sum;
     rs[2] = __uint_as_float(st.thr_key);
     rs[3] = __int_as_float(st.tie_id_max);
+    rs[4] = rr.sum_full;
+    rs[5] = rr.R;
     accept_flags[b * R + r] = flag;
     __threadfence();
     int prev = atomicAdd(&counters[b], 1);
@@ -331,18 +413,20 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
   }
   __syncthreads();
   const int k = sm.k_acc;
-  const float* rs = row_stats + ((size_t)b * R + k) * 4;
+  const float* rs = row_stats + ((size_t)b * R + k) * RS_STRIDE;
   RowStats sk;
   sk.zmax = __ldcg(rs + 0);
   sk.sum = __ldcg(rs + 1);
   sk.thr_key = __float_as_uint(__ldcg(rs + 2));
   sk.tie_id_max = __float_as_int(__ldcg(rs + 3));
+  const RasRow rk{__ldcg(rs + 4), __ldcg(rs + 5)};
+  if (ras.win > 0) ras_window(ras, draft_tokens, gamma, b, k, V, sm);  // row k's repeated ids
   const float* krow = logits + ((size_t)b * R + k) * V;
   const float* prow = k < gamma ? draft_probs + ((size_t)b * gamma + k) * V : nullptr;
   // Eq. 6: w = max(0, q_k - p_k) on a rejection; the bonus row q_{gamma+1} otherwise
   for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
     float zz = krow[t] * inv_t;
-    float q = is_kept(zz, t, sk) ? expf(zz - sk.zmax) / sk.sum : 0.f;
+    float q = q_value(zz, t, sk, ras.win, rk, sm);
     z[t] = prow ? fmaxf(0.f, q - prow[t]) : q;
   }
   __syncthreads();
@@ -352,7 +436,7 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
   if (y < 0) {  // residual has no mass (numerical corner): draw from q_k itself
     for (int t = threadIdx.x; t < V; t += SAMP_THREADS) {
       float zz = krow[t] * inv_t;
-      z[t] = is_kept(zz, t, sk) ? expf(zz - sk.zmax) / sk.sum : 0.f;
+      z[t] = q_value(zz, t, sk, ras.win, rk, sm);
     }
     __syncthreads();
     y = block_inverse_cdf(z, V, u, sm, &total);
@@ -367,9 +451,15 @@ verify_sampler_kernel(const float* __restrict__ logits, int V,
 cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* draft_tokens,
                                   const float* draft_probs, const float* uniforms, int B,
                                   int gamma, float inv_temperature, int top_k, float top_p, float beta,
+                                  int ras_window, float ras_tau, const int32_t* recent_tokens,
                                   float* row_stats, int32_t* accept_flags, int32_t* counters,
                                   int32_t* accepted_len, int32_t* next_token, int32_t* status,
                                   cudaStream_t st) {
+  Ras ras{0, 0.f, nullptr};
+  if (ras_window > 0) {
+    if (ras_window > RAS_MAX_WIN || !recent_tokens) return cudaErrorInvalidValue;
+    ras = Ras{ras_window, (float)ras_window * ras_tau, recent_tokens};
+  }
   size_t smem = sizeof(SampSmem) + (size_t)V * sizeof(float);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   if (smem > 48 * 1024) {
@@ -379,7 +469,7 @@ cudaError_t launch_verify_sampler(const float* logits, int V, const int32_t* dra
   }
   dim3 grid(gamma + 1, B);
   verify_sampler_kernel<<<grid, SAMP_THREADS, smem, st>>>(
-      logits, V, draft_tokens, draft_probs, uniforms, gamma, inv_temperature, top_k, top_p, beta,
+      logits, V, draft_tokens, draft_probs, uniforms, gamma, inv_temperature, top_k, top_p, beta, ras,
       row_stats, accept_flags, counters, accepted_len, next_token, status);
   count_launch();
   return cudaGetLastError();
@@ -480,7 +570,7 @@ void launch_kv_commit(int32_t* len, int32_t* pending, const int32_t* accepted_le
 // whose memory pool is fixed at start-up, or a plug-in that is handed device pointers by its host
 // process and owns none.  ssd_verify needs a workspace such callers cannot provide.  This entry
 // point runs the same fused acceptance kernel on logits the caller already has, and keeps the
-// kernel's scratch (four statistics words and one flag per row, one counter per stream, one status
+// kernel's scratch (eight statistics words and one flag per row, one counter per stream, one status
 // word) in the fixed device array below instead.
 namespace {
 
@@ -488,13 +578,13 @@ constexpr int NOALLOC_MAX_STREAMS = 256;  // streams per call
 constexpr int NOALLOC_MAX_ROWS = ssd::R_MAX;  // gamma + 1 <= 16
 
 struct NoAllocScratch {
-  float row_stats[NOALLOC_MAX_STREAMS * NOALLOC_MAX_ROWS * 4];
+  float row_stats[NOALLOC_MAX_STREAMS * NOALLOC_MAX_ROWS * ssd::RS_STRIDE];
   int32_t accept_flags[NOALLOC_MAX_STREAMS * NOALLOC_MAX_ROWS];
   int32_t counters[NOALLOC_MAX_STREAMS];
   int32_t status;
 };
 
-// About 84 KB, resident on every GPU that loads the library until the process exits.  In host
+// About 148 KB, resident on every GPU that loads the library until the process exits.  In host
 // code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
@@ -544,7 +634,8 @@ extern "C" int ssd_accept_noalloc(const float* dev_logits, const int32_t* dev_dr
   if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: cudaMemsetAsync");
   e = ssd::launch_verify_sampler(dev_logits, vocab, dev_draft_tokens, dev_draft_probs, dev_uniforms,
                                  batch, params->gamma, 1.0f / params->temperature, params->top_k,
-                                 params->top_p, params->beta, sc->row_stats, sc->accept_flags, sc->counters,
+                                 params->top_p, params->beta, params->ras_window, params->ras_tau,
+                                 params->dev_recent_tokens, sc->row_stats, sc->accept_flags, sc->counters,
                                  dev_accepted_len, dev_next_token, &sc->status, st);
   if (e != cudaSuccess) return ssd::report_cuda_error(e, "ssd_accept_noalloc: launch");
   return SSD_OK;

@@ -109,7 +109,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
              uniform_seed: int = 0, commit_and_repeat: bool = False,
              capacity: Optional[int] = None, path: int = 0, split: bool = True,
              max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34, top_p: float = 0.0,
-             paged: Optional[tuple] = None) -> CaseResult:
+             paged: Optional[tuple] = None, ras: Optional[tuple] = None) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -146,6 +146,14 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
     for b in which:
         assert lens_g[b] == ostreams[b].length and pend_g[b] == ostreams[b].pending
 
+    # repetition-aware sampling (window, tau): the last `window` tokens of each T_in, pending last
+    win, tau = ras if ras else (0, 0.0)
+    recent = np.full((B, max(win, 1)), -1, dtype=np.int32)
+    for b in range(B):
+        tail = prefixes[b][-win:] if win else prefixes[b][:0]
+        if win:
+            recent[b, win - len(tail):] = tail
+    n_ras_active = 0
     n_steps = 2 if commit_and_repeat else 1
     res = CaseResult(0.0, 0, 0, 0, [])
     dev = gmodel.device
@@ -171,7 +179,9 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
                 draft[b, i] = tok
             st.length = base_len
         # ---- GPU
-        params = binding.VerifyParams(gamma, wl.temperature, wl.top_k, beta, top_p)
+        d_recent = torch.from_numpy(recent).to(dev)
+        params = binding.VerifyParams(gamma, wl.temperature, wl.top_k, beta, top_p, win, tau,
+                                      d_recent.data_ptr() if win else None)
         d_tok = torch.from_numpy(draft.astype(np.int32)).to(dev)
         d_p = torch.from_numpy(p_rows.astype(np.float32)).to(dev)
         d_u = torch.from_numpy(uni).to(dev)
@@ -192,13 +202,20 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
         for b in which:
             st = ostreams[b]
             o = orc.verify(omodel, st, draft[b], p_rows[b], uni[b], temperature=wl.temperature,
-                           top_k=wl.top_k, beta=beta, top_p=top_p)
+                           top_k=wl.top_k, beta=beta, top_p=top_p, recent=recent[b], win_size=win, tau_r=tau)
             err = float(np.abs(o["logits"] - g_logits[b]).max())
             res.max_logit_err = max(res.max_logit_err, err)
             assert err <= logit_tol, f"stream {b}: logits differ by {err}"
             # strict: oracle arithmetic on the GPU's logits
             gl = g_logits[b].astype(np.float64)
-            q_g = np.stack([orc.transform(r, wl.temperature, wl.top_k, top_p) for r in gl])
+            if win:
+                hist = np.concatenate([recent[b].astype(np.int64), draft[b].astype(np.int64)])
+                q_g = np.stack([orc.transform_ras(r, wl.temperature, wl.top_k, top_p, hist[:win + i], win, tau)
+                                for i, r in enumerate(gl)])
+                n_ras_active += int(any(not np.allclose(q_g[i], orc.transform(gl[i], wl.temperature, wl.top_k, top_p))
+                                        for i in range(R)))
+            else:
+                q_g = np.stack([orc.transform(r, wl.temperature, wl.top_k, top_p) for r in gl])
             o2 = orc.accept_step(q_g, p_rows[b], draft[b], uni[b], beta)
             res.n_streams += 1
             res.ks.append(int(g_k[b]))
@@ -246,6 +263,9 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
             res.n_e2e_excluded += int(e2e_excl)
             if commit_and_repeat:
                 orc.commit(st, int(g_k[b]), int(g_y[b]))      # follow the GPU's trajectory
+                if win:
+                    emitted = np.concatenate([draft[b][:int(g_k[b])], [int(g_y[b])]]).astype(np.int32)
+                    recent[b] = np.concatenate([recent[b], emitted])[-win:]
         if commit_and_repeat:
             gs.kv_commit(d_k, d_y)
             torch.cuda.synchronize()
@@ -255,4 +275,6 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
     print(f"[{wl.name}] streams-steps {res.n_streams}, strict excluded {res.n_strict_excluded}, "
           f"e2e excluded {res.n_e2e_excluded}, max|dlogit| {res.max_logit_err:.2e}, k {res.ks}")
     check_exclusions(res, max_strict_frac, max_e2e_frac)
+    if win:
+        assert n_ras_active >= 1, "no row had a repeated id in its window: the case does not test the mixture"
     return res

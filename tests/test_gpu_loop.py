@@ -32,7 +32,7 @@ def _pool(seed, n_iter, B, gamma):
                     ).astype(np.float32)
 
 
-def _setup(tshape, dshape, lens, gamma, seed, n_iter, out_cap=256):
+def _setup(tshape, dshape, lens, gamma, seed, n_iter, out_cap=256, ras_window=0):
     from paper_2505_15380_b200 import binding
     B = len(lens)
     wl = synth.Workload("loop", tshape, dshape, B, gamma, 1.0, 0, tuple(lens), 2, seed, seed + 1)
@@ -45,14 +45,16 @@ def _setup(tshape, dshape, lens, gamma, seed, n_iter, out_cap=256):
     ts.prefill(prefixes)
     ds.prefill(prefixes)
     pool = _pool(seed + 3, n_iter, B, gamma)
-    loop = binding.Loop(ts, ds, prefixes, gamma, pool, out_cap)
+    loop = binding.Loop(ts, ds, prefixes, gamma, pool, out_cap, ras_window=ras_window)
     return tm, dm, ts, ds, prefixes, pool, loop, tw, dw, cap
 
 
 def _run_against_oracle(tshape, dshape, lens, gamma, temperature, top_k, beta, n_iter, p_tol, draw_eps,
-                        seed=5):
+                        seed=5, ras=None):
     from paper_2505_15380_b200 import binding
-    tm, dm, ts, ds, prefixes, pool, loop, tw, dw, cap = _setup(tshape, dshape, lens, gamma, seed, n_iter)
+    win, tau = ras if ras else (0, 0.0)
+    tm, dm, ts, ds, prefixes, pool, loop, tw, dw, cap = _setup(tshape, dshape, lens, gamma, seed, n_iter,
+                                                               ras_window=win)
     B, V = len(lens), tshape.vocab_out
     otm, odm = oracle_model(tshape, tw), oracle_model(dshape, dw)
     ot, od, in_ids = [], [], []
@@ -64,7 +66,9 @@ def _run_against_oracle(tshape, dshape, lens, gamma, temperature, top_k, beta, n
         ot.append(st)
         od.append(sd)
         in_ids.append([int(prefixes[b][-2]), int(prefixes[b][-1])])
-    par = binding.VerifyParams(gamma, temperature, top_k, beta)
+    par = binding.VerifyParams(gamma, temperature, top_k, beta, 0.0, win, tau,
+                               loop.recent.data_ptr() if win else None)
+    recent = loop.recent.cpu().numpy().copy() if win else None
     emitted = [[] for _ in range(B)]
     n_dec = n_excl = 0
     seen_k = set()
@@ -108,7 +112,8 @@ def _run_against_oracle(tshape, dshape, lens, gamma, temperature, top_k, beta, n
                 ids = np.array([g_x[b, i]])               # follow the GPU
             # ---- verify and accept (Eq. 4-6) with the GPU's draft as input on both sides
             uni = u[gamma:].reshape(gamma + 1, 2)
-            o = orc.verify(otm, st, g_x[b], g_p[b], uni, temperature=temperature, top_k=top_k, beta=beta)
+            o = orc.verify(otm, st, g_x[b], g_p[b], uni, temperature=temperature, top_k=top_k, beta=beta,
+                           recent=recent[b] if win else None, win_size=win, tau_r=tau)
             near = any(abs(a - float(uni[i, 0])) < WINDOW for i, a in enumerate(o["thresholds"]))
             if not near:
                 assert g_k[b] == o["k"], f"iteration {it} stream {b}: accepted length"
@@ -134,9 +139,13 @@ def _run_against_oracle(tshape, dshape, lens, gamma, temperature, top_k, beta, n
             sd.pending = y
             in_ids[b] = [prev, y]
             emitted[b] += [int(t) for t in g_x[b, :k]] + [y]
+            if win:
+                recent[b] = np.concatenate([recent[b], np.array(emitted[b][-(k + 1):], np.int32)])[-win:]
             assert tl[b] == st.length and tp[b] == st.pending
             assert dl[b] == sd.length and dp[b] == y
             assert tl[b] == dl[b] + 1                    # the draft stays one token behind
+    if win:
+        assert np.array_equal(loop.recent.cpu().numpy(), recent)     # the device kept the window up to date
     out = loop.out_tokens.cpu().numpy()
     cnt = loop.out_count.cpu().numpy()
     assert np.array_equal(loop.in_ids.cpu().numpy(), np.array(in_ids))
@@ -167,6 +176,14 @@ def test_loop_bf16_models_top_k():
     t = synth.ModelShape(3, 256, 8, 2, 64, 512, 700, 16, 1e6)
     d = synth.ModelShape(1, 128, 4, 2, 32, 256, 700, 16, 1e6)
     _run_against_oracle(t, d, [40, 65, 17], 4, 0.8, 25, 0.4, 20, p_tol=2e-4, draw_eps=1e-3)
+
+
+def test_loop_with_repetition_aware_target_sampling():
+    """The window of recent tokens is kept on the device across iterations (60-id vocabulary, so
+    repeats do occur)."""
+    t = synth.ModelShape(2, 128, 4, 2, 64, 256, 60, 16, 1e6)
+    d = synth.ModelShape(1, 128, 4, 2, 32, 256, 60, 16, 1e6)
+    _run_against_oracle(t, d, [40, 21], 3, 0.9, 20, 0.4, 15, p_tol=2e-4, draw_eps=1e-3, ras=(8, 0.25))
 
 
 def test_loop_batched_streams_take_the_tensor_core_path():

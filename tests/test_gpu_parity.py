@@ -82,6 +82,17 @@ def test_nucleus_sampling_in_the_fused_kernel(top_p, top_k, temperature):
           sigma=1.0, top_p=top_p)
 
 
+@pytest.mark.parametrize("win,tau,top_p,top_k", [(10, 0.1, 0.8, 25), (4, 0.5, 0.0, 0), (16, 0.125, 0.9, 0)])
+def test_repetition_aware_sampling_in_the_fused_kernel(win, tau, top_p, top_k):
+    """The target samples repetition-aware: q_i in Eq. 5-6 is the mixture of the nucleus row and the
+    full row weighted by the nucleus mass of the ids repeated in row i's window (recent tokens of
+    T_in followed by x_1..x_{i-1}); the window moves on with the committed tokens."""
+    shape = _small(synth.BF16, 64, v=60)        # small vocabulary: windows do hit the kept ids
+    wl = _wl(shape, 6, 5, [50, 64, 100, 17, 33, 80], temperature=0.9, top_k=top_k)
+    _case(wl, beta=0.0, sigma=0.5, top_p=top_p, ras=(win, tau), commit_and_repeat=True)
+    _case(wl, beta=0.4, sigma=1.5, top_p=top_p, ras=(win, tau))
+
+
 def test_accepted_length_never_shrinks_with_beta():
     """Table 3's mechanism on the GPU: with the inputs and uniforms held fixed, a larger
     tolerance beta accepts at least as many draft tokens, and beta >= 1 accepts all of them."""
