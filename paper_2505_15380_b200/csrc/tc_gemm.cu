@@ -31,6 +31,8 @@ constexpr int TC_MAX_STAGES = 12;
 // eight lanes issuing 8 KB pieces 46-90 GB/s.
 constexpr int TC_ISSUERS = 8;
 constexpr uint32_t TC_PIECE = 8192;
+// SwiGLU epilogue staging: 32 token rows of 16 bytes per (column half, part), padded against bank conflicts
+constexpr uint32_t TC_STG_STRIDE = 528;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -126,6 +128,7 @@ struct TcKernelParams {
   int n_rows, KS, M, Mpad, ld_part;  // KS = k-steps of the whole projection; ld_part = tiles * 128
   int sk, stages;                    // k-steps per stage, pipeline depth
   int wide;                          // 1: one instruction multiplies both parts (N over 2 * Mpad rows)
+  int dual;                          // wide, and even / odd k-steps accumulate into two column sets
   int nchunks, chunk_n;              // row ranges of the activation operand per MMA (<= 256 each)
   int tmem_cols;
   int epi;
@@ -153,6 +156,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
   TcShared& S = *reinterpret_cast<TcShared*>(smem_a + (size_t)P.stages * stage_a);
   const int ks0 = (int)(((long long)split * P.KS) / nsplit), ks1 = (int)(((long long)(split + 1) * P.KS) / nsplit);
   const int n_iter = (ks1 - ks0 + P.sk - 1) / P.sk;
+  const bool dual = P.dual && ks1 - ks0 >= 2;  // the second column set needs a k-step of its own
 
   if (tid == 0) {
     for (int s = 0; s < P.stages; ++s) {
@@ -242,7 +246,14 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         for (int j = 0; j < nks; ++j) {
           const uint64_t da = umma_desc(wb + (uint32_t)j * TC_WBLOCK, 2048u, 128u);
           const uint32_t blk = ab + (uint32_t)j * act_block, lead = (uint32_t)P.Mpad * 32u;
-          if (P.wide) {
+          if (dual) {
+            // Back-to-back instructions into the same accumulator columns wait for one another
+            // (~280 cycles each, measured, against ~165 when they alternate between column
+            // ranges): even k-steps add into columns [0, 2 Mpad), odd ones into [2 Mpad, 4 Mpad).
+            const int kk = it * P.sk + j;
+            umma_bf16(tmem + (uint32_t)((kk & 1) * 2 * P.Mpad), da, umma_desc(blk, lead, 128u), umma_idesc(2 * P.Mpad),
+                      kk >= 2 ? 1u : 0u);
+          } else if (P.wide) {
             // the operand's 2 * Mpad rows (leading parts, then remainders) in ranges of <= 256:
             // accumulator columns [0, Mpad) receive W x_hi, [Mpad, 2 Mpad) receive W x_lo
             for (int c = 0; c < P.nchunks; ++c) {
@@ -280,6 +291,14 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
           tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(P.Mpad + c0), w);
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(w[i]));
+          if (dual) {  // and the odd k-steps' column set, in a fixed order
+            uint32_t x[32];
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(2 * P.Mpad + c0), x);
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(3 * P.Mpad + c0), w);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              v[i] = __float_as_uint(__uint_as_float(v[i]) + (__uint_as_float(x[i]) + __uint_as_float(w[i])));
+          }
         }
         if (P.epi == TC_EPI_PARTIAL) {
           float* dst = P.part + ((size_t)split * P.Mpad + c0) * P.ld_part + n;
@@ -292,23 +311,37 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             for (int i = 0; i < 32; ++i)
               if (c0 + i < P.M) P.out[(size_t)(c0 + i) * P.ldo + n] = __uint_as_float(v[i]);
           }
-        } else {  // TC_EPI_SWIGLU: even lanes hold gate_j, odd lanes up_j, j = n / 2
-          const int j = n >> 1;
-          uint8_t* dst = P.act_out + (size_t)(j >> 4) * ((size_t)P.Mpad * 64) + (size_t)((j >> 3) & 1) * ((size_t)P.Mpad * 32) +
-                         (size_t)(j & 7) * 2;
+        } else {
+          // TC_EPI_SWIGLU: even lanes hold gate_j, odd lanes up_j, j = n / 2.  The warp's 16 columns j
+          // are one k-step block of the output operand.  The two lanes of a pair share the work
+          // (even lane: even tokens of the range, odd lane: odd tokens); the bf16 parts go through
+          // a small staging area in shared memory (the pipeline stages are idle by now) so that
+          // global memory sees whole 16-byte rows, 512 contiguous bytes per warp store, instead
+          // of two-byte pieces (measured: the epilogue of a 448-row tile 41 -> 6 us).
+          const int j0 = (tile * TC_TILE_ROWS + q * 32) >> 1, jl = lane >> 1, odd = lane & 1;
+          uint8_t* stg = smem + (size_t)(warp - 2) * (4 * TC_STG_STRIDE);
+          const uint32_t my = (uint32_t)((jl >> 3) * 2) * TC_STG_STRIDE + (uint32_t)(jl & 7) * 2u;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float mine = __uint_as_float(v[i]);
-            const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-            if ((lane & 1) == 0 && n < P.n_rows && c0 + i < P.M) {
-              const float x = __fdividef(mine, 1.f + __expf(-mine)) * other;
-              const bf16 hi = __float2bfloat16_rn(x);
-              const bf16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
-              uint8_t* e = dst + (size_t)(c0 + i) * 16;
-              *reinterpret_cast<bf16*>(e) = hi;
-              *reinterpret_cast<bf16*>(e + (size_t)P.Mpad * 16) = lo;
-            }
+          for (int i = 0; i < 32; i += 2) {
+            const float a = __uint_as_float(v[i]), b = __uint_as_float(v[i + 1]);
+            const float got = __shfl_xor_sync(0xffffffffu, odd ? a : b, 1);
+            const float gate = odd ? got : a, up = odd ? b : got;
+            const float x = __fdividef(gate, 1.f + __expf(-gate)) * up;
+            const bf16 hi = __float2bfloat16_rn(x);
+            const bf16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+            uint8_t* e = stg + my + (uint32_t)(i + odd) * 16u;
+            *reinterpret_cast<bf16*>(e) = hi;
+            *reinterpret_cast<bf16*>(e + TC_STG_STRIDE) = lo;
           }
+          __syncwarp();
+          if (j0 < ((P.n_rows / 2 + 15) & ~15) && c0 + lane < P.M) {
+            uint8_t* blk = P.act_out + (size_t)(j0 >> 4) * ((size_t)P.Mpad * 64) + (size_t)(c0 + lane) * 16;
+#pragma unroll
+            for (int hp = 0; hp < 4; ++hp)  // hp = half * 2 + part
+              *reinterpret_cast<uint4*>(blk + (size_t)hp * ((size_t)P.Mpad * 16)) =
+                  *reinterpret_cast<const uint4*>(stg + (uint32_t)hp * TC_STG_STRIDE + (uint32_t)lane * 16u);
+          }
+          __syncwarp();
         }
       }
     }
@@ -415,8 +448,9 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   const int op_rows = p.wide ? 2 * p.Mpad : p.Mpad;
   p.nchunks = (op_rows + 255) / 256;
   p.chunk_n = tc_round16((op_rows + p.nchunks - 1) / p.nchunks);
+  p.dual = p.wide && 4 * p.Mpad <= 512 && !two_per_sm;  // two CTAs on an SM have 256 columns each
   p.tmem_cols = 32;
-  while (p.tmem_cols < op_rows) p.tmem_cols <<= 1;
+  while (p.tmem_cols < (p.dual ? 2 : 1) * op_rows) p.tmem_cols <<= 1;
   const size_t smem = (size_t)p.stages * p.sk * per_ks + sizeof(TcShared) + 64;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
