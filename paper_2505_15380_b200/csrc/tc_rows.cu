@@ -23,29 +23,35 @@ __device__ __forceinline__ void store_pair(uint8_t* apack, int Mpad, int t, int 
 }
 
 // Sum over the K slices of a projection's partial sums for two adjacent columns, in slice order
-// (bit-reproducible); the loads of eight slices are in flight together.
+// (bit-reproducible).  The loads of up to 24 slices are in flight together: the kernels that call
+// this are one dependent round trip to L2 after another, so every slice waited for separately is
+// a microsecond (measured: rounds of eight cost 1.5 us more on 21 slices).  With many rows the
+// kernels are built with eight in flight instead, which keeps them at four CTAs per SM: 448 rows
+// then still run as one wave.
+template <int NF>
 __device__ __forceinline__ float2 sum_slices(float2 v, const float* __restrict__ p, size_t slice_stride, int nsplit) {
-  int s = 0;
-  for (; s + 8 <= nsplit; s += 8) {
-    float2 t[8];
+  for (int s = 0; s < nsplit; s += NF) {
+    float2 t[NF];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) t[i] = __ldcg(reinterpret_cast<const float2*>(p + (size_t)(s + i) * slice_stride));
+    for (int i = 0; i < NF; ++i)
+      t[i] = s + i < nsplit ? __ldcg(reinterpret_cast<const float2*>(p + (size_t)(s + i) * slice_stride))
+                            : make_float2(0.f, 0.f);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      v.x += t[i].x;
-      v.y += t[i].y;
+    for (int i = 0; i < NF; ++i) {
+      if (s + i < nsplit) {
+        v.x += t[i].x;
+        v.y += t[i].y;
+      }
     }
-  }
-  for (; s < nsplit; ++s) {
-    const float2 t = __ldcg(reinterpret_cast<const float2*>(p + (size_t)s * slice_stride));
-    v.x += t.x;
-    v.y += t.y;
   }
   return v;
 }
 
+constexpr int TC_ROWS_DEEP = 256;  // up to this many rows (CTAs) the deep variant still is one wave
+
 // One CTA per row.  h[m, :] += sum_s part[s][m][:]; out = h / rms(h) * gain, packed.
-__global__ void __launch_bounds__(256)
+template <int NF, int MINB>
+__global__ void __launch_bounds__(256, MINB)
 tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
                     int d, const bf16* __restrict__ gain, float eps, uint8_t* __restrict__ apack) {
   extern __shared__ float row[];
@@ -57,7 +63,7 @@ tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int n
   for (int j = tid * 2; j < d; j += 512) {
     float2 v = *reinterpret_cast<const float2*>(h + (size_t)m * d + j);
     if (nsplit > 0) {
-      v = sum_slices(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
+      v = sum_slices<NF>(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
       *reinterpret_cast<float2*>(h + (size_t)m * d + j) = v;
     }
     row[j] = v.x;
@@ -86,7 +92,8 @@ __global__ void tc_pack_rows_kernel(const float* __restrict__ x, int K, int Mpad
 // One CTA per row: q/k/v = sum of the K slices + bias; rotate q and k by the row's position
 // (rotate-half pairs (j, j + hd/2)); q scaled by 1/sqrt(hd) to qrot; K (rotated) and V to the
 // cache at slot len + r.
-__global__ void __launch_bounds__(256)
+template <int NF, int MINB>
+__global__ void __launch_bounds__(256, MINB)
 tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
                    const bf16* __restrict__ bias, const float* __restrict__ cs, float* __restrict__ qrot,
                    bf16* __restrict__ kv_layer, const int32_t* __restrict__ len, RowMap rm, int cap, int Hq,
@@ -100,7 +107,7 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
   const int pos = len[b] + r, half = hd >> 1, nq = (Hq + 2 * Hkv) * hd;
   for (int j = tid * 2; j < nq; j += 512) {
     float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bias + j));
-    v = sum_slices(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
+    v = sum_slices<NF>(v, part + (size_t)m * ld_part + j, (size_t)Mpad * ld_part, nsplit);
     row[j] = v.x;
     row[j + 1] = v.y;
   }
@@ -147,8 +154,12 @@ tc_qkv_post_kernel(const float* __restrict__ part, int nsplit, int ld_part, int 
 
 void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, int M, int d,
                          const bf16* gain, float eps, uint8_t* apack, cudaStream_t st) {
-  tc_launch_pdl(tc_norm_pack_kernel, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0, ld_part,
-                tc_round16(M), d, gain, eps, apack);
+  if (M <= TC_ROWS_DEEP)
+    tc_launch_pdl(tc_norm_pack_kernel<24, 1>, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0,
+                  ld_part, tc_round16(M), d, gain, eps, apack);
+  else
+    tc_launch_pdl(tc_norm_pack_kernel<8, 4>, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0,
+                  ld_part, tc_round16(M), d, gain, eps, apack);
   count_launch();
 }
 
@@ -163,8 +174,12 @@ void launch_tc_qkv_post(const float* part, int nsplit, int ld_part, int Mpad, co
                         int32_t* status, cudaStream_t st) {
   const int M = rm.nb * rm.R;
   const size_t smem = (size_t)(Hq + 2 * Hkv) * hd * 4;
-  tc_launch_pdl(tc_qkv_post_kernel, dim3(M), dim3(256), smem, st, part, nsplit, ld_part, Mpad, bias, cs, qrot,
-                kv_layer, len, rm, cap, Hq, Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
+  if (M <= TC_ROWS_DEEP)
+    tc_launch_pdl(tc_qkv_post_kernel<24, 1>, dim3(M), dim3(256), smem, st, part, nsplit, ld_part, Mpad, bias, cs, qrot,
+                  kv_layer, len, rm, cap, Hq, Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
+  else
+    tc_launch_pdl(tc_qkv_post_kernel<8, 4>, dim3(M), dim3(256), smem, st, part, nsplit, ld_part, Mpad, bias, cs, qrot,
+                  kv_layer, len, rm, cap, Hq, Hkv, hd, 1.0f / sqrtf((float)hd), page_table, max_pages, status);
   count_launch();
 }
 
