@@ -149,13 +149,12 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
   const int n_tiles = (k_end - k_begin + TA_TILE - 1) / TA_TILE;
   for (int it = 0; it < n_tiles; ++it) {
     const int key0 = k_begin + it * TA_TILE;
-    if (it + 1 < n_tiles) {
-      stage_tile((it + 1) & 1, key0 + TA_TILE);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
+    // One barrier per tile: it makes this tile's copies (all threads') visible, and it says that
+    // every warp is done with the previous tile, whose buffer the next tile's copies may now
+    // overwrite while this one is being used.
+    cp_async_wait<0>();
     __syncthreads();
+    if (it + 1 < n_tiles) stage_tile((it + 1) & 1, key0 + TA_TILE);
     if (warp_active) {
       const uint8_t* ks = kv_s + (size_t)(it & 1) * 2 * TILE_BYTES;
       const uint32_t k_addr = smem_u32(ks) + ((lane >> 4) * 8 + (lane & 7)) * ROWB + ((lane >> 3) & 1) * 16;
@@ -172,9 +171,9 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
         for (int nt = 0; nt < TA_TILE / 8; nt += 2) {
           uint32_t b0, b1, b2, b3;
           ldmatrix_x4(k_addr + nt * 8 * ROWB + s * 32, b0, b1, b2, b3);
-          mma_bf16(sc[nt], ahi, b0, b1);
-          mma_bf16(sc[nt], alo, b0, b1);
+          mma_bf16(sc[nt], ahi, b0, b1);  // alternate the accumulators: no instruction waits for the one before
           mma_bf16(sc[nt + 1], ahi, b2, b3);
+          mma_bf16(sc[nt], alo, b0, b1);
           mma_bf16(sc[nt + 1], alo, b2, b3);
         }
       }
@@ -230,13 +229,12 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
           uint32_t b0, b1, b2, b3;
           ldmatrix_x4_trans(v_addr + kk * 16 * ROWB + dt * 16, b0, b1, b2, b3);
           mma_bf16(o[dt], phi, b0, b1);
-          if (TA_SPLIT_P) mma_bf16(o[dt], plo, b0, b1);
           mma_bf16(o[dt + 1], phi, b2, b3);
+          if (TA_SPLIT_P) mma_bf16(o[dt], plo, b0, b1);
           if (TA_SPLIT_P) mma_bf16(o[dt + 1], plo, b2, b3);
         }
       }
     }
-    __syncthreads();  // the tile's buffer is refilled two iterations on
   }
   if (!warp_active) return;
 #pragma unroll
