@@ -177,15 +177,28 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
           mma_bf16(sc[nt + 1], alo, b2, b3);
         }
       }
-      // mask, running max and sum (the sum stays per thread until the end)
+      // mask, running max and sum (the sum stays per thread until the end).  Only the last
+      // tile of a row's keys needs the mask: a tile that every row of the warp sees whole skips
+      // it (rows that do not exist hold zeros; their results are never written).
+      const int last_key = key0 + TA_TILE - 1;
+      const bool whole = __all_sync(0xffffffffu, last_key < k_end && (!ok0 || last_key <= lim0) &&
+                                                     (!ok1 || last_key <= lim1));
       float mt[2] = {-CUDART_INF_F, -CUDART_INF_F};
+      if (!whole) {
+#pragma unroll
+        for (int nt = 0; nt < TA_TILE / 8; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int key = key0 + nt * 8 + 2 * t + e;
+            if (!(ok0 && key < k_end && key <= lim0)) sc[nt][e] = -CUDART_INF_F;
+            if (!(ok1 && key < k_end && key <= lim1)) sc[nt][2 + e] = -CUDART_INF_F;
+          }
+        }
+      }
 #pragma unroll
       for (int nt = 0; nt < TA_TILE / 8; ++nt) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int key = key0 + nt * 8 + 2 * t + e;
-          if (!(ok0 && key < k_end && key <= lim0)) sc[nt][e] = -CUDART_INF_F;
-          if (!(ok1 && key < k_end && key <= lim1)) sc[nt][2 + e] = -CUDART_INF_F;
           mt[0] = fmaxf(mt[0], sc[nt][e]);
           mt[1] = fmaxf(mt[1], sc[nt][2 + e]);
         }
@@ -207,14 +220,26 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
         o[dt][2] *= corr[1];
         o[dt][3] *= corr[1];
       }
+      if (whole) {
 #pragma unroll
-      for (int nt = 0; nt < TA_TILE / 8; ++nt) {
+        for (int nt = 0; nt < TA_TILE / 8; ++nt) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float mm = mn[e >> 1];
-          const float p = sc[nt][e] == -CUDART_INF_F ? 0.f : __expf(sc[nt][e] - mm);
-          sc[nt][e] = p;
-          l_run[e >> 1] += p;
+          for (int e = 0; e < 4; ++e) {
+            const float p = __expf(sc[nt][e] - mn[e >> 1]);
+            sc[nt][e] = p;
+            l_run[e >> 1] += p;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int nt = 0; nt < TA_TILE / 8; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float mm = mn[e >> 1];
+            const float p = sc[nt][e] == -CUDART_INF_F ? 0.f : __expf(sc[nt][e] - mm);
+            sc[nt][e] = p;
+            l_run[e >> 1] += p;
+          }
         }
       }
 #pragma unroll
