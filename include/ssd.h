@@ -359,9 +359,12 @@ int ssd_fast_pack_roundtrip_host(const ssd_model_config* cfg, int32_t n_cta, con
  *   epilogue 1: ksplit must be 1; dev_out float [M, n_rows] = acc (the LM-head form).
  *   epilogue 2: ksplit must be 1; weight rows are (gate_j, up_j) pairs; dev_out receives
  *               SiLU(gate_j) * up_j as a packed operand of n_rows / 2 columns:
- *               byte(part, t, j) = (j / 16) * Mpad * 64 + ((j / 8) % 2) * Mpad * 32 + part * Mpad * 16
- *                                  + t * 16 + (j % 8) * 2,  part 0 = bf16 leading part of the
- *               value, part 1 = bf16 of the remainder ((n_rows / 2 rounded up to 16) * Mpad * 4 bytes).
+ *               byte(part, t, j) = ((t / Mc) * KS + j / 16) * Mc * 64 + ((j / 8) % 2) * Mc * 32
+ *                                  + part * Mc * 16 + (t % Mc) * 16 + (j % 8) * 2,
+ *               part 0 = bf16 leading part of the value, part 1 = bf16 of the remainder; KS =
+ *               n_rows / 2 columns rounded up to 16, over 16; the rows are stored in C chunks of
+ *               Mc rows: C = 1, Mc = Mpad up to 256 rows, else C = ceil(Mpad / 256) and Mc = Mpad / C
+ *               rounded up to 16 (KS * C * Mc * 64 bytes in all).
  * Enqueues on `stream`; SSD_ERR_BAD_PARAM for sizes outside the ranges above. */
 size_t ssd_tc_gemm_scratch_bytes(int32_t M, int32_t n_rows, int32_t K);
 int ssd_tc_gemm_check(const void* dev_w, const float* dev_x, int32_t M, int32_t n_rows, int32_t K,

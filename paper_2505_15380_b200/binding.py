@@ -427,7 +427,9 @@ def tc_gemm_check(w: torch.Tensor, x: torch.Tensor, ksplit: int, epilogue: int, 
         elif epilogue == 1:
             out = torch.zeros((M, n_rows), dtype=torch.float32, device=w.device)
         else:
-            out = torch.zeros(((n_rows // 2 + 15) // 16) * Mpad * 64, dtype=torch.uint8, device=w.device)
+            chunks = 1 if Mpad <= 256 else (Mpad + 255) // 256
+            mc = Mpad if chunks == 1 else ((Mpad + chunks - 1) // chunks + 15) // 16 * 16
+            out = torch.zeros(((n_rows // 2 + 15) // 16) * chunks * mc * 64, dtype=torch.uint8, device=w.device)
         check(L.ssd_tc_gemm_check(w.data_ptr(), x.data_ptr(), M, n_rows, K, ksplit, epilogue,
                                   scratch.data_ptr(), need, out.data_ptr(), status.data_ptr(),
                                   _stream_ptr(stream)))

@@ -210,9 +210,15 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap, int n_p
   p.tc_xa = p.tc_xattn = p.tc_xact = p.tc_part = 0;
   if (c.weight_dtype == 1 && M > FAST_MAX_T && M <= TC_MAX_ROWS) {
     const int Mpad = tc_round16((int)M), n_sm = fast_cta_count();
-    p.tc_xa = take(tc_act_bytes(Mpad, (int)d));
-    p.tc_xattn = take(tc_act_bytes(Mpad, (int)qd));
-    p.tc_xact = take(tc_act_bytes(Mpad, (int)F));
+    // the row chunks of an operand depend on the rows of the forward: room for the largest
+    size_t rows_max = 0;
+    for (int mp = 16; mp <= Mpad; mp += 16) {
+      const TcChunks ch = tc_chunks(mp);
+      rows_max = std::max(rows_max, (size_t)ch.n * ch.rows);
+    }
+    p.tc_xa = take((size_t)((d + 15) / 16) * rows_max * 64);
+    p.tc_xattn = take((size_t)((qd + 15) / 16) * rows_max * 64);
+    p.tc_xact = take((size_t)((F + 15) / 16) * rows_max * 64);
     size_t part = 0;
     const int rows[3] = {(int)(qd + 2 * kvd), (int)d, (int)d}, ks[3] = {(int)d, (int)qd, (int)F};
     for (int i = 0; i < 3; ++i) {

@@ -18,15 +18,23 @@
 //
 //   weights, per (tile of 128 rows, k-step of 16 columns) one 4 KB block:
 //       byte(r, k) = (k / 8) * 2048 + r * 16 + (k % 8) * 2           leading 2048, stride 128
-//   activations (Mpad token rows, a multiple of 16), per k-step one block of Mpad * 64 bytes:
-//       byte(part, t, k) = (k / 8) * Mpad * 32 + part * Mpad * 16 + t * 16 + (k % 8) * 2
+//   activations (Mpad token rows, a multiple of 16): up to 256 rows are one chunk of Mc = Mpad
+//   rows; more are ceil(Mpad / 256) chunks of Mc = Mpad / chunks (rounded up to 16) rows each.
+//   A chunk is stored whole, per k-step one block of Mc * 64 bytes:
+//       byte(part, t, k) = ((t / Mc) * KS + k / 16) * Mc * 64
+//                          + ((k / 8) % 2) * Mc * 32 + part * Mc * 16 + (t % Mc) * 16 + (k % 8) * 2
+//   (KS = k-steps of the operand), so that a CTA that multiplies one chunk of rows - see below -
+//   reads its share of a k-step as one contiguous run,
 //   with part 0 = bf16 leading part of the fp32 activation, part 1 = bf16 of the remainder: the
 //   tensor cores multiply both with the exact bf16 weights, so products are exact to ~2^-17
 //   relative, as in the small-batch kernel.  The two parts of a token sit Mpad rows apart in one
 //   2 * Mpad-row operand: with up to 256 token rows one instruction multiplies both (N = 2 Mpad,
 //   the two halves of the accumulator are added in the epilogue), which matters because an
 //   instruction costs ~190 cycles whatever its N (measured); with more rows the two parts are
-//   separate instructions into the same accumulator columns.
+//   separate instructions into the same accumulator columns, and a CTA owns TWO tiles of weight
+//   rows x one chunk of token rows (2 x Mc <= 512 accumulator columns): at 448 rows the
+//   projections are bound by the operand traffic from L2 into the SMs, and two tiles per CTA
+//   share every activation block they load (5.5 KB per instruction instead of 8).
 //
 // K is split across CTAs where a projection has too few row tiles to occupy the GPU; the partial
 // sums go to a workspace and the row-wise kernel that consumes the projection adds them in a
@@ -80,10 +88,49 @@ inline int tc_round16(int m) { return (m + 15) / 16 * 16; }
 inline size_t tc_weight_bytes(int n_rows, int K) {
   return (size_t)((n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS) * ((K + 15) / 16) * TC_WBLOCK;
 }
-// Bytes of a packed activation operand of K columns for Mpad rows.
-inline size_t tc_act_bytes(int Mpad, int K) { return (size_t)((K + 15) / 16) * Mpad * 64; }
+// Row chunks of a packed activation operand of M rows (see the layout above).
+struct TcChunks {
+  int n, rows;  // chunks, rows per chunk (a multiple of 16)
+};
+inline TcChunks tc_chunks(int M) {
+  const int Mpad = tc_round16(M);
+  TcChunks c;
+  c.n = Mpad <= 256 ? 1 : (Mpad + 255) / 256;
+  c.rows = c.n == 1 ? Mpad : tc_round16((Mpad + c.n - 1) / c.n);
+  return c;
+}
+// Bytes of a packed activation operand of K columns for M rows.
+inline size_t tc_act_bytes(int M, int K) {
+  const TcChunks c = tc_chunks(M);
+  return (size_t)((K + 15) / 16) * c.n * c.rows * 64;
+}
+// Byte offset of element (part, t, k) of a packed operand with chunks of Mc rows and KS k-steps.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline size_t tc_act_off(int Mc, int KS, int part, int t, int k) {
+  const int ch = t / Mc, tl = t - ch * Mc;
+  return ((size_t)ch * KS + (size_t)(k >> 4)) * ((size_t)Mc * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mc * 32) +
+         (size_t)part * ((size_t)Mc * 16) + (size_t)tl * 16 + (size_t)(k & 7) * 2;
+}
+// The same offset in two terms, for code that writes many columns of one row: the row's term
+// (its chunk and its place in it) and the column's.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline size_t tc_act_row_off(int Mc, int KS, int t) {
+  const int ch = t / Mc, tl = t - ch * Mc;
+  return (size_t)ch * KS * ((size_t)Mc * 64) + (size_t)tl * 16;
+}
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline size_t tc_act_col_off(int Mc, int k) {
+  return (size_t)(k >> 4) * ((size_t)Mc * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mc * 32) + (size_t)(k & 7) * 2;
+}
 // K slices for a projection of n_rows x K on n_sm SMs: enough CTAs to occupy the GPU, at least
-// four k-steps each.
+// four k-steps each.  (With more than 256 token rows a CTA owns two tiles of one row chunk, and
+// there are at least two chunks: the grid is no smaller than one CTA per tile.)
 inline int tc_ksplit(int n_rows, int K, int n_sm) {
   const int tiles = (n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS, ks = (K + 15) / 16;
   int s = n_sm / tiles;

@@ -292,7 +292,7 @@ tc_attn_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_layer
 template <int HD>
 __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32_t* __restrict__ len, RowMap rm,
                                      int cap, int Hq, int nsplit, int keys_per_split,
-                                     uint8_t* __restrict__ apack, int Mpad) {
+                                     uint8_t* __restrict__ apack, int Mc) {
   const int h = blockIdx.x, m = blockIdx.y;
   const int bi = m / rm.R, b = rm.b0 + bi;
   tc_pdl_trigger();
@@ -317,6 +317,7 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
   for (int s = threadIdx.x; s < ns; s += blockDim.x) s_w[s] = s_m[s] == -CUDART_INF_F ? 0.f : __expf(s_m[s] - m_tot);
   __syncthreads();
   const float inv = 1.f / denom;
+  uint8_t* arow = apack + tc_act_row_off(Mc, (Hq * HD + 15) >> 4, m);
   for (int d = threadIdx.x * 2; d < HD; d += blockDim.x * 2) {
     float o0 = 0.f, o1 = 0.f;
 #pragma unroll 4
@@ -330,10 +331,9 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
     const int k = h * HD + d;
     const __nv_bfloat162 hi = __floats2bfloat162_rn(o0, o1);
     const __nv_bfloat162 lo = __floats2bfloat162_rn(o0 - __low2float(hi), o1 - __high2float(hi));
-    uint8_t* e = apack + (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mpad * 32) +
-                 (size_t)m * 16 + (size_t)(k & 7) * 2;
+    uint8_t* e = arow + tc_act_col_off(Mc, k);
     *reinterpret_cast<__nv_bfloat162*>(e) = hi;
-    *reinterpret_cast<__nv_bfloat162*>(e + (size_t)Mpad * 16) = lo;
+    *reinterpret_cast<__nv_bfloat162*>(e + (size_t)Mc * 16) = lo;
   }
 }
 
@@ -351,7 +351,8 @@ cudaError_t launch_t(const float* qrot, const bf16* kv_layer, const int32_t* len
   if (e != cudaSuccess) return e;
   count_launch();
   e = tc_launch_pdl(tc_attn_merge_kernel<HD>, dim3(Hq, rm.nb * rm.R), dim3(HD / 2 < 32 ? 32 : HD / 2), 0, st,
-                    (const float*)part, len, rm, cap, Hq, nsplit, keys_per_split, apack_out, Mpad);
+                    (const float*)part, len, rm, cap, Hq, nsplit, keys_per_split, apack_out,
+                    tc_chunks(rm.nb * rm.R).rows);
   if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();

@@ -2,13 +2,14 @@
 // memory (QKV, O, gate/up + SwiGLU, down, LM head of Eq. 4's decoder pass when more than 16 rows
 // are in flight).  Layouts and the reasons for them: tc.h.
 //
-// One CTA = one tile of 128 weight rows x one K slice x all token rows.  Warp 0 streams the
+// One CTA = one tile of 128 weight rows x one K slice x all token rows - or, with more than 256
+// token rows, two tiles x one K slice x one chunk of the rows.  Warp 0 streams the
 // operands: per pipeline stage, eight of its lanes issue bulk copies of the stage's weight blocks
-// (read once, marked evict-first) and of the matching activation blocks (re-read by every tile,
-// so they stay in L2), in pieces of 8 KB, all completing on the stage's "full" barrier.  Warp 1 owns tensor
-// memory and issues the MMAs: per k-step of 16 columns, for the leading and the remainder part of
-// the activations and for each range of at most 256 token columns, one tcgen05.mma (128 x N x 16,
-// bf16 x bf16 -> fp32) reading both operands straight from shared memory; a tcgen05.commit hands
+// (read once from HBM, marked evict-first) and of the matching activation blocks (re-read by every
+// tile, so they stay in L2), in pieces of 8 KB, all completing on the stage's "full" barrier.  Warp 1 owns tensor
+// memory and issues the MMAs: per k-step of 16 columns one tcgen05.mma over both parts of the
+// activations (up to 256 rows: 128 x 2 Mpad x 16), or one per part and tile (128 x Mc x 16), bf16 x
+// bf16 -> fp32, reading both operands straight from shared memory; a tcgen05.commit hands
 // the stage back to the copy warp through its "empty" barrier, a last one tells the epilogue
 // warps that the accumulator is complete.  Warps 2..5 read the accumulator, 32 lanes x 32 columns
 // at a time (lane = weight row, column = token), and apply the epilogue.
@@ -126,6 +127,8 @@ struct TcKernelParams {
   const uint8_t* w;
   const uint8_t* a;
   int n_rows, KS, M, Mpad, ld_part;  // KS = k-steps of the whole projection; ld_part = tiles * 128
+  int Mc;                            // token rows of a row chunk (= Mpad up to 256 rows)
+  int ntile;                         // weight-row tiles per CTA: 2 where the rows are chunked, else 1
   int sk, stages;                    // k-steps per stage, pipeline depth
   int wide;                          // 1: one instruction multiplies both parts (N over 2 * Mpad rows)
   int dual;                          // wide, and even / odd k-steps accumulate into two column sets
@@ -148,8 +151,14 @@ struct TcShared {
 __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_constant__ TcKernelParams P) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tile = blockIdx.x, split = blockIdx.y, nsplit = gridDim.y;
-  const uint32_t stage_w = (uint32_t)P.sk * TC_WBLOCK, act_block = (uint32_t)P.Mpad * 64u;
+  const int split = blockIdx.y, nsplit = gridDim.y, chunk = blockIdx.z;
+  const int tile0 = (int)blockIdx.x * P.ntile;                       // first weight-row tile of this CTA
+  const int n_tiles_all = P.ld_part / TC_TILE_ROWS;
+  const int ntile = min(P.ntile, n_tiles_all - tile0);               // a last odd tile stands alone
+  const int t0 = chunk * P.Mc;                                       // first token row of this CTA
+  const int rows_here = min(P.M - t0, P.Mc);                         // valid token rows
+  const uint32_t tile_w = (uint32_t)P.sk * TC_WBLOCK;                // one tile's weights of a stage
+  const uint32_t stage_w = (uint32_t)P.ntile * tile_w, act_block = (uint32_t)P.Mc * 64u;
   const uint32_t stage_a = (uint32_t)P.sk * act_block;
   uint8_t* smem_w = smem;
   uint8_t* smem_a = smem + (size_t)P.stages * stage_w;
@@ -187,35 +196,40 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     if (lane >= TC_ISSUERS) tc_pdl_wait();
     if (lane < TC_ISSUERS) {  // ---- operand copies: piece i of a stage is issued by lane i % TC_ISSUERS
       const uint64_t pol = policy_evict_first();
-      const uint8_t* wsrc = P.w + ((size_t)tile * P.KS + ks0) * TC_WBLOCK;
-      const uint8_t* asrc = P.a + (size_t)ks0 * act_block;
+      const uint8_t* wsrc = P.w + ((size_t)tile0 * P.KS + ks0) * TC_WBLOCK;
+      const size_t wtile = (size_t)P.KS * TC_WBLOCK;  // from one tile's weights to the next tile's
+      const uint8_t* asrc = P.a + ((size_t)chunk * P.KS + ks0) * act_block;
       // One stage's pieces; which = 1: weights, 2: activations, 3: both.  A lane arrives once per
-      // stage (with the weights, or with `both`), announcing all the bytes it will bring.
+      // stage (with the weights, or with `both`), announcing all the bytes it will bring.  Each
+      // tile's weights of the stage and the stage's activations are contiguous runs, cut into
+      // pieces of at most 8 KB.
       auto issue = [&](int it, int which) {
         const int s = it % P.stages;
         const int nks = min(P.sk, ks1 - ks0 - it * P.sk);
         const uint32_t bar = smem_u32(&S.full[s]);
         const uint32_t wbytes = (uint32_t)nks * TC_WBLOCK, abytes = (uint32_t)nks * act_block;
-        const uint32_t wp = (wbytes + TC_PIECE - 1) / TC_PIECE, ap = (abytes + TC_PIECE - 1) / TC_PIECE;
+        const uint32_t wp1 = (wbytes + TC_PIECE - 1) / TC_PIECE, wp = wp1 * (uint32_t)ntile;
+        const uint32_t ap = (abytes + TC_PIECE - 1) / TC_PIECE;
         const uint8_t* ws = wsrc + (size_t)it * P.sk * TC_WBLOCK;
         const uint8_t* as = asrc + (size_t)it * P.sk * act_block;
-        if (which & 1) {
-          uint32_t mine = 0;
-          for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS)
-            mine += i < wp ? min(TC_PIECE, wbytes - i * TC_PIECE) : min(TC_PIECE, abytes - (i - wp) * TC_PIECE);
-          mbar_expect_tx(bar, mine);
-        }
+        // one pass: issue, and add up what this lane announces (the arrival may follow the
+        // copies: the phase cannot complete before all issuing lanes have arrived)
+        uint32_t mine = 0;
         for (uint32_t i = lane; i < wp + ap; i += TC_ISSUERS) {
           if (i < wp) {
-            const uint32_t off = i * TC_PIECE;
+            const uint32_t tl = i >= wp1 ? 1u : 0u, off = (i - tl * wp1) * TC_PIECE;  // at most two tiles
+            const uint32_t nb = min(TC_PIECE, wbytes - off);
+            mine += nb;
             if (which & 1)
-              bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w) + off, ws + off, min(TC_PIECE, wbytes - off), bar, pol);
+              bulk_g2s_hint(smem_u32(smem_w + (size_t)s * stage_w) + tl * tile_w + off, ws + (size_t)tl * wtile + off, nb,
+                            bar, pol);
           } else {
-            const uint32_t off = (i - wp) * TC_PIECE;
-            if (which & 2)
-              bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a) + off, as + off, min(TC_PIECE, abytes - off), bar);
+            const uint32_t off = (i - wp) * TC_PIECE, nb = min(TC_PIECE, abytes - off);
+            mine += nb;
+            if (which & 2) bulk_g2s(smem_u32(smem_a + (size_t)s * stage_a) + off, as + off, nb, bar);
           }
         }
+        if (which & 1) mbar_expect_tx(bar, mine);
       };
       // first fill of the ring: the weights at once, the activations when the predecessor is done
       const int first = min(n_iter, P.stages);
@@ -245,31 +259,31 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
         const uint32_t wb = smem_u32(smem_w + (size_t)s * stage_w), ab = smem_u32(smem_a + (size_t)s * stage_a);
         for (int j = 0; j < nks; ++j) {
           const uint64_t da = umma_desc(wb + (uint32_t)j * TC_WBLOCK, 2048u, 128u);
-          const uint32_t blk = ab + (uint32_t)j * act_block, lead = (uint32_t)P.Mpad * 32u;
+          const uint32_t blk = ab + (uint32_t)j * act_block, lead = (uint32_t)P.Mc * 32u;
           if (dual) {
             // Back-to-back instructions into the same accumulator columns wait for one another
             // (~280 cycles each, measured, against ~165 when they alternate between column
-            // ranges): even k-steps add into columns [0, 2 Mpad), odd ones into [2 Mpad, 4 Mpad).
+            // ranges): even k-steps add into columns [0, 2 Mc), odd ones into [2 Mc, 4 Mc).
             const int kk = it * P.sk + j;
-            umma_bf16(tmem + (uint32_t)((kk & 1) * 2 * P.Mpad), da, umma_desc(blk, lead, 128u), umma_idesc(2 * P.Mpad),
+            umma_bf16(tmem + (uint32_t)((kk & 1) * 2 * P.Mc), da, umma_desc(blk, lead, 128u), umma_idesc(2 * P.Mc),
                       kk >= 2 ? 1u : 0u);
           } else if (P.wide) {
-            // the operand's 2 * Mpad rows (leading parts, then remainders) in ranges of <= 256:
-            // accumulator columns [0, Mpad) receive W x_hi, [Mpad, 2 Mpad) receive W x_lo
+            // the operand's 2 * Mc rows (leading parts, then remainders) in ranges of <= 256:
+            // accumulator columns [0, Mc) receive W x_hi, [Mc, 2 Mc) receive W x_lo
             for (int c = 0; c < P.nchunks; ++c) {
-              const int n = min(P.chunk_n, 2 * P.Mpad - c * P.chunk_n);
+              const int n = min(P.chunk_n, 2 * P.Mc - c * P.chunk_n);
               umma_bf16(tmem + (uint32_t)(c * P.chunk_n), da, umma_desc(blk + (uint32_t)(c * P.chunk_n) * 16u, lead, 128u),
                         umma_idesc(n), (it > 0 || j > 0) ? 1u : 0u);
             }
           } else {
+            // more than 256 token rows: this CTA's chunk of Mc rows against its one or two tiles;
+            // tile u accumulates in columns [u Mc, (u + 1) Mc), both parts into the same columns
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-              for (int c = 0; c < P.nchunks; ++c) {
-                const int n = min(P.chunk_n, P.Mpad - c * P.chunk_n);
-                umma_bf16(tmem + (uint32_t)(c * P.chunk_n), da,
-                          umma_desc(blk + (uint32_t)(part * P.Mpad + c * P.chunk_n) * 16u, lead, 128u), umma_idesc(n),
+              for (int u = 0; u < ntile; ++u)
+                umma_bf16(tmem + (uint32_t)(u * P.Mc), umma_desc(wb + (uint32_t)u * tile_w + (uint32_t)j * TC_WBLOCK, 2048u, 128u),
+                          umma_desc(blk + (uint32_t)(part * P.Mc) * 16u, lead, 128u), umma_idesc(P.Mc),
                           (it > 0 || j > 0 || part > 0) ? 1u : 0u);
-              }
             }
           }
         }
@@ -279,37 +293,40 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
     }
   } else {
     // ---- epilogue: warp w may read the 32 tensor-memory lanes of quarter w % 4
-    const int q = warp & 3, row = q * 32 + lane, n = tile * TC_TILE_ROWS + row;
+    const int q = warp & 3, row = q * 32 + lane;
     const bool ok = mbar_wait(smem_u32(&S.accum), 0u, abort);
     tc_fence_after();
     if (ok && !*abort) {
-      for (int c0 = 0; c0 < P.M; c0 += 32) {
+     for (int u = 0; u < ntile; ++u) {
+      const int tile = tile0 + u, n = tile * TC_TILE_ROWS + row;
+      const uint32_t cb = (uint32_t)(u * P.Mc);  // the tile's accumulator columns (two-tile CTAs)
+      for (int c0 = 0; c0 < rows_here; c0 += 32) {
         uint32_t v[32];
-        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + cb + (uint32_t)c0, v);
         if (P.wide) {  // add the remainder part's products
           uint32_t w[32];
-          tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(P.Mpad + c0), w);
+          tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(P.Mc + c0), w);
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(w[i]));
           if (dual) {  // and the odd k-steps' column set, in a fixed order
             uint32_t x[32];
-            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(2 * P.Mpad + c0), x);
-            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(3 * P.Mpad + c0), w);
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(2 * P.Mc + c0), x);
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(3 * P.Mc + c0), w);
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               v[i] = __float_as_uint(__uint_as_float(v[i]) + (__uint_as_float(x[i]) + __uint_as_float(w[i])));
           }
         }
         if (P.epi == TC_EPI_PARTIAL) {
-          float* dst = P.part + ((size_t)split * P.Mpad + c0) * P.ld_part + n;
+          float* dst = P.part + ((size_t)split * P.Mpad + t0 + c0) * P.ld_part + n;
 #pragma unroll
           for (int i = 0; i < 32; ++i)
-            if (c0 + i < P.M) dst[(size_t)i * P.ld_part] = __uint_as_float(v[i]);
+            if (c0 + i < rows_here) dst[(size_t)i * P.ld_part] = __uint_as_float(v[i]);
         } else if (P.epi == TC_EPI_STORE) {
           if (n < P.n_rows) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (c0 + i < P.M) P.out[(size_t)(c0 + i) * P.ldo + n] = __uint_as_float(v[i]);
+              if (c0 + i < rows_here) P.out[(size_t)(t0 + c0 + i) * P.ldo + n] = __uint_as_float(v[i]);
           }
         } else {
           // TC_EPI_SWIGLU: even lanes hold gate_j, odd lanes up_j, j = n / 2.  The warp's 16 columns j
@@ -334,16 +351,19 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
             *reinterpret_cast<bf16*>(e + TC_STG_STRIDE) = lo;
           }
           __syncwarp();
-          if (j0 < ((P.n_rows / 2 + 15) & ~15) && c0 + lane < P.M) {
-            uint8_t* blk = P.act_out + (size_t)(j0 >> 4) * ((size_t)P.Mpad * 64) + (size_t)(c0 + lane) * 16;
+          if (j0 < ((P.n_rows / 2 + 15) & ~15) && c0 + lane < rows_here) {
+            // the output operand has the same rows, so the same chunks, and n_rows / 2 columns
+            uint8_t* blk = P.act_out + ((size_t)chunk * ((P.n_rows / 2 + 15) >> 4) + (size_t)(j0 >> 4)) * ((size_t)P.Mc * 64) +
+                           (size_t)(c0 + lane) * 16;
 #pragma unroll
             for (int hp = 0; hp < 4; ++hp)  // hp = half * 2 + part
-              *reinterpret_cast<uint4*>(blk + (size_t)hp * ((size_t)P.Mpad * 16)) =
+              *reinterpret_cast<uint4*>(blk + (size_t)hp * ((size_t)P.Mc * 16)) =
                   *reinterpret_cast<const uint4*>(stg + (uint32_t)hp * TC_STG_STRIDE + (uint32_t)lane * 16u);
           }
           __syncwarp();
         }
       }
+     }
     }
   }
   tc_fence_before();
@@ -428,7 +448,11 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   // by a little leaves room for a second CTA per SM so that it still runs in one wave; any other
   // grid takes the whole shared memory: with few token rows the weight stream is latency-bound,
   // and what a CTA keeps in flight is what it gets.
-  const size_t per_ks = (size_t)TC_WBLOCK + (size_t)p.Mpad * 64;
+  const TcChunks ch = tc_chunks(g.M);
+  p.Mc = ch.rows;
+  p.ntile = ch.n > 1 ? 2 : 1;
+  const int grid_x = (tiles + p.ntile - 1) / p.ntile;
+  const size_t per_ks = (size_t)p.ntile * TC_WBLOCK + (size_t)p.Mc * 64;
   int n_sm = 148;
   {
     int dev = 0;
@@ -436,7 +460,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
       n_sm = 148;
   }
-  const int ctas = tiles * g.ksplit;
+  const int ctas = grid_x * g.ksplit * ch.n;
   const bool two_per_sm = p.Mpad <= 128 && ctas > n_sm && ctas <= 2 * n_sm;  // 2 x 256 columns
   const size_t budget = two_per_sm ? 100 * 1024 : 216 * 1024;
   p.sk = 4;
@@ -444,17 +468,17 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   p.stages = (int)(budget / (p.sk * per_ks));
   if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
   if (p.stages < 2) return cudaErrorInvalidValue;
-  p.wide = p.Mpad <= 256;  // both parts' products fit the 512 tensor-memory columns side by side
-  const int op_rows = p.wide ? 2 * p.Mpad : p.Mpad;
-  p.nchunks = (op_rows + 255) / 256;
-  p.chunk_n = tc_round16((op_rows + p.nchunks - 1) / p.nchunks);
-  p.dual = p.wide && 4 * p.Mpad <= 512 && !two_per_sm;  // two CTAs on an SM have 256 columns each
+  p.wide = ch.n == 1;  // both parts' products fit the 512 tensor-memory columns side by side
+  const int op_rows = p.wide ? 2 * p.Mc : p.ntile * p.Mc;  // accumulator columns
+  p.nchunks = p.wide ? (op_rows + 255) / 256 : 1;
+  p.chunk_n = p.wide ? tc_round16((op_rows + p.nchunks - 1) / p.nchunks) : p.Mc;
+  p.dual = p.wide && 4 * p.Mc <= 512 && !two_per_sm;  // two CTAs on an SM have 256 columns each
   p.tmem_cols = 32;
   while (p.tmem_cols < (p.dual ? 2 : 1) * op_rows) p.tmem_cols <<= 1;
   const size_t smem = (size_t)p.stages * p.sk * per_ks + sizeof(TcShared) + 64;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
-  e = tc_launch_pdl(tc_gemm_kernel, dim3(tiles, g.ksplit), dim3(TC_THREADS), smem, st, p);
+  e = tc_launch_pdl(tc_gemm_kernel, dim3(grid_x, g.ksplit, ch.n), dim3(TC_THREADS), smem, st, p);
   if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();

@@ -9,17 +9,14 @@ namespace ssd {
 
 namespace {
 
-// Byte offset of element (part, t, k) of a packed activation operand (tc.h).
-__device__ __forceinline__ size_t act_off(int Mpad, int part, int t, int k) {
-  return (size_t)(k >> 4) * ((size_t)Mpad * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mpad * 32) +
-         (size_t)part * ((size_t)Mpad * 16) + (size_t)t * 16 + (size_t)(k & 7) * 2;
-}
-// Columns (k, k + 1), k even, of token t: bf16 leading parts and remainders.
-__device__ __forceinline__ void store_pair(uint8_t* apack, int Mpad, int t, int k, float x0, float x1) {
+// Columns (k, k + 1), k even, of one token of a packed operand (chunks of Mc rows: tc.h); `row`
+// points at the token's row term (tc_act_row_off): bf16 leading parts and remainders.
+__device__ __forceinline__ void store_pair(uint8_t* row, int Mc, int k, float x0, float x1) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
   const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
-  *reinterpret_cast<__nv_bfloat162*>(apack + act_off(Mpad, 0, t, k)) = h;
-  *reinterpret_cast<__nv_bfloat162*>(apack + act_off(Mpad, 1, t, k)) = l;
+  const size_t off = tc_act_col_off(Mc, k);
+  *reinterpret_cast<__nv_bfloat162*>(row + off) = h;
+  *reinterpret_cast<__nv_bfloat162*>(row + off + (size_t)Mc * 16) = l;
 }
 
 // Sum over the K slices of a projection's partial sums for two adjacent columns, in slice order
@@ -53,7 +50,7 @@ constexpr int TC_ROWS_DEEP = 256;  // up to this many rows (CTAs) the deep varia
 template <int NF, int MINB>
 __global__ void __launch_bounds__(256, MINB)
 tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int nsplit, int ld_part, int Mpad,
-                    int d, const bf16* __restrict__ gain, float eps, uint8_t* __restrict__ apack) {
+                    int Mc, int d, const bf16* __restrict__ gain, float eps, uint8_t* __restrict__ apack) {
   extern __shared__ float row[];
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
@@ -77,16 +74,18 @@ tc_norm_pack_kernel(float* __restrict__ h, const float* __restrict__ part, int n
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float inv = rsqrtf(tot / (float)d + eps);
+  uint8_t* arow = apack + tc_act_row_off(Mc, (d + 15) >> 4, m);
   for (int j = tid * 2; j < d; j += 512) {
     const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + j));
-    store_pair(apack, Mpad, m, j, row[j] * inv * g.x, row[j + 1] * inv * g.y);
+    store_pair(arow, Mc, j, row[j] * inv * g.x, row[j + 1] * inv * g.y);
   }
 }
 
-__global__ void tc_pack_rows_kernel(const float* __restrict__ x, int K, int Mpad, uint8_t* __restrict__ apack) {
+__global__ void tc_pack_rows_kernel(const float* __restrict__ x, int K, int Mc, uint8_t* __restrict__ apack) {
   const int m = blockIdx.x;
+  uint8_t* arow = apack + tc_act_row_off(Mc, (K + 15) >> 4, m);
   for (int j = threadIdx.x * 2; j < K; j += blockDim.x * 2)
-    store_pair(apack, Mpad, m, j, x[(size_t)m * K + j], x[(size_t)m * K + j + 1]);
+    store_pair(arow, Mc, j, x[(size_t)m * K + j], x[(size_t)m * K + j + 1]);
 }
 
 // One CTA per row: q/k/v = sum of the K slices + bias; rotate q and k by the row's position
@@ -156,15 +155,15 @@ void launch_tc_norm_pack(float* h, const float* part, int nsplit, int ld_part, i
                          const bf16* gain, float eps, uint8_t* apack, cudaStream_t st) {
   if (M <= TC_ROWS_DEEP)
     tc_launch_pdl(tc_norm_pack_kernel<24, 1>, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0,
-                  ld_part, tc_round16(M), d, gain, eps, apack);
+                  ld_part, tc_round16(M), tc_chunks(M).rows, d, gain, eps, apack);
   else
     tc_launch_pdl(tc_norm_pack_kernel<8, 4>, dim3(M), dim3(256), (size_t)d * 4, st, h, part, part ? nsplit : 0,
-                  ld_part, tc_round16(M), d, gain, eps, apack);
+                  ld_part, tc_round16(M), tc_chunks(M).rows, d, gain, eps, apack);
   count_launch();
 }
 
 void launch_tc_pack_rows(const float* x, int M, int K, uint8_t* apack, cudaStream_t st) {
-  tc_pack_rows_kernel<<<M, 128, 0, st>>>(x, K, tc_round16(M), apack);
+  tc_pack_rows_kernel<<<M, 128, 0, st>>>(x, K, tc_chunks(M).rows, apack);
   count_launch();
 }
 

@@ -71,11 +71,14 @@ def test_swiglu_epilogue_writes_a_packed_operand(M, F, K):
     ref = gate / (1.0 + np.exp(-gate)) * up
     raw = out.cpu().numpy().view(np.uint16)                        # bf16 bit patterns
     Mpad = (M + 15) // 16 * 16
+    chunks = 1 if Mpad <= 256 else (Mpad + 255) // 256       # rows are stored in chunks of Mc
+    Mc = Mpad if chunks == 1 else ((Mpad + chunks - 1) // chunks + 15) // 16 * 16
+    KS = (F + 15) // 16
     t = np.arange(M)[:, None]
     j = np.arange(F)[None, :]
-    base = (j // 16) * (Mpad * 64) + ((j // 8) % 2) * (Mpad * 32) + t * 16 + (j % 8) * 2
+    base = ((t // Mc) * KS + j // 16) * (Mc * 64) + ((j // 8) % 2) * (Mc * 32) + (t % Mc) * 16 + (j % 8) * 2
     hi = synth.from_bf16_bits(raw[(base // 2)]).astype(np.float64)
-    lo = synth.from_bf16_bits(raw[((base + Mpad * 16) // 2)]).astype(np.float64)
+    lo = synth.from_bf16_bits(raw[((base + Mc * 16) // 2)]).astype(np.float64)
     assert np.abs(hi + lo - ref).max() <= 3e-5 * np.abs(ref).max() + 1e-6
     assert np.abs(hi - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6     # hi alone is the bf16 rounding
     assert np.abs(lo).max() > 0
