@@ -332,10 +332,11 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
   const int n_sm = m->tc.n_sm;
   auto ld_of = [](int rows) { return (rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS * TC_TILE_ROWS; };
   const int ks_qkv = tc_ksplit(nq, d, n_sm), ks_o = tc_ksplit(d, qd, n_sm), ks_d = tc_ksplit(d, F, n_sm);
-  // key splits of the attention: whole 64-key tiles, and at most two CTAs per SM in all, which
-  // is what fits at once (a second, partly filled wave would cost as much as the first)
+  // key splits of the attention: whole 64-key tiles, and no more CTAs in all than the SMs hold
+  // at once (a second, partly filled wave would cost as much as the first)
   const int G = c.n_q_heads / c.n_kv_heads, rowgroups = (G * rm.R + 63) / 64;
-  long long want = (2LL * n_sm) / ((long long)rm.nb * c.n_kv_heads * rowgroups);  // splits that still fit one wave
+  long long want = ((long long)tc_attention_ctas_per_sm(c.head_dim) * n_sm) /
+                   ((long long)rm.nb * c.n_kv_heads * rowgroups);  // splits that still fit one wave
   if (want < 1) want = 1;
   long long kps = ((s->cap + want - 1) / want + 63) / 64 * 64;
   if (kps < 64) kps = 64;
@@ -363,7 +364,7 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
                        s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim, s->page_table, s->max_pages,
                        s->status, st);
     SSD_CUDA(launch_tc_attention(s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim,
-                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, s->page_table, s->max_pages, st));
+                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, s->page_table, s->max_pages, s->status, st));
     g.w = t.w_o; g.a = s->tc_xattn; g.n_rows = d; g.K = qd; g.ksplit = ks_o;
     SSD_CUDA(launch_tc_gemm(g, st));
     launch_tc_norm_pack(s->h, s->tc_part, ks_o, ld_of(d), M, d, (const bf16*)w.norm2, c.rms_eps, s->tc_xa, st);
