@@ -176,6 +176,13 @@ int ssd_paged_state(ssd_streams* s, int32_t* host_pages_used, int32_t* host_free
  * kernels only.  Both produce the same results up to fp32 summation order. */
 int ssd_streams_set_path(ssd_streams* s, int32_t path);
 
+/* Diagnostics of the batched forward (more than 16 rows, or a paged cache): which kernel computes
+ * the attention of Eq. 4.  0 (default): the tcgen05 kernel where a CTA's key range is long
+ * enough to pay for its set-up (1024 keys or more; head sizes 64 and 128), else the warp-level
+ * tensor-core kernel; 1: the warp-level kernel always; 2: the tcgen05 kernel wherever the head
+ * size allows.  Both produce the same results up to fp32 summation order. */
+int ssd_streams_set_attention_kernel(ssd_streams* s, int32_t which);
+
 /* Precision of the activations that enter the tensor cores in the persistent kernel (weights and
  * K/V are bf16 as stored, accumulation is fp32, the residual stream is kept in fixed point, in
  * both modes).  on = 1 (default): each activation enters as its bf16 leading part plus the bf16

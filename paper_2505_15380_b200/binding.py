@@ -21,6 +21,7 @@ EXPORTS = [
     "ssd_model_arena_bytes", "ssd_model_create", "ssd_model_destroy", "ssd_kv_bytes",
     "ssd_workspace_bytes", "ssd_streams_create", "ssd_streams_destroy", "ssd_streams_set_path",
     "ssd_streams_set_activation_split",
+    "ssd_streams_set_attention_kernel",
     "ssd_streams_set_trace", "ssd_forward", "ssd_fast_plan_host",
     "ssd_fast_pack_roundtrip_host", "ssd_kv_truncate",
     "ssd_streams_get_state", "ssd_prefill", "ssd_draft_step", "ssd_verify", "ssd_verify_host",
@@ -89,6 +90,7 @@ def lib() -> ctypes.CDLL:
     L.ssd_streams_destroy.argtypes = [vp]
     L.ssd_streams_set_path.argtypes = [vp, i32]
     L.ssd_streams_set_activation_split.argtypes = [vp, i32]
+    L.ssd_streams_set_attention_kernel.argtypes = [vp, i32]
     L.ssd_streams_set_trace.argtypes = [vp, vp, i32, i32]
     L.ssd_forward.argtypes = [vp, vp, vp, i32, vp, vp]
     L.ssd_fast_plan_host.argtypes = [cfgp, i32, ctypes.POINTER(ctypes.c_int64)]
@@ -236,6 +238,11 @@ class Streams:
     def set_path(self, path: int) -> None:
         """0: persistent small-batch kernel where the forward fits it (default); 1: generic kernels."""
         check(lib().ssd_streams_set_path(self.handle, path))
+
+    def set_attention_kernel(self, which: int) -> None:
+        """Batched forward: 0 picks the attention kernel by the key range per CTA (default), 1 the
+        warp-level tensor-core kernel always, 2 the tcgen05 kernel wherever the head size allows."""
+        check(lib().ssd_streams_set_attention_kernel(self.handle, which))
 
     def set_activation_split(self, on: bool) -> None:
         """Persistent kernel: True (default) feeds activations to the tensor cores as bf16 leading

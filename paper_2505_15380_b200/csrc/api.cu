@@ -364,7 +364,8 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
                        s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim, s->page_table, s->max_pages,
                        s->status, st);
     SSD_CUDA(launch_tc_attention(s->qrot, kv_layer, s->len, rm, s->cap, c.n_q_heads, c.n_kv_heads, c.head_dim,
-                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, s->page_table, s->max_pages, s->status, st));
+                                 s->part, nsplit, (int)kps, s->tc_xattn, Mpad, s->page_table, s->max_pages, s->attn_kernel,
+                                 s->status, st));
     g.w = t.w_o; g.a = s->tc_xattn; g.n_rows = d; g.K = qd; g.ksplit = ks_o;
     SSD_CUDA(launch_tc_gemm(g, st));
     launch_tc_norm_pack(s->h, s->tc_part, ks_o, ld_of(d), M, d, (const bf16*)w.norm2, c.rms_eps, s->tc_xa, st);
@@ -829,6 +830,7 @@ int streams_create_impl(const ssd_model* m, int32_t batch, int32_t capacity_toke
   s->free_top = paged ? (int32_t*)(W + p.free_top) : nullptr;
   if (paged) s->key_split = 0;
   s->path = 0;
+  s->attn_kernel = 0;
   s->split_act = 1;
   s->trace = nullptr;
   s->trace_cap = 0;
@@ -903,6 +905,13 @@ int ssd_forward(ssd_model* model, ssd_streams* s, const int32_t* dev_draft_token
   if (use_fast(model, s, rm)) return forward_fast(model, s, rm, nullptr, dev_draft_tokens, dev_logits, st);
   launch_gather_verify_ids(s->pending, dev_draft_tokens, gamma, s->B, s->row_ids, st);
   return forward(model, s, rm, dev_logits, st);
+}
+
+int ssd_streams_set_attention_kernel(ssd_streams* s, int32_t which) {
+  if (!s) return SSD_ERR_NULL;
+  if (which < 0 || which > 2) return SSD_ERR_BAD_PARAM;
+  s->attn_kernel = which;
+  return SSD_OK;
 }
 
 int ssd_streams_set_activation_split(ssd_streams* s, int32_t on) {

@@ -148,6 +148,7 @@ struct ssd_streams {
   size_t h_stage_in = 0;
   int split_act;     // persistent kernel: activations as bf16 hi + lo pairs (1) or plain bf16 (0)
   int path;          // 0: pick the persistent kernel when the forward fits it, 1: generic kernels only
+  int attn_kernel;   // batched path: 0 by key range per CTA, 1 warp-level kernel, 2 tcgen05 kernel
   long long* trace;  // optional phase-boundary clock trace of the persistent kernel (null: off)
   int trace_cap;
 };

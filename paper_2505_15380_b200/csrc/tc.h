@@ -188,10 +188,15 @@ void launch_page_release(const int32_t* len, int B, int32_t* page_table, int32_t
 cudaError_t launch_tc_attention(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm,
                                 int cap, int Hq, int Hkv, int hd, float* part, int nsplit,
                                 int keys_per_split, uint8_t* apack_out, int Mpad,
-                                const int32_t* page_table, int max_pages, int32_t* status, cudaStream_t st);
+                                const int32_t* page_table, int max_pages, int which_kernel, int32_t* status,
+                                cudaStream_t st);
 int tc_attention_ctas_per_sm(int hd);  // CTAs of the attention kernel an SM holds at once
 // tc_attention5.cu: the same partial results (one per row, head and key split) on tcgen05 tensor
-// cores, for head sizes 64 and 128; launch_tc_attention uses it where it applies.
+// cores, for head sizes 64 and 128.  It costs less per key and more per CTA than the warp-level
+// kernel (measured: 3.0 against 3.5 us per 64 keys, ~6 us more to start and finish), so
+// launch_tc_attention uses it from TC_ATTN5_MIN_KEYS keys per CTA on (which_kernel 0), always
+// (2, where the head size allows) or never (1).
+constexpr int TC_ATTN5_MIN_KEYS = 1024;
 cudaError_t launch_tc_attention5(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm, int cap,
                                  int Hq, int Hkv, int hd, float* part, int nsplit, int keys_per_split,
                                  const int32_t* page_table, int max_pages, int32_t* status, cudaStream_t st);

@@ -340,11 +340,12 @@ __global__ void tc_attn_merge_kernel(const float* __restrict__ part, const int32
 template <int HD>
 cudaError_t launch_t(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm, int cap, int Hq,
                      int Hkv, float* part, int nsplit, int keys_per_split, uint8_t* apack_out, int Mpad,
-                     const int32_t* page_table, int max_pages, int32_t* status, cudaStream_t st) {
+                     const int32_t* page_table, int max_pages, int which_kernel, int32_t* status, cudaStream_t st) {
   const int NQ = (Hq / Hkv) * rm.R, n_rowgroups = (NQ + TA_WARPS * 16 - 1) / (TA_WARPS * 16);
   const size_t smem = (size_t)4 * TA_TILE * (HD * 2 + 16) + (size_t)TA_WARPS * (HD / 16) * 32 * 32;
   cudaError_t e;
-  if (HD >= 64) {  // tcgen05 contractions
+  const bool t5 = HD >= 64 && (which_kernel == 2 || (which_kernel == 0 && keys_per_split >= TC_ATTN5_MIN_KEYS));
+  if (t5) {  // tcgen05 contractions
     e = launch_tc_attention5(qrot, kv_layer, len, rm, cap, Hq, Hkv, HD, part, nsplit, keys_per_split, page_table,
                              max_pages, status, st);
     if (e != cudaSuccess) return e;
@@ -372,12 +373,13 @@ int tc_attention_ctas_per_sm(int) { return 2; }
 cudaError_t launch_tc_attention(const float* qrot, const bf16* kv_layer, const int32_t* len, RowMap rm,
                                 int cap, int Hq, int Hkv, int hd, float* part, int nsplit,
                                 int keys_per_split, uint8_t* apack_out, int Mpad,
-                                const int32_t* page_table, int max_pages, int32_t* status, cudaStream_t st) {
+                                const int32_t* page_table, int max_pages, int which_kernel, int32_t* status,
+                                cudaStream_t st) {
   if (page_table && keys_per_split % TC_PAGE_TOKENS) return cudaErrorInvalidValue;
   switch (hd) {
-    case 32: return launch_t<32>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, status, st);
-    case 64: return launch_t<64>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, status, st);
-    case 128: return launch_t<128>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, status, st);
+    case 32: return launch_t<32>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, which_kernel, status, st);
+    case 64: return launch_t<64>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, which_kernel, status, st);
+    case 128: return launch_t<128>(qrot, kv_layer, len, rm, cap, Hq, Hkv, part, nsplit, keys_per_split, apack_out, Mpad, page_table, max_pages, which_kernel, status, st);
   }
   return cudaErrorInvalidValue;
 }

@@ -109,7 +109,8 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
              uniform_seed: int = 0, commit_and_repeat: bool = False,
              capacity: Optional[int] = None, path: int = 0, split: bool = True,
              max_strict_frac: float = 0.10, max_e2e_frac: float = 0.34, top_p: float = 0.0,
-             paged: Optional[tuple] = None, ras: Optional[tuple] = None) -> CaseResult:
+             paged: Optional[tuple] = None, ras: Optional[tuple] = None,
+             attn_kernel: int = 0) -> CaseResult:
     """kv_mode 'prefill': both sides load the seeded prefix through their own forward;
     'synthetic': seeded random K/V is written to the cache and handed to the oracle as input."""
     shape = wl.target
@@ -126,6 +127,7 @@ def run_case(wl: synth.Workload, *, beta: float, sigma: float, kv_mode: str = "p
     else:
         gs = binding.Streams(gmodel, B, cap, gamma)
     gs.set_path(path)          # 0: persistent kernel where the forward fits it, 1: generic kernels
+    gs.set_attention_kernel(attn_kernel)   # batched forward: 0 by key range, 1 warp-level, 2 tcgen05
     gs.set_activation_split(split)   # persistent kernel: bf16 activations, or bf16 hi + lo pairs
     which = list(range(B)) if oracle_streams is None else list(oracle_streams)
     prefixes = [synth.make_prefix(wl, b) for b in range(B)]

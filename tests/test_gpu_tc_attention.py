@@ -1,4 +1,5 @@
-"""The tcgen05 attention of the batched forward (head sizes 64 and 128) at its edges, through the
+"""The tcgen05 attention of the batched forward (head sizes 64 and 128; forced on, since by
+default it serves long key ranges only) at its edges, through the
 whole verify step against the float64 oracle: prefixes on both sides of the 64-key tile and of the
 page size, a stream with a single cached token, more than 64 query rows per kv head (two row
 groups per CTA column), several key splits, contiguous and paged caches.
@@ -29,9 +30,9 @@ def test_verify_matches_oracle_at_the_edges(hd, hq, hkv, gamma, lens):
     from tests.gpu_case import run_case
     shape = _shape(hd, hq, hkv)
     wl = _wl(shape, len(lens), gamma, lens, seed=hd + hq)
-    run_case(wl, beta=0.4, sigma=1.0, commit_and_repeat=True, logit_tol=2e-3)
+    run_case(wl, beta=0.4, sigma=1.0, commit_and_repeat=True, logit_tol=2e-3, attn_kernel=2)
     pages = sum(-(-(n + gamma + 1) // 64) for n in lens) + len(lens) + 2
-    run_case(wl, beta=0.0, sigma=0.5, logit_tol=2e-3,
+    run_case(wl, beta=0.0, sigma=0.5, logit_tol=2e-3, attn_kernel=2,
              paged=(pages, max(-(-(max(lens) + 2 * gamma + 2) // 64) + 1, 4)))
 
 
@@ -41,4 +42,5 @@ def test_many_key_splits():
     from tests.gpu_case import run_case
     shape = _shape(64, 6, 2)
     wl = _wl(shape, 3, 5, [2500, 1999, 70], seed=5)
-    run_case(wl, beta=0.2, sigma=1.0, logit_tol=2e-3)
+    run_case(wl, beta=0.2, sigma=1.0, logit_tol=2e-3, attn_kernel=2)
+    run_case(wl, beta=0.2, sigma=1.0, logit_tol=2e-3, attn_kernel=1)   # the warp-level kernel on the same case
