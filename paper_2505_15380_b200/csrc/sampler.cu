@@ -115,15 +115,37 @@ __device__ RowStats compute_row_stats(const float* z, int V, int top_k, float to
         if ((k & mask) == prefix) atomicAdd(&sm.hist[(k >> shift) & 0xFF], 1);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        int rem = sm.k_rem, bin = 255;
-        for (; bin > 0; --bin) {
-          if (sm.hist[bin] >= rem) break;
-          rem -= sm.hist[bin];
+      if (threadIdx.x < 32) {
+        // the highest bin at which the count from the top reaches k_rem (bin 0 if none does), found
+        // by the first warp: 8 bins per lane, a suffix sum over the lanes, then a walk of 8 bins
+        const int lane = threadIdx.x, rem0 = sm.k_rem;
+        int h[8], tot = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { h[i] = sm.hist[8 * lane + i]; tot += h[i]; }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
         }
-        sm.prefix = prefix | ((uint32_t)bin << shift);
-        sm.k_rem = rem;
-        sm.eq_count = sm.hist[bin];
+        const int above = incl - tot;  // in the bins of the higher lanes
+        const bool mine = above < rem0 && above + tot >= rem0;
+        const unsigned bal = __ballot_sync(0xffffffffu, mine);
+        if (bal == 0u ? lane == 0 : mine) {
+          int run = above, bin = 8 * lane;  // no crossing: bin 0, everything above it counted
+          if (bal == 0u) {
+            run = incl - h[0];
+          } else {
+#pragma unroll
+            for (int i = 7; i >= 0; --i) {
+              if (run + h[i] >= rem0) { bin = 8 * lane + i; break; }
+              run += h[i];
+            }
+          }
+          sm.prefix = prefix | ((uint32_t)bin << shift);
+          sm.k_rem = rem0 - run;
+          sm.eq_count = sm.hist[bin];
+        }
       }
       __syncthreads();
     }
@@ -168,16 +190,39 @@ __device__ RowStats compute_row_stats(const float* z, int V, int top_k, float to
         }
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        unsigned long long acc = sm.mass_above;
-        int bin = 255;
-        for (; bin > 0; --bin) {
-          if (acc + sm.hist_fx[bin] >= target) break;
-          acc += sm.hist_fx[bin];
+      if (threadIdx.x < 32) {
+        // the highest bin at which the mass from the top reaches the target (bin 0 if none does):
+        // the same walk as for the counts, on the mass histogram
+        const int lane = threadIdx.x;
+        const unsigned long long base = sm.mass_above;
+        unsigned long long h[8], tot = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { h[i] = sm.hist_fx[8 * lane + i]; tot += h[i]; }
+        unsigned long long incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned long long v = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += v;
         }
-        sm.prefix = prefix | ((uint32_t)bin << shift);
-        sm.mass_above = acc;
-        sm.eq_count = sm.hist[bin];
+        const unsigned long long above = base + (incl - tot);
+        const bool mine = above < target && above + tot >= target;
+        const unsigned bal = __ballot_sync(0xffffffffu, mine);
+        if (bal == 0u ? lane == 0 : mine) {
+          unsigned long long run = above;
+          int bin = 8 * lane;
+          if (bal == 0u) {
+            run = base + (incl - h[0]);
+          } else {
+#pragma unroll
+            for (int i = 7; i >= 0; --i) {
+              if (run + h[i] >= target) { bin = 8 * lane + i; break; }
+              run += h[i];
+            }
+          }
+          sm.prefix = prefix | ((uint32_t)bin << shift);
+          sm.mass_above = run;
+          sm.eq_count = sm.hist[bin];
+        }
       }
       __syncthreads();
     }
