@@ -3,26 +3,29 @@
 // sizes 64 and 128 and forwards of more than 16 rows.
 //
 // Grid (key split, kv head x row group, stream), one CTA = up to 64 of the G * R query rows that
-// share a kv head, over one range of keys, in tiles of 128 keys.  Both contractions are
+// share a kv head, over one range of keys, in tiles of 64 keys; two CTAs fit an SM, so that the
+// row work of one overlaps the instructions of the other.  Both contractions are
 // tcgen05.mma 128 x N x 16 with the accumulators in tensor memory:
 //
 //   S[row, key] = sum_d q[row, d] k[key, d]     A = q, rows 0..63 the bf16 leading parts, rows
 //                                               64..127 the remainders of the same rows (one
 //                                               instruction multiplies both; the two halves of S
-//                                               are added by the softmax threads); B = the K tile
+//                                               are added by the row threads); B = the K tile
 //   O[row, d]  += sum_key p[row, key] v[key, d] A = p, split and stacked the same way; B = the V
 //                                               tile transposed (keys contiguous)
 //
 // Operands sit in shared memory in the canonical K-major layout without swizzle (tc.h): byte
-// (k / 8) * rows * 16 + row * 16 + (k % 8) * 2.  K arrives by 16-byte async copies straight into
-// that layout (double buffered); V arrives row by row and is transposed by the row threads.
-// Threads 0..127 own one tensor-memory lane each (lane = row of S and O): the threads of the
-// remainder rows hand their half of S to the threads of the leading rows through shared memory,
-// those apply mask, running max and sum, and write p as the next operand; when a running max
-// grows, every thread rescales its row of O in tensor memory.  Warp 4 issues the instructions:
-// the O contraction of tile t and the S contraction of tile t + 1 alternately (instructions that
+// (k / 8) * rows * 16 + row * 16 + (k % 8) * 2.  A copy warp brings K by 16-byte async copies
+// straight into that layout and V row by row; the row threads transpose V with transposing
+// matrix loads.  Threads 0..127 own one tensor-memory lane each (lane r: leading parts of row r,
+// lane r + 64: its remainders).  The two threads of a row split the tile's columns, pass each
+// other the half of S they do not keep through shared memory (in the place of the raw V tile),
+// apply mask, running max and sum, and write p as the next operand; when a running max grows,
+// every thread rescales its lane of O in tensor memory.  Warp 4 issues the instructions: the O
+// contraction of tile t and the S contraction of tile t + 1 alternately (instructions that
 // follow one another into the same accumulator wait for each other, measured ~280 against ~165
-// cycles), one commit for both.
+// cycles); a first commit tells the row threads that O is up to date while S is still being
+// computed, so that they transpose the next V tile meanwhile.
 //
 // The un-normalised partial (O, max, sum) of each (row, head, split) goes to global memory in the
 // format of the warp-level kernel (tc_attention.cu), whose merge kernel finishes the job.
@@ -130,6 +133,7 @@ __device__ __forceinline__ void row_sync() { asm volatile("bar.sync 1, 128;" :::
 
 struct T5Shared {
   unsigned long long mma_done;  // completes when the instructions of one issue round have finished
+  unsigned long long o_done;    // completes earlier in the round: when its O += p V part has finished
   unsigned long long k_full, v_full;  // the copy warp's K / V tile has landed
   unsigned long long v_free;    // the row threads are done with the raw V tile and the exchange area
   uint32_t tmem_base;
@@ -189,6 +193,7 @@ tc_attn5_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_laye
 
   if (tid == 0) {
     mbar_init(smem_u32(&S.mma_done), 1);
+    mbar_init(smem_u32(&S.o_done), 1);
     mbar_init(smem_u32(&S.k_full), 32);
     mbar_init(smem_u32(&S.v_full), 32);
     mbar_init(smem_u32(&S.v_free), 1);
@@ -206,7 +211,7 @@ tc_attn5_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_laye
   const uint32_t tmem = S.tmem_base;
   const uint32_t t_s = tmem, t_o = tmem + T5_TILE;  // columns of S and of O
   volatile int* abort = &S.abort;
-  const uint32_t bar = smem_u32(&S.mma_done), bar_k = smem_u32(&S.k_full), bar_v = smem_u32(&S.v_full),
+  const uint32_t bar = smem_u32(&S.mma_done), bar_o = smem_u32(&S.o_done), bar_k = smem_u32(&S.k_full), bar_v = smem_u32(&S.v_full),
                  bar_vf = smem_u32(&S.v_free);
 
   // ---- row threads' view: threads r and r + 64 (r < 64) share query row i = rg * 64 + r.  Lane r
@@ -308,10 +313,9 @@ tc_attn5_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_laye
     for (int t = 0; t < n_tiles; ++t) {
       const int key0 = k_begin + t * T5_TILE;
       if (warp < 4) {
-        // round t has finished: S(t) is complete and, for t > 0, O includes tile t - 1, so the
-        // transposed V and p of that tile may be overwritten
-        if (!mbar_wait(bar, (uint32_t)t & 1u, abort)) S.abort = 1;
-        t5_fence_after();
+        // O includes tile t - 1 (the first part of round t): the transposed V and p of that tile
+        // may be overwritten.  The rest of the round, S(t), finishes while V(t) is transposed.
+        if (t > 0 && !mbar_wait(bar_o, (uint32_t)(t - 1) & 1u, abort)) S.abort = 1;
         if (!mbar_wait(bar_v, (uint32_t)t & 1u, abort)) S.abort = 1;  // V(t) has landed
         // V(t): [key][d] -> [key / 8][d][key % 8] with transposing matrix loads: an 8 x 8 block
         // (8 keys x 8 d) comes back with thread T holding keys 2 (T % 4), + 1 of d = T / 4, one
@@ -328,6 +332,8 @@ tc_attn5_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_laye
           *reinterpret_cast<uint32_t*>(dst + 16 * 16) = w2;
           *reinterpret_cast<uint32_t*>(dst + 24 * 16) = w3;
         }
+        if (!mbar_wait(bar, (uint32_t)t & 1u, abort)) S.abort = 1;  // round t has finished: S(t) is complete
+        t5_fence_after();
         row_sync();  // the raw tile is dead: its place becomes the exchange area
         // Every thread reads its lane's columns of S: the half it keeps stays in registers, the
         // other half goes to the partner (thread r gives the upper columns, thread r + 64 the lower).
@@ -445,6 +451,7 @@ tc_attn5_kernel(const float* __restrict__ qrot, const bf16* __restrict__ kv_laye
             umma_bf16(t_s, umma_desc(smem_u32(Qs) + s * 4096, 2048u, 128u),
                       umma_desc(smem_u32(Ks) + s * (2 * T5_TILE * 16), (uint32_t)T5_TILE * 16u, 128u),
                       umma_idesc(T5_TILE), s > 0 ? 1u : 0u);
+          if (s == NPV - 1) umma_commit(bar_o);  // everything issued so far, the whole O part among it
         }
         umma_commit(bar);
       }
