@@ -1057,10 +1057,22 @@ namespace {
 // ssd_verify's body; `probs_ready` (may be null) is an event the acceptance kernel waits for: the
 // host-buffer entry uploads the draft rows on a side stream while the forward, which does not
 // read them, is already running.
+// The draft rows of the host-buffer entry: an upload on a side stream that is enqueued only after
+// the forward has been launched (the forward does not read them, and every call made before its
+// launch delays its start), and that the acceptance kernel then waits for.
+struct ProbsUpload {
+  cudaStream_t side;
+  const void* host_src;
+  void* dev_dst;
+  size_t bytes;
+  cudaEvent_t dst_free;  // already recorded on the main stream: earlier readers of dev_dst are done
+  cudaEvent_t ready;
+};
+
 int verify_impl(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_tokens,
                 const float* dev_draft_probs, const float* dev_uniforms, const ssd_verify_params* params,
                 int32_t* dev_accepted_len, int32_t* dev_next_token, float* dev_logits_or_null,
-                cudaStream_t st, cudaEvent_t probs_ready) {
+                cudaStream_t st, const ProbsUpload* upload) {
   const int gamma = params->gamma;
   float* logits = dev_logits_or_null ? dev_logits_or_null : s->logits;
   const RowMap rm{0, s->B, gamma + 1};
@@ -1072,7 +1084,12 @@ int verify_impl(ssd_model* target, ssd_streams* s, const int32_t* dev_draft_toke
     rc = forward(target, s, rm, logits, st);
   }
   if (rc != SSD_OK) return rc;
-  if (probs_ready) SSD_CUDA(cudaStreamWaitEvent(st, probs_ready, 0));
+  if (upload) {
+    SSD_CUDA(cudaStreamWaitEvent(upload->side, upload->dst_free, 0));
+    SSD_CUDA(cudaMemcpyAsync(upload->dev_dst, upload->host_src, upload->bytes, cudaMemcpyHostToDevice, upload->side));
+    SSD_CUDA(cudaEventRecord(upload->ready, upload->side));
+    SSD_CUDA(cudaStreamWaitEvent(st, upload->ready, 0));
+  }
   SSD_CUDA(launch_verify_sampler(logits, target->cfg.vocab_out, dev_draft_tokens, dev_draft_probs,
                                  dev_uniforms, s->B, gamma, 1.0f / params->temperature,
                                  params->top_k, params->top_p, params->beta, params->ras_window, params->ras_tau,
@@ -1132,19 +1149,16 @@ int ssd_verify_host(ssd_model* target, ssd_streams* s, const int32_t* host_draft
     SSD_CUDA(cudaHostAlloc((void**)&s->h_stage, s->h_stage_in + 2 * B * 4, cudaHostAllocDefault));
   }
   // The draft rows are by far the largest input and only the acceptance kernel reads them: they
-  // travel on the side stream (after whatever still reads the staging buffer on `stream`) while
-  // the small inputs go ahead and the forward starts.
+  // travel on the side stream (after whatever still reads the staging buffer on `stream`), and
+  // that copy is enqueued once the forward has been launched; the small inputs go ahead.
   SSD_CUDA(cudaEventRecord(s->ev_free, st));
-  SSD_CUDA(cudaStreamWaitEvent(s->copy_stream, s->ev_free, 0));
-  SSD_CUDA(cudaMemcpyAsync(s->st_probs, host_draft_probs, B * g * V * 4, cudaMemcpyHostToDevice, s->copy_stream));
-  SSD_CUDA(cudaEventRecord(s->ev_probs, s->copy_stream));
+  const ProbsUpload upload{s->copy_stream, host_draft_probs, s->st_probs, B * g * V * 4, s->ev_free, s->ev_probs};
   // tokens and uniforms: gathered in the pinned staging buffer (a few hundred bytes), one copy
   const size_t uni_off = (size_t)((char*)s->st_uni - (char*)s->st_tokens), uni_bytes = B * (g + 1) * 2 * 4;
   memcpy(s->h_stage, host_draft_tokens, B * g * 4);
   memcpy(s->h_stage + uni_off, host_uniforms, uni_bytes);
   SSD_CUDA(cudaMemcpyAsync(s->st_tokens, s->h_stage, uni_off + uni_bytes, cudaMemcpyHostToDevice, st));
-  rc = verify_impl(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr, st,
-                   s->ev_probs);
+  rc = verify_impl(target, s, s->st_tokens, s->st_probs, s->st_uni, params, s->st_k, s->st_y, nullptr, st, &upload);
   if (rc != SSD_OK) return rc;
   rc = ssd_kv_commit(s, s->st_k, s->st_y, stream);
   if (rc != SSD_OK) return rc;
