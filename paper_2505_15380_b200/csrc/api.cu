@@ -223,8 +223,10 @@ WsPlan plan_ws(const ssd_model_config& c, int B, int max_gamma, int cap, int n_p
     const int rows[3] = {(int)(qd + 2 * kvd), (int)d, (int)d}, ks[3] = {(int)d, (int)qd, (int)F};
     for (int i = 0; i < 3; ++i) {
       const size_t tiles = (rows[i] + TC_TILE_ROWS - 1) / TC_TILE_ROWS;
-      const size_t b = (size_t)tc_ksplit(rows[i], ks[i], n_sm) * Mpad * tiles * TC_TILE_ROWS * 4;
-      part = b > part ? b : part;
+      for (int mp = 16; mp <= Mpad; mp += 16) {  // the K split depends on the rows of the forward
+        const size_t b = (size_t)tc_ksplit(rows[i], ks[i], mp, n_sm) * mp * tiles * TC_TILE_ROWS * 4;
+        part = b > part ? b : part;
+      }
     }
     p.tc_part = take(part);
   }
@@ -331,7 +333,7 @@ int forward_tc(const ssd_model* m, ssd_streams* s, RowMap rm, float* logits_out,
   const int qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim, F = c.d_ffn, nq = qd + 2 * kvd;
   const int n_sm = m->tc.n_sm;
   auto ld_of = [](int rows) { return (rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS * TC_TILE_ROWS; };
-  const int ks_qkv = tc_ksplit(nq, d, n_sm), ks_o = tc_ksplit(d, qd, n_sm), ks_d = tc_ksplit(d, F, n_sm);
+  const int ks_qkv = tc_ksplit(nq, d, M, n_sm), ks_o = tc_ksplit(d, qd, M, n_sm), ks_d = tc_ksplit(d, F, M, n_sm);
   // key splits of the attention: whole 64-key tiles, and no more CTAs in all than the SMs hold
   // at once (a second, partly filled wave would cost as much as the first)
   const int G = c.n_q_heads / c.n_kv_heads, rowgroups = (G * rm.R + 63) / 64;

@@ -128,12 +128,21 @@ __host__ __device__
 inline size_t tc_act_col_off(int Mc, int k) {
   return (size_t)(k >> 4) * ((size_t)Mc * 64) + (size_t)((k >> 3) & 1) * ((size_t)Mc * 32) + (size_t)(k & 7) * 2;
 }
-// K slices for a projection of n_rows x K on n_sm SMs: enough CTAs to occupy the GPU, at least
-// four k-steps each.  (With more than 256 token rows a CTA owns two tiles of one row chunk, and
-// there are at least two chunks: the grid is no smaller than one CTA per tile.)
-inline int tc_ksplit(int n_rows, int K, int n_sm) {
+// Weight-row tiles per CTA: two where the token rows come in chunks (more than 256 rows) and the
+// projection is long (many tiles, or a deep K): the tiles then share the activation blocks the
+// CTA loads.  A short projection keeps one tile per CTA, which doubles its CTAs per K slice, so
+// that half as many slices - and half the partial sums, whose stores and re-reads are what such
+// a projection mostly costs - occupy the GPU.
+inline int tc_tiles_per_cta(int n_rows, int K, int M) {
+  const int tiles = (n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS;
+  return tc_chunks(M).n > 1 && (tiles >= 64 || K > 4096) ? 2 : 1;
+}
+// K slices for a projection of n_rows x K over M token rows on n_sm SMs: enough CTAs to occupy
+// the GPU, at least four k-steps each.
+inline int tc_ksplit(int n_rows, int K, int M, int n_sm) {
   const int tiles = (n_rows + TC_TILE_ROWS - 1) / TC_TILE_ROWS, ks = (K + 15) / 16;
-  int s = n_sm / tiles;
+  const int ntile = tc_tiles_per_cta(n_rows, K, M);
+  int s = n_sm / ((tiles + ntile - 1) / ntile * tc_chunks(M).n);
   if (s > ks / 4) s = ks / 4;
   return s < 1 ? 1 : s;
 }

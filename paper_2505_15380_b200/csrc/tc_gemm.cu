@@ -450,7 +450,7 @@ cudaError_t launch_tc_gemm(const TcGemm& g, cudaStream_t st) {
   // and what a CTA keeps in flight is what it gets.
   const TcChunks ch = tc_chunks(g.M);
   p.Mc = ch.rows;
-  p.ntile = ch.n > 1 ? 2 : 1;
+  p.ntile = tc_tiles_per_cta(g.n_rows, g.K, g.M);
   const int grid_x = (tiles + p.ntile - 1) / p.ntile;
   const size_t per_ks = (size_t)p.ntile * TC_WBLOCK + (size_t)p.Mc * 64;
   int n_sm = 148;
