@@ -49,7 +49,7 @@ namespace ssd {
 constexpr int TC_TILE_ROWS = 128;                 // weight rows per tile = M of the MMA
 constexpr int TC_WBLOCK = TC_TILE_ROWS * 16 * 2;  // bytes of one (tile, k-step) weight block
 constexpr int TC_MAX_ROWS = 512;                  // token rows per forward (tensor-memory columns)
-constexpr int TC_THREADS = 192;                   // copy warp, MMA warp, four epilogue warps
+constexpr int TC_THREADS = 256;                   // copy warp, MMA warp, six more; all eight run the epilogue
 
 enum TcEpilogue {
   TC_EPI_PARTIAL = 0,  // part[split][token][row] = acc                (summed by the consumer)

@@ -11,8 +11,9 @@
 // activations (up to 256 rows: 128 x 2 Mpad x 16), or one per part and tile (128 x Mc x 16), bf16 x
 // bf16 -> fp32, reading both operands straight from shared memory; a tcgen05.commit hands
 // the stage back to the copy warp through its "empty" barrier, a last one tells the epilogue
-// warps that the accumulator is complete.  Warps 2..5 read the accumulator, 32 lanes x 32 columns
-// at a time (lane = weight row, column = token), and apply the epilogue.
+// warps that the accumulator is complete.  Then all eight warps (two per quarter of the tensor-memory
+// lanes) read the accumulator, 32 lanes x 32 columns at a time (lane = weight row, column = token),
+// and apply the epilogue.
 //
 // Every wait is bounded: when one runs out the CTA raises SSD_STATUS_TIMEOUT, stops issuing, waits
 // (bounded again) for the copies it has in flight, frees its tensor memory and returns.
@@ -291,16 +292,20 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
       }
       umma_commit(smem_u32(&S.accum));       // also in the abort path: dealloc waits for it below
     }
-  } else {
-    // ---- epilogue: warp w may read the 32 tensor-memory lanes of quarter w % 4
-    const int q = warp & 3, row = q * 32 + lane;
+  }
+  {
+    // ---- epilogue, by all eight warps (the copy and the issuing warp have finished their parts):
+    // warp w may read the 32 tensor-memory lanes of quarter w % 4, so each quarter has two warps,
+    // which take the 32-column ranges alternately
+    __syncwarp();
+    const int q = warp & 3, sub = warp >> 2, row = q * 32 + lane;
     const bool ok = mbar_wait(smem_u32(&S.accum), 0u, abort);
     tc_fence_after();
     if (ok && !*abort) {
      for (int u = 0; u < ntile; ++u) {
       const int tile = tile0 + u, n = tile * TC_TILE_ROWS + row;
       const uint32_t cb = (uint32_t)(u * P.Mc);  // the tile's accumulator columns (two-tile CTAs)
-      for (int c0 = 0; c0 < rows_here; c0 += 32) {
+      for (int c0 = sub * 32; c0 < rows_here; c0 += 64) {
         uint32_t v[32];
         tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + cb + (uint32_t)c0, v);
         if (P.wide) {  // add the remainder part's products
@@ -336,7 +341,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_gemm_kernel(const __grid_consta
           // global memory sees whole 16-byte rows, 512 contiguous bytes per warp store, instead
           // of two-byte pieces (measured: the epilogue of a 448-row tile 41 -> 6 us).
           const int j0 = (tile * TC_TILE_ROWS + q * 32) >> 1, jl = lane >> 1, odd = lane & 1;
-          uint8_t* stg = smem + (size_t)(warp - 2) * (4 * TC_STG_STRIDE);
+          uint8_t* stg = smem + (size_t)warp * (4 * TC_STG_STRIDE);
           const uint32_t my = (uint32_t)((jl >> 3) * 2) * TC_STG_STRIDE + (uint32_t)(jl & 7) * 2u;
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
