@@ -74,6 +74,7 @@ def test_null_and_alignment_errors_without_touching_a_device(L):
     assert L.ssd_verify(None, None, None, None, None, None, None, None, None, None) == -1
     assert L.ssd_draft_step(None, None, None, 1, None, None, None, None, None) == -1
     assert L.ssd_kv_commit(None, None, None, None) == -1
+    assert L.ssd_streams_set_attention_kernel(None, 0) == -1 and L.ssd_streams_set_path(None, 0) == -1
     assert L.ssd_strerror(0) == b"ok" and b"gamma" in L.ssd_strerror(-3)
     assert L.ssd_strerror(-99) == b"unknown error"
 
